@@ -1,0 +1,173 @@
+/*
+ * strads.h -- C ABI of the B200 scheduled-Lasso library (libstrads_b200.so).
+ *
+ * One scheduled round of parallel coordinate descent for the Lasso, after
+ * Lee, Kim, Ho, Gibson, Xing, "Structure-Aware Dynamic Scheduler for Parallel
+ * Machine Learning" (Section 2, SAP steps 1-4; Section 2.1, Algorithm 1, Eq. 1,
+ * Eq. 2; Section 4, Theorem 1 for the sampling weight).
+ *
+ * Notation (the paper's): X is N x J with standardised columns x_j, y has N
+ * entries, beta has J; P' candidates are drawn per round (n_candidates), at
+ * most P of them are updated in parallel (n_keep); eta, rho, lambda as in
+ * Algorithm 1; delta_j = |beta_j^(t_j-1) - beta_j^(t_j-2)| is the stored last
+ * change of coefficient j and starts at the "very large constant" C (c_init).
+ *
+ * Conventions for every call
+ *   - plain C, no exceptions; returns STRADS_OK (0) or a negative strads_status_t;
+ *   - "device" pointers are CUDA device addresses on the device that was current
+ *     at strads_lasso_init; "host" pointers are ordinary host addresses;
+ *   - every array is allocated, owned and freed by the caller; the handle owns
+ *     only host bookkeeping.  X and y are never written and must outlive the
+ *     handle, as must beta, resid, delta and the workspace;
+ *   - the library allocates no device memory;
+ *   - arguments are validated on the host before anything is launched; nothing
+ *     traps, aborts or waits without a bound;
+ *   - calls are asynchronous on the configured stream unless stated otherwise;
+ *   - one handle <-> one stream <-> one host thread at a time;
+ *   - same inputs, seed and round index give bit-identical outputs (no
+ *     floating-point atomics anywhere).
+ */
+#ifndef STRADS_H_
+#define STRADS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct strads_lasso_s* strads_handle_t;   /* opaque host object */
+
+typedef enum {
+  STRADS_OK = 0,
+  STRADS_ERR_INVALID_ARG = -1,          /* NULL / out-of-range / misaligned argument          */
+  STRADS_ERR_BAD_LAYOUT = -2,           /* unknown layout, ld too small or not a multiple of 4 */
+  STRADS_ERR_WORKSPACE_TOO_SMALL = -3,
+  STRADS_ERR_CUDA = -4,                 /* a CUDA runtime call failed (see strads_last_cuda_error) */
+  STRADS_ERR_NUMERIC = -5,              /* NaN / Inf met by a kernel (from strads_status)      */
+  STRADS_ERR_TIMEOUT = -6,              /* a bounded device-side wait expired                  */
+  STRADS_ERR_UNSUPPORTED = -7           /* size beyond a documented limit                      */
+} strads_status_t;
+
+typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
+
+/* flags */
+#define STRADS_FLAG_NONE          0u
+#define STRADS_FLAG_UNIFORM_DRAW  1u   /* p(j) uniform instead of delta_j^2 + eta (the random
+                                          scheduler the paper compares with, Section 5.1)      */
+#define STRADS_FLAG_NO_FILTER     2u   /* skip the rho test: keep the first P candidates       */
+
+/* limits */
+#define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (one CTA sorts the winners in shared memory) */
+
+typedef struct {
+  int32_t  layout;                      /* strads_layout_t                                          */
+  int64_t  n_rows, n_cols;              /* N, J;  1 <= N,  1 <= J < 2^31                            */
+  int64_t  nnz;                         /* CSC: number of stored entries; dense: ignored            */
+  int64_t  ld;                          /* dense: floats between column starts, ld >= N, ld % 4 == 0 */
+  const float*   x_values;              /* device, 16-byte aligned. dense: [J][ld]; CSC: [nnz]      */
+  const int32_t* x_row_idx;             /* device, CSC: [nnz], strictly ascending inside a column   */
+  const int64_t* x_col_ptr;             /* device, CSC: [J+1], col_ptr[0] = 0, col_ptr[J] = nnz     */
+  const float*   y;                     /* device [N], 16-byte aligned                              */
+  float*   beta;                        /* device [J]; in: beta^(0) (normally 0); out: current beta */
+  float*   resid;                       /* device [N], 16-byte aligned; written by init: y - X beta */
+  float*   delta;                       /* device [J], 16-byte aligned; written by init: c_init     */
+  float    lambda;                      /* > = 0                                                    */
+  float    eta;                         /* > 0   (paper: 1e-6 in the experiments)                   */
+  float    rho;                         /* > 0   (paper: 0.1)                                       */
+  float    c_init;                      /* > 0, Algorithm 1's "very large" C; 1e4 recommended       */
+  int32_t  n_candidates;                /* P': 1 <= P' <= min(J, STRADS_MAX_CANDIDATES)             */
+  int32_t  n_keep;                      /* P : 1 <= P <= P'                                         */
+  uint64_t seed;                        /* Philox key                                               */
+  void*    workspace;                   /* device, 256-byte aligned, strads_workspace_bytes() long  */
+  size_t   workspace_bytes;
+  void*    stream;                      /* cudaStream_t (NULL = legacy default stream)              */
+  uint32_t flags;
+} strads_lasso_config_t;
+
+/* Optional per-round outputs; every pointer is a DEVICE address or NULL (= not wanted). */
+typedef struct {
+  int32_t* cand;      /* [P'] candidates, best first (SAP step 1)                         */
+  int32_t* kept;      /* [P]  coefficients that passed the rho test, in walk order; -1 after n_kept */
+  float*   dbeta;     /* [P]  signed change beta_j^(t_j) - beta_j^(t_j - 1) per kept entry; 0 after n_kept */
+  int32_t* counts;    /* [4]  n_candidates, n_examined, n_kept, n_nonzero_changes          */
+  float*   gram;      /* [P'*P'] x_a^T x_b of all candidate pairs in candidate order;
+                         (debug aid: costs 4 P'^2 bytes of traffic per round)               */
+} strads_round_out_t;
+
+/* Bytes of device workspace that `cfg` needs (pointer fields of cfg are not read). */
+int strads_workspace_bytes(const strads_lasso_config_t* cfg, size_t* out_bytes);
+
+/* Algorithm 1's initialisation: n_j = ||x_j||^2 for all j, resid = y - X beta, delta_j = C,
+ * round index t = 0.  Validates cfg, creates the handle.  Asynchronous. */
+int strads_lasso_init(const strads_lasso_config_t* cfg, strads_handle_t* out_handle);
+
+/* One whole round of Algorithm 1's loop body (SAP steps 1, 2, 4; step 3 is "block size one"
+ * for the Lasso, Section 2.1):
+ *   1. draw P' candidates without replacement with p(j) ~ delta_j^2 + eta
+ *      (Philox4x32-10 word of (seed, t, j); exponential race; best first);
+ *   2. walk them best first and keep a candidate when its |correlation| with every candidate
+ *      kept before is < rho; stop at P kept;
+ *   3. for all kept j, from the same pre-round residual r:
+ *        g_j = x_j^T r,  beta_j' = S(beta_j + g_j / n_j, lambda / n_j)     (Eq. 2)
+ *      then beta_j <- beta_j', delta_j <- |beta_j' - beta_j|, r <- r - sum_j x_j (beta_j' - beta_j);
+ *   4. t <- t + 1.
+ * `out` may be NULL.  Asynchronous. */
+int strads_round(strads_handle_t h, const strads_round_out_t* out);
+
+/* n_rounds rounds back to back with no host synchronisation in between. */
+int strads_run(strads_handle_t h, int64_t n_rounds);
+
+/* The same round as strads_round for callers whose state lives in HOST memory: copies
+ * beta[J], resid[N], delta[J] host->device, runs one round, copies them back together with
+ * the optional host outputs (kept [P], dbeta [P], counts [4]; NULL = not wanted), and waits
+ * for the stream.  Host buffers should be pinned for the copies to be asynchronous. */
+int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, float* delta_host,
+                      int32_t* kept_host, float* dbeta_host, int32_t* counts_host);
+
+/* Eq. 1 with squared loss from the maintained residual: F = 1/2 ||r||^2 + lambda ||beta||_1,
+ * accumulated in FP64.  Synchronises the stream. */
+int strads_objective(strads_handle_t h, double* host_out);
+
+/* Split-phase entry points (each is one step of the round, for step-by-step checking).
+ * strads_sample : SAP step 1 for the current (delta, seed, t); cand_dev [P'] device.
+ * strads_filter : SAP step 2 on a caller-supplied ordered candidate list (device, n_cand <= P');
+ *                 kept_dev [P] device, counts_dev [4] device (as strads_round_out_t.counts).
+ * strads_update : Eq. 2 + residual + delta refresh for a caller-supplied kept list (device; may be NULL when n_kept is 0;
+ *                 distinct indices, n_kept <= P); dbeta_dev [P] device or NULL.
+ * None of them advances the round index. */
+int strads_sample(strads_handle_t h, int32_t* cand_dev);
+int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand,
+                  int32_t* kept_dev, int32_t* counts_dev, float* gram_dev_or_null);
+int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, float* dbeta_dev);
+
+/* Round index t (0-based; the Philox counter).  With beta, resid, delta and the seed it is the
+ * whole resumable state. */
+int strads_get_round(strads_handle_t h, int64_t* t_host_out);
+int strads_set_round(strads_handle_t h, int64_t t);
+
+/* Cumulative counters since init: totals[0] rounds, [1] candidates examined, [2] coefficients
+ * updated (sum of n_kept), [3] non-zero changes.  Synchronises the stream. */
+int strads_totals(strads_handle_t h, int64_t* totals_host_out /* [4] */);
+
+/* Reads the device status word (synchronises).  *bits_host_out receives the raw bits;
+ * the return value is STRADS_OK, STRADS_ERR_NUMERIC or STRADS_ERR_TIMEOUT. */
+#define STRADS_STATUS_SAMPLER_REFINED 1u   /* informational: the sampler needed extra select passes */
+#define STRADS_STATUS_NONFINITE       2u   /* a gradient x_j^T r was NaN or Inf                     */
+#define STRADS_STATUS_WAIT_EXPIRED    4u   /* a bounded wait in a kernel gave up                     */
+int strads_status(strads_handle_t h, uint32_t* bits_host_out);
+
+/* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */
+int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);
+
+int strads_destroy(strads_handle_t h);
+
+const char* strads_error_string(int code);
+/* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
+const char* strads_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* STRADS_H_ */

@@ -1,0 +1,312 @@
+// C ABI of libstrads_b200.so: argument checks, workspace carve-up and the order of kernels in a round.
+// See include/strads.h for the contract of every entry point.
+#include <climits>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "strads_internal.cuh"
+
+using namespace strads;
+
+struct strads_lasso_s {
+  Problem p;
+  cudaStream_t stream;
+  int device;
+  long long round_host;     // mirrors DeviceState::round (every round adds exactly one)
+};
+
+namespace {
+
+thread_local char g_cuda_err[256] = "";
+
+int cuda_fail(cudaError_t e, const char* where) {
+  snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", where, cudaGetErrorString(e));
+  return STRADS_ERR_CUDA;
+}
+#define CK(call)                                            \
+  do {                                                      \
+    cudaError_t e__ = (call);                               \
+    if (e__ != cudaSuccess) return cuda_fail(e__, #call);   \
+  } while (0)
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
+
+struct Layout {
+  size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_dbeta, off_dbeta64,
+      off_conflict, off_dot_partial, off_dot_ticket, off_obj, total;
+  int cap_sure, cap_boundary, mask_words, dot_parts;
+};
+
+// Checks everything about cfg that does not need its pointers.
+int check_sizes(const strads_lasso_config_t* c) {
+  if (c == nullptr) return STRADS_ERR_INVALID_ARG;
+  if (c->layout != STRADS_DENSE_COLMAJOR && c->layout != STRADS_CSC) return STRADS_ERR_BAD_LAYOUT;
+  if (c->n_rows < 1 || c->n_cols < 1 || c->n_cols >= (1ll << 31) || c->n_rows >= (1ll << 31)) return STRADS_ERR_INVALID_ARG;
+  if (c->layout == STRADS_DENSE_COLMAJOR && (c->ld < c->n_rows || (c->ld & 3) != 0)) return STRADS_ERR_BAD_LAYOUT;
+  if (c->layout == STRADS_CSC && c->nnz < 0) return STRADS_ERR_INVALID_ARG;
+  if (c->n_candidates < 1 || c->n_candidates > c->n_cols) return STRADS_ERR_INVALID_ARG;
+  if (c->n_candidates > STRADS_MAX_CANDIDATES) return STRADS_ERR_UNSUPPORTED;
+  if (c->n_keep < 1 || c->n_keep > c->n_candidates) return STRADS_ERR_INVALID_ARG;
+  return STRADS_OK;
+}
+
+Layout carve(const strads_lasso_config_t* c) {
+  Layout L;
+  L.cap_sure = c->n_candidates;
+  L.cap_boundary = pow2_ceil(c->n_candidates / 2 > 2048 ? c->n_candidates / 2 : 2048);
+  L.mask_words = (c->n_candidates + 31) / 32;
+  long long parts = (1024 + c->n_keep - 1) / c->n_keep;
+  const long long max_parts = c->n_rows / 2048 > 1 ? c->n_rows / 2048 : 1;
+  if (parts > max_parts) parts = max_parts;
+  L.dot_parts = (int)parts;
+  size_t o = 0;
+  auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
+  L.off_state = take(sizeof(DeviceState));
+  L.off_n2 = take(sizeof(double) * (size_t)c->n_cols);
+  L.off_hist = take(sizeof(unsigned int) * kHistBins);
+  L.off_sure = take(sizeof(unsigned long long) * (size_t)L.cap_sure);
+  L.off_boundary = take(sizeof(unsigned long long) * (size_t)L.cap_boundary);
+  L.off_cand = take(sizeof(int) * (size_t)c->n_candidates);
+  L.off_kept = take(sizeof(int) * (size_t)c->n_keep);
+  L.off_dbeta = take(sizeof(float) * (size_t)c->n_keep);
+  L.off_dbeta64 = take(sizeof(double) * (size_t)c->n_keep);
+  L.off_conflict = take(sizeof(unsigned int) * (size_t)c->n_candidates * L.mask_words);
+  L.off_dot_partial = take(sizeof(double) * (size_t)c->n_keep * L.dot_parts);
+  L.off_dot_ticket = take(sizeof(unsigned int) * (size_t)c->n_keep);
+  L.off_obj = take(sizeof(double) * 2 * kObjBlocks);
+  L.total = o;
+  return L;
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg) {
+  const Problem& p = h->p;
+  if (!(p.flags & STRADS_FLAG_NO_FILTER)) {
+    if (p.layout == STRADS_DENSE_COLMAJOR) CK(launch_gram_dense_simt(p, cand, n_cand, gram_dbg, h->stream));
+    else CK(launch_gram_csc(p, cand, n_cand, gram_dbg, h->stream));
+  }
+  CK(launch_filter(p, cand, n_cand, p.kept, h->stream));
+  return STRADS_OK;
+}
+
+int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
+  const Problem& p = h->p;
+  CK(launch_sample(p, p.cand, h->stream));
+  int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr);
+  if (rc) return rc;
+  CK(launch_update(p, p.kept, 1, h->stream));
+  h->round_host += 1;
+  if (out != nullptr) {
+    if (out->cand) CK(cudaMemcpyAsync(out->cand, p.cand, sizeof(int) * p.n_cand, cudaMemcpyDeviceToDevice, h->stream));
+    if (out->kept || out->dbeta || out->counts) CK(launch_export(p, p.kept, out->kept, out->dbeta, out->counts, h->stream));
+  }
+  return STRADS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int strads_workspace_bytes(const strads_lasso_config_t* cfg, size_t* out_bytes) {
+  if (out_bytes == nullptr) return STRADS_ERR_INVALID_ARG;
+  const int rc = check_sizes(cfg);
+  if (rc) return rc;
+  *out_bytes = carve(cfg).total;
+  return STRADS_OK;
+}
+
+int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handle) {
+  if (out_handle == nullptr) return STRADS_ERR_INVALID_ARG;
+  *out_handle = nullptr;
+  int rc = check_sizes(c);
+  if (rc) return rc;
+  if (!c->x_values || !c->y || !c->beta || !c->resid || !c->delta || !c->workspace) return STRADS_ERR_INVALID_ARG;
+  if (c->layout == STRADS_CSC && (!c->x_row_idx || !c->x_col_ptr)) return STRADS_ERR_INVALID_ARG;
+  if (!aligned(c->x_values, 16) || !aligned(c->y, 16) || !aligned(c->resid, 16) || !aligned(c->delta, 16) ||
+      !aligned(c->beta, 4) || !aligned(c->workspace, 256))
+    return STRADS_ERR_INVALID_ARG;
+  if (!(c->lambda >= 0.f) || !(c->eta > 0.f) || !(c->rho > 0.f) || !(c->c_init > 0.f)) return STRADS_ERR_INVALID_ARG;
+  if (!std::isfinite(c->lambda) || !std::isfinite(c->eta) || !std::isfinite(c->c_init)) return STRADS_ERR_INVALID_ARG;
+  const Layout L = carve(c);
+  if (c->workspace_bytes < L.total) return STRADS_ERR_WORKSPACE_TOO_SMALL;
+
+  strads_lasso_s* h = new (std::nothrow) strads_lasso_s();
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  Problem& p = h->p;
+  p.layout = c->layout; p.N = c->n_rows; p.J = c->n_cols; p.ld = c->ld;
+  p.xv = c->x_values; p.xrow = c->x_row_idx; p.xptr = reinterpret_cast<const long long*>(c->x_col_ptr);
+  p.y = c->y; p.beta = c->beta; p.resid = c->resid; p.delta = c->delta;
+  p.lambda = c->lambda; p.eta = c->eta; p.rho = c->rho; p.c_init = c->c_init;
+  p.n_cand = c->n_candidates; p.n_keep = c->n_keep; p.seed = c->seed; p.flags = c->flags;
+  char* ws = static_cast<char*>(c->workspace);
+  p.st = reinterpret_cast<DeviceState*>(ws + L.off_state);
+  p.n2 = reinterpret_cast<double*>(ws + L.off_n2);
+  p.hist = reinterpret_cast<unsigned int*>(ws + L.off_hist);
+  p.sure = reinterpret_cast<unsigned long long*>(ws + L.off_sure);
+  p.boundary = reinterpret_cast<unsigned long long*>(ws + L.off_boundary);
+  p.cap_sure = L.cap_sure; p.cap_boundary = L.cap_boundary;
+  p.cand = reinterpret_cast<int*>(ws + L.off_cand);
+  p.kept = reinterpret_cast<int*>(ws + L.off_kept);
+  p.dbeta = reinterpret_cast<float*>(ws + L.off_dbeta);
+  p.dbeta64 = reinterpret_cast<double*>(ws + L.off_dbeta64);
+  p.conflict = reinterpret_cast<unsigned int*>(ws + L.off_conflict);
+  p.mask_words = L.mask_words;
+  p.dot_partial = reinterpret_cast<double*>(ws + L.off_dot_partial);
+  p.dot_ticket = reinterpret_cast<unsigned int*>(ws + L.off_dot_ticket);
+  p.dot_parts = L.dot_parts;
+  p.obj_partial = reinterpret_cast<double*>(ws + L.off_obj);
+  h->stream = static_cast<cudaStream_t>(c->stream);
+  h->round_host = 0;
+
+  auto fail = [&](int code) { delete h; return code; };
+  cudaError_t e = cudaGetDevice(&h->device);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
+  e = cudaDeviceGetAttribute(&p.sm_count, cudaDevAttrMultiProcessorCount, h->device);
+  if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceGetAttribute"));
+  if ((e = prepare_sample(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_sample"));
+  if ((e = prepare_filter(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_filter"));
+  if ((e = launch_init(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
+  if ((e = launch_resid_from_beta(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
+  *out_handle = h;
+  return STRADS_OK;
+}
+
+int strads_round(strads_handle_t h, const strads_round_out_t* out) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  return one_round(h, out);
+}
+
+int strads_run(strads_handle_t h, int64_t n_rounds) {
+  if (h == nullptr || n_rounds < 0) return STRADS_ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n_rounds; ++i) {
+    const int rc = one_round(h, nullptr);
+    if (rc) return rc;
+  }
+  return STRADS_OK;
+}
+
+int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, float* delta_host,
+                      int32_t* kept_host, float* dbeta_host, int32_t* counts_host) {
+  if (h == nullptr || !beta_host || !resid_host || !delta_host) return STRADS_ERR_INVALID_ARG;
+  const Problem& p = h->p;
+  CK(cudaMemcpyAsync(p.beta, beta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
+  CK(cudaMemcpyAsync(p.resid, resid_host, sizeof(float) * p.N, cudaMemcpyHostToDevice, h->stream));
+  CK(cudaMemcpyAsync(p.delta, delta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
+  const int rc = one_round(h, nullptr);
+  if (rc) return rc;
+  CK(cudaMemcpyAsync(beta_host, p.beta, sizeof(float) * p.J, cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaMemcpyAsync(resid_host, p.resid, sizeof(float) * p.N, cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaMemcpyAsync(delta_host, p.delta, sizeof(float) * p.J, cudaMemcpyDeviceToHost, h->stream));
+  if (kept_host) CK(cudaMemcpyAsync(kept_host, p.kept, sizeof(int) * p.n_keep, cudaMemcpyDeviceToHost, h->stream));
+  if (dbeta_host) CK(cudaMemcpyAsync(dbeta_host, p.dbeta, sizeof(float) * p.n_keep, cudaMemcpyDeviceToHost, h->stream));
+  if (counts_host) CK(cudaMemcpyAsync(counts_host, p.st->counts, sizeof(int) * 4, cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaStreamSynchronize(h->stream));
+  return STRADS_OK;
+}
+
+int strads_objective(strads_handle_t h, double* host_out) {
+  if (h == nullptr || host_out == nullptr) return STRADS_ERR_INVALID_ARG;
+  CK(launch_objective(h->p, h->stream));
+  CK(cudaMemcpyAsync(host_out, &h->p.st->objective, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaStreamSynchronize(h->stream));
+  return STRADS_OK;
+}
+
+int strads_sample(strads_handle_t h, int32_t* cand_dev) {
+  if (h == nullptr || cand_dev == nullptr) return STRADS_ERR_INVALID_ARG;
+  CK(launch_sample(h->p, cand_dev, h->stream));
+  return STRADS_OK;
+}
+
+int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand, int32_t* kept_dev, int32_t* counts_dev,
+                  float* gram_dev_or_null) {
+  if (h == nullptr || cand_dev == nullptr || kept_dev == nullptr) return STRADS_ERR_INVALID_ARG;
+  if (n_cand < 0 || n_cand > h->p.n_cand) return STRADS_ERR_INVALID_ARG;
+  CK(launch_set_counts(h->p, n_cand, 0, 0, h->stream));
+  const int rc = gram_and_filter(h, cand_dev, n_cand, gram_dev_or_null);
+  if (rc) return rc;
+  CK(launch_export(h->p, h->p.kept, kept_dev, nullptr, counts_dev, h->stream));
+  return STRADS_OK;
+}
+
+int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, float* dbeta_dev) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  if (n_kept < 0 || n_kept > h->p.n_keep || (n_kept > 0 && kept_dev == nullptr)) return STRADS_ERR_INVALID_ARG;
+  const Problem& p = h->p;
+  CK(launch_set_counts(p, n_kept, n_kept, n_kept, h->stream));
+  if (n_kept > 0)
+    CK(cudaMemcpyAsync(p.kept, kept_dev, sizeof(int) * n_kept, cudaMemcpyDeviceToDevice, h->stream));
+  CK(launch_update(p, p.kept, 0, h->stream));
+  if (dbeta_dev) CK(launch_export(p, p.kept, nullptr, dbeta_dev, nullptr, h->stream));
+  return STRADS_OK;
+}
+
+int strads_get_round(strads_handle_t h, int64_t* t) {
+  if (h == nullptr || t == nullptr) return STRADS_ERR_INVALID_ARG;
+  *t = h->round_host;
+  return STRADS_OK;
+}
+
+int strads_set_round(strads_handle_t h, int64_t t) {
+  if (h == nullptr || t < 0) return STRADS_ERR_INVALID_ARG;
+  h->round_host = t;
+  const unsigned long long v = (unsigned long long)t;
+  CK(cudaMemcpyAsync(&h->p.st->round, &v, sizeof(v), cudaMemcpyHostToDevice, h->stream));
+  CK(cudaStreamSynchronize(h->stream));   // `v` lives on this stack frame
+  return STRADS_OK;
+}
+
+int strads_totals(strads_handle_t h, int64_t* totals) {
+  if (h == nullptr || totals == nullptr) return STRADS_ERR_INVALID_ARG;
+  unsigned long long t[4];
+  CK(cudaMemcpyAsync(t, h->p.st->totals, sizeof(t), cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaStreamSynchronize(h->stream));
+  for (int i = 0; i < 4; ++i) totals[i] = (int64_t)t[i];
+  return STRADS_OK;
+}
+
+int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  unsigned int bits = 0;
+  CK(cudaMemcpyAsync(&bits, &h->p.st->status, sizeof(bits), cudaMemcpyDeviceToHost, h->stream));
+  CK(cudaStreamSynchronize(h->stream));
+  if (bits_host_out) *bits_host_out = bits;
+  if (bits & STRADS_STATUS_WAIT_EXPIRED) return STRADS_ERR_TIMEOUT;
+  if (bits & STRADS_STATUS_NONFINITE) return STRADS_ERR_NUMERIC;
+  return STRADS_OK;
+}
+
+int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out) {
+  if (h == nullptr || dev_ptr_out == nullptr) return STRADS_ERR_INVALID_ARG;
+  *dev_ptr_out = h->p.n2;
+  return STRADS_OK;
+}
+
+int strads_destroy(strads_handle_t h) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  cudaStreamSynchronize(h->stream);
+  delete h;
+  return STRADS_OK;
+}
+
+const char* strads_error_string(int code) {
+  switch (code) {
+    case STRADS_OK: return "ok";
+    case STRADS_ERR_INVALID_ARG: return "invalid argument";
+    case STRADS_ERR_BAD_LAYOUT: return "bad matrix layout";
+    case STRADS_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+    case STRADS_ERR_CUDA: return "CUDA runtime error";
+    case STRADS_ERR_NUMERIC: return "non-finite value met on the device";
+    case STRADS_ERR_TIMEOUT: return "bounded device wait expired";
+    case STRADS_ERR_UNSUPPORTED: return "size beyond a documented limit";
+    default: return "unknown error";
+  }
+}
+
+const char* strads_last_cuda_error(void) { return g_cuda_err; }
+
+}  // extern "C"

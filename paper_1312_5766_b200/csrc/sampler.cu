@@ -1,0 +1,229 @@
+// SAP step 1 / Algorithm 1 "draw a set U of P' coefficients from p(j)": priority sampling without
+// replacement, p(j) ~ delta_j^2 + eta (Theorem 1's weight with Algorithm 1's floor eta).
+//
+// Every coefficient gets the race key (bits of T_j) << 32 | j, T_j = E_j / w_j with E_j a unit
+// exponential made from the Philox4x32-10 word of (seed, t, j).  The P' smallest keys, in ascending
+// order, are the candidates.  They are found by a multi-CTA radix select that recomputes the keys in
+// every pass instead of storing them (one read of delta[J] per pass, no 8J-byte key array):
+//
+//   k_sample_hist    pass 1: histogram of the top 12 key bits; the last CTA to finish scans it and
+//                    publishes the boundary bin (all keys below it are winners, the bin itself holds
+//                    the rest).  For an exponential race the boundary bin holds < ~0.1 P' keys in
+//                    expectation whatever the weights are; if it ever exceeds the boundary buffer,
+//                    that CTA alone refines the boundary over further 12-bit digits (rare, exact).
+//   k_sample_collect pass 2: appends "sure" and "boundary" keys to two small buffers.
+//   k_sample_sort    one CTA: bitonic sort of both buffers in shared memory, writes cand[P'].
+#include "strads_internal.cuh"
+
+namespace strads {
+
+namespace {
+
+constexpr int kThreads = 256;
+
+// Calls f(key) for each of the (up to) four coefficients of Philox block g.
+template <typename F>
+__device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned long long t, long long g, F&& f) {
+  uint32_t w[4];
+  philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
+  const long long j0 = g * 4;
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  if (j0 + 3 < p.J) {
+    const float4 d = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
+    f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, uniform));
+    f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, uniform));
+    f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, uniform));
+    f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, uniform));
+  } else {
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      if (j0 + i < p.J) f(race_key64(p.delta[j0 + i], p.eta, w[i], (uint32_t)(j0 + i), uniform));
+  }
+}
+
+// Whole CTA (kThreads threads): the bin b with before(b) < k_rem <= before(b) + h[b], where before(b)
+// is the number of keys in bins below b.  Exactly one thread finds it and writes *bin / *before.
+__device__ void find_bin(const unsigned int* h, int nbins, long long k_rem, int* bin, long long* before) {
+  __shared__ long long warp_tot[kThreads / 32];
+  const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+  const int per = (nbins + kThreads - 1) / kThreads;
+  const int b0 = tid * per;
+  long long mine = 0;
+  for (int b = b0; b < b0 + per && b < nbins; ++b) mine += h[b];
+  long long incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const long long v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) warp_tot[wid] = incl;
+  __syncthreads();
+  long long base = 0;
+  for (int w = 0; w < wid; ++w) base += warp_tot[w];
+  incl += base;
+  const long long excl = incl - mine;
+  if (excl < k_rem && k_rem <= incl) {
+    long long cum = excl;
+    int b = b0;
+    for (; b < b0 + per - 1 && b < nbins - 1; ++b) {
+      if (cum + h[b] >= k_rem) break;
+      cum += h[b];
+    }
+    *bin = b;
+    *before = cum;
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
+  __shared__ unsigned int sh[kHistBins];
+  __shared__ int s_last;
+  __shared__ SelectState s_sel;
+  const int tid = threadIdx.x;
+  for (int b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
+  __syncthreads();
+  const unsigned long long t = p.st->round;
+  const long long groups = (p.J + 3) >> 2;
+  for (long long g = (long long)blockIdx.x * kThreads + tid; g < groups; g += (long long)gridDim.x * kThreads)
+    for_keys_of_group(p, t, g, [&](unsigned long long key) { atomicAdd(&sh[key >> (64 - kHistBits)], 1u); });
+  __syncthreads();
+  for (int b = tid; b < kHistBins; b += kThreads)
+    if (sh[b]) atomicAdd(&p.hist[b], sh[b]);
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = (atomicAdd(&p.st->hist_ticket, 1u) == gridDim.x - 1);
+  __syncthreads();
+  if (!s_last) return;
+
+  // ---- last CTA: every other CTA's histogram is visible now ----
+  __threadfence();
+  for (int b = tid; b < kHistBins; b += kThreads) {
+    sh[b] = __ldcg(&p.hist[b]);
+    p.hist[b] = 0;                                   // ready for the next round
+  }
+  __syncthreads();
+  __shared__ int s_bin;
+  __shared__ long long s_before;
+  find_bin(sh, kHistBins, p.n_cand, &s_bin, &s_before);
+  if (tid == 0) {
+    p.st->hist_ticket = 0;
+    s_sel.prefix = (unsigned long long)s_bin;
+    s_sel.bits = kHistBits;
+    s_sel.n_sure = (int)s_before;
+    s_sel.n_boundary = (int)sh[s_bin];
+  }
+  __syncthreads();
+  // Rare: the boundary bin does not fit the buffer -> refine digit by digit with this CTA alone.
+  while (s_sel.n_boundary > p.cap_boundary && s_sel.bits < 64) {
+    const int bits = s_sel.bits;
+    const int width = min(kHistBits, 64 - bits);
+    const unsigned long long prefix = s_sel.prefix;
+    __syncthreads();
+    for (int b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
+    __syncthreads();
+    for (long long g = tid; g < groups; g += kThreads)
+      for_keys_of_group(p, t, g, [&](unsigned long long key) {
+        if ((key >> (64 - bits)) == prefix)
+          atomicAdd(&sh[(key >> (64 - bits - width)) & ((1u << width) - 1u)], 1u);
+      });
+    __syncthreads();
+    find_bin(sh, 1 << width, (long long)p.n_cand - s_sel.n_sure, &s_bin, &s_before);
+    if (tid == 0) {
+      s_sel.prefix = (prefix << width) | (unsigned long long)s_bin;
+      s_sel.bits = bits + width;
+      s_sel.n_sure += (int)s_before;
+      s_sel.n_boundary = (int)sh[s_bin];
+      atomicOr(&p.st->status, STRADS_STATUS_SAMPLER_REFINED);
+    }
+    __syncthreads();
+  }
+  if (tid == 0) p.st->sel = s_sel;
+}
+
+__global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
+  const SelectState sel = p.st->sel;
+  const unsigned long long t = p.st->round;
+  const long long groups = (p.J + 3) >> 2;
+  const int shift = 64 - sel.bits;
+  for (long long g = (long long)blockIdx.x * kThreads + threadIdx.x; g < groups;
+       g += (long long)gridDim.x * kThreads)
+    for_keys_of_group(p, t, g, [&](unsigned long long key) {
+      const unsigned long long pfx = key >> shift;
+      if (pfx < sel.prefix) {
+        const unsigned int i = atomicAdd(&p.st->sure_count, 1u);
+        if (i < (unsigned)p.cap_sure) p.sure[i] = key;
+      } else if (pfx == sel.prefix) {
+        const unsigned int i = atomicAdd(&p.st->boundary_count, 1u);
+        if (i < (unsigned)p.cap_boundary) p.boundary[i] = key;
+      }
+    });
+}
+
+// Ascending bitonic sort of n (a power of two) keys in shared memory by the whole CTA.
+__device__ void bitonic_sort(unsigned long long* a, int n) {
+  for (int k = 2; k <= n; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int i = threadIdx.x; i < (n >> 1); i += blockDim.x) {
+        const int lo = ((i & ~(j - 1)) << 1) | (i & (j - 1));
+        const int hi = lo | j;
+        const unsigned long long x = a[lo], y = a[hi];
+        const bool up = (lo & k) == 0;
+        if ((x > y) == up) { a[lo] = y; a[hi] = x; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+__device__ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
+
+__global__ void __launch_bounds__(1024) k_sample_sort(Problem p, int* cand_out) {
+  extern __shared__ unsigned long long keys[];
+  const SelectState sel = p.st->sel;
+  const int n_sure = min(sel.n_sure, p.cap_sure);
+  const int n_bnd = min(sel.n_boundary, p.cap_boundary);
+  const int need = p.n_cand - n_sure;              // winners taken from the boundary set
+  int n = pow2_ceil(max(n_sure, 1));
+  for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = i < n_sure ? p.sure[i] : ~0ull;
+  __syncthreads();
+  bitonic_sort(keys, n);
+  for (int i = threadIdx.x; i < n_sure; i += blockDim.x) cand_out[i] = (int)(keys[i] & 0xffffffffull);
+  __syncthreads();
+  n = pow2_ceil(max(n_bnd, 1));
+  for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = i < n_bnd ? p.boundary[i] : ~0ull;
+  __syncthreads();
+  bitonic_sort(keys, n);
+  for (int i = threadIdx.x; i < need && i < n_bnd; i += blockDim.x)
+    cand_out[n_sure + i] = (int)(keys[i] & 0xffffffffull);
+  if (threadIdx.x == 0) {
+    p.st->sure_count = 0;
+    p.st->boundary_count = 0;
+    p.st->counts[0] = p.n_cand;
+  }
+}
+
+}  // namespace
+
+static size_t sort_smem_bytes(const Problem& p) {
+  int n = 1;
+  while (n < p.cap_sure || n < p.cap_boundary) n <<= 1;
+  return (size_t)n * sizeof(unsigned long long);
+}
+
+cudaError_t prepare_sample(const Problem& p) {
+  return cudaFuncSetAttribute(k_sample_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem_bytes(p));
+}
+
+cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
+  const long long groups = (p.J + 3) >> 2;
+  long long blocks = (groups + kThreads - 1) / kThreads;
+  const long long cap = (long long)p.sm_count * 8;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  k_sample_hist<<<(unsigned)blocks, kThreads, 0, s>>>(p);
+  k_sample_collect<<<(unsigned)blocks, kThreads, 0, s>>>(p);
+  k_sample_sort<<<1, 1024, sort_smem_bytes(p), s>>>(p, cand_out);
+  return cudaGetLastError();
+}
+
+}  // namespace strads

@@ -1,0 +1,156 @@
+// Internal declarations shared by the kernels of libstrads_b200.so (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include "strads.h"
+
+namespace strads {
+
+// ---------------------------------------------------------------------------------------------
+// Device-resident state of one handle (lives at the start of the caller's workspace).
+// ---------------------------------------------------------------------------------------------
+struct SelectState {            // written by the sampler's histogram kernel, read by collect / sort
+  unsigned long long prefix;    // boundary value of the top `bits` bits of the 64-bit key
+  int bits;                     // how many top bits `prefix` covers
+  int n_sure;                   // keys whose top bits are < prefix (all of them are winners)
+  int n_boundary;               // keys whose top bits are == prefix
+  int pad;
+};
+
+struct DeviceState {
+  unsigned long long round;     // t, the Philox counter word
+  unsigned long long totals[4]; // rounds, examined, kept, nonzero
+  unsigned int status;          // STRADS_STATUS_* bits
+  unsigned int hist_ticket;     // "last block done" tickets
+  unsigned int sure_count;      // append cursors of the collect kernel
+  unsigned int boundary_count;
+  int counts[4];                // n_cand, n_examined, n_kept, n_nonzero of the current round
+  SelectState sel;
+  double objective;             // result slot of the objective reduction
+  float x_abs_max;              // max |x_ij| (CSC: bounds the fixed-point residual update)
+  int beta0_nonzero;            // set at init when the starting beta has a non-zero entry
+};
+
+static constexpr int kHistBits = 12;
+static constexpr int kHistBins = 1 << kHistBits;
+
+// Everything a launch needs; filled once at init (host copy in the handle).
+struct Problem {
+  int layout;
+  long long N, J, ld;
+  const float* xv;
+  const int* xrow;
+  const long long* xptr;
+  const float* y;
+  float* beta;
+  float* resid;
+  float* delta;
+  float lambda, eta, rho, c_init;
+  int n_cand, n_keep;
+  unsigned long long seed;
+  unsigned int flags;
+  // workspace carve-up
+  DeviceState* st;
+  double* n2;                   // [J]
+  unsigned int* hist;           // [kHistBins]
+  unsigned long long* sure;     // [cap_sure]
+  unsigned long long* boundary; // [cap_boundary]
+  int cap_sure, cap_boundary;
+  int* cand;                    // [n_cand]
+  int* kept;                    // [n_keep]
+  float* dbeta;                 // [n_keep]
+  double* dbeta64;              // [n_keep]
+  unsigned int* conflict;       // [n_cand][mask_words]
+  int mask_words;
+  double* dot_partial;          // [n_keep][dot_parts]
+  unsigned int* dot_ticket;     // [n_keep]
+  int dot_parts;
+  double* obj_partial;          // [2 * kObjBlocks]
+  int sm_count;
+};
+static constexpr int kObjBlocks = 296;
+
+// ---------------------------------------------------------------------------------------------
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) and the FP32 race key.
+// The key is a fixed sequence of correctly rounded binary32 operations (explicit _rn intrinsics,
+// never contracted), so that any IEEE implementation of the same sequence agrees bit for bit.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                              uint32_t k0, uint32_t k1, uint32_t out[4]) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+    const uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+    const uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+    c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+    k0 += 0x9E3779B9u;
+    k1 += 0xBB67AE85u;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+__device__ __forceinline__ float two_atanh_rn(float s) {
+  const float z = __fmul_rn(s, s);
+  float p = __uint_as_float(0x3d70f0f1u);                       // 1/17
+  p = __fmaf_rn(p, z, __uint_as_float(0x3d888889u));            // 1/15
+  p = __fmaf_rn(p, z, __uint_as_float(0x3d9d89d9u));            // 1/13
+  p = __fmaf_rn(p, z, __uint_as_float(0x3dba2e8cu));            // 1/11
+  p = __fmaf_rn(p, z, __uint_as_float(0x3de38e39u));            // 1/9
+  p = __fmaf_rn(p, z, __uint_as_float(0x3e124925u));            // 1/7
+  p = __fmaf_rn(p, z, __uint_as_float(0x3e4ccccdu));            // 1/5
+  p = __fmaf_rn(p, z, __uint_as_float(0x3eaaaaabu));            // 1/3
+  const float r = __fmul_rn(z, p);
+  const float s2 = __fadd_rn(s, s);
+  return __fmaf_rn(s2, r, s2);
+}
+
+// Unit exponential E = -ln(1 - v), v = (x + 1/2) / 2^32.
+__device__ __forceinline__ float unit_exponential_rn(uint32_t x) {
+  const float xf = __uint2float_rn(x);
+  float v = __fmaf_rn(xf, __uint_as_float(0x2f800000u), __uint_as_float(0x2f000000u));
+  const float vmax = __uint_as_float(0x3f7fffffu);
+  if (v > vmax) v = vmax;
+  if (v <= 0.5f) {
+    const float s = __fdiv_rn(v, __fsub_rn(2.0f, v));
+    return two_atanh_rn(s);
+  }
+  const float q = __fsub_rn(1.0f, v);
+  const uint32_t qb = __float_as_uint(q);
+  int e = (int)(qb >> 23) - 127;
+  float m = __uint_as_float((qb & 0x007fffffu) | 0x3f800000u);
+  if (m >= __uint_as_float(0x3fb504f3u)) { m = __fmul_rn(m, 0.5f); e += 1; }
+  const float s = __fdiv_rn(__fsub_rn(m, 1.0f), __fadd_rn(m, 1.0f));
+  const float a = two_atanh_rn(s);
+  const float ef = __int2float_rn(e);
+  const float lo = __fmaf_rn(ef, __uint_as_float(0x3805fdf4u), a);
+  const float lnq = __fmaf_rn(ef, __uint_as_float(0x3f317000u), lo);
+  return -lnq;
+}
+
+// 64-bit ranking key of coefficient j: (bits of T_j) << 32 | j, T_j = E_j / (delta_j^2 + eta).
+// All keys are distinct; ascending key order = ascending T, ties to the smaller j.
+__device__ __forceinline__ unsigned long long race_key64(float delta_j, float eta, uint32_t word, uint32_t j,
+                                                         bool uniform) {
+  const float w = uniform ? 1.0f : __fmaf_rn(delta_j, delta_j, eta);
+  const float T = __fdiv_rn(unit_exponential_rn(word), w);
+  return ((unsigned long long)__float_as_uint(T) << 32) | j;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Launchers (one per step; all enqueue on `s` and return a cudaError_t).
+// ---------------------------------------------------------------------------------------------
+cudaError_t launch_init(const Problem& p, cudaStream_t s);
+cudaError_t launch_resid_from_beta(const Problem& p, cudaStream_t s);
+cudaError_t launch_objective(const Problem& p, cudaStream_t s);
+cudaError_t prepare_sample(const Problem& p);
+cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
+cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
+cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
+cudaError_t prepare_filter(const Problem& p);
+cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s);
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s);
+cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s);
+cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,
+                          cudaStream_t s);
+
+}  // namespace strads

@@ -1,0 +1,259 @@
+// Algorithm 1 "in parallel on P workers: update beta_j using Eq. 2" + SAP step 4 (progress monitoring).
+//
+// With r = y - X beta, Eq. 2's argument x_j^T y - sum_{k != j} x_j^T x_k beta_k equals
+// x_j^T r + n_j beta_j, so for every kept j, all from the SAME pre-round r:
+//     g_j = x_j^T r,   beta_j' = S(beta_j + g_j / n_j, lambda / n_j),   S(a, k) = sign(a) max(|a| - k, 0)
+// then beta_j <- beta_j', delta_j <- |beta_j' - beta_j|, r <- r - sum_j x_j (beta_j' - beta_j).
+//
+// Two kernels per layout.  "dot" streams the kept columns once against r (FP64 accumulation in a fixed
+// order; the last CTA of a column sums the partials in index order and applies the soft threshold).
+// "apply" updates r with every row owned by exactly one CTA: dense rows are summed over the kept
+// columns in list order; CSC contributions are added as 64-bit fixed-point integers in shared memory
+// (integer addition is associative, so hot rows shared by thousands of columns still give the same
+// bits whatever the order) -- no floating-point atomics anywhere.
+#include <climits>
+
+#include "strads_internal.cuh"
+
+namespace strads {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// Soft threshold + bookkeeping for kept entry a (one thread).
+__device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
+  const double n = p.n2[j];
+  const float b_old = p.beta[j];
+  float b_new = b_old;
+  if (n > 0.0) {
+    const double z = (double)b_old + g / n;
+    const double m = fabs(z) - (double)p.lambda / n;
+    b_new = (float)(m <= 0.0 ? 0.0 : (z > 0.0 ? m : -m));
+  }
+  const double d = (double)b_new - (double)b_old;        // the change that beta (FP32) really makes
+  p.beta[j] = b_new;
+  p.delta[j] = (float)fabs(d);
+  p.dbeta[a] = (float)d;
+  p.dbeta64[a] = d;
+  if (d != 0.0) atomicAdd(&p.st->counts[3], 1);
+  if (!isfinite(g)) atomicOr(&p.st->status, STRADS_STATUS_NONFINITE);
+}
+
+// ------------------------------------------------------------------------------------------------
+// dense
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __restrict__ kept) {
+  const int a = blockIdx.y;
+  if (a >= p.st->counts[2]) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) p.dbeta[a] = 0.f;
+    return;
+  }
+  const int part = blockIdx.x, parts = gridDim.x;
+  const int j = kept[a];
+  const float* x = p.xv + (long long)j * p.ld;
+  const long long n4 = (p.N + 3) >> 2;                       // float4 groups (the last may be partial)
+  const long long per = (n4 + parts - 1) / parts;
+  const long long g0 = part * per, g1 = min(n4, g0 + per);
+  double acc0 = 0.0, acc1 = 0.0;
+  for (long long g = g0 + threadIdx.x; g < g1; g += kThreads) {
+    const long long i = g << 2;
+    float4 xv = __ldg(reinterpret_cast<const float4*>(x) + g);
+    float4 rv;
+    if (i + 3 < p.N) {
+      rv = *(reinterpret_cast<const float4*>(p.resid) + g);
+    } else {
+      rv.x = p.resid[i];
+      rv.y = i + 1 < p.N ? p.resid[i + 1] : 0.f;
+      rv.z = i + 2 < p.N ? p.resid[i + 2] : 0.f;
+      rv.w = 0.f;
+      if (i + 1 >= p.N) xv.y = 0.f;
+      if (i + 2 >= p.N) xv.z = 0.f;
+      xv.w = 0.f;
+    }
+    acc0 += (double)xv.x * (double)rv.x + (double)xv.z * (double)rv.z;
+    acc1 += (double)xv.y * (double)rv.y + (double)xv.w * (double)rv.w;
+  }
+  __shared__ double wsum[kThreads / 32];
+  __shared__ int s_last;
+  double v = warp_sum(acc0 + acc1);
+  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double s = 0.0;
+    for (int w = 0; w < kThreads / 32; ++w) s += wsum[w];
+    p.dot_partial[(long long)a * parts + part] = s;
+    __threadfence();
+    s_last = atomicAdd(&p.dot_ticket[a], 1u) == (unsigned)parts - 1;
+    if (s_last) {
+      __threadfence();
+      double g = 0.0;
+      for (int q = 0; q < parts; ++q) g += __ldcg(&p.dot_partial[(long long)a * parts + q]);
+      p.dot_ticket[a] = 0;
+      finish_coefficient(p, a, j, g);
+    }
+  }
+}
+
+constexpr int kRowsPerCta = 128;       // 32 lanes x float4
+
+__global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* __restrict__ kept, int advance) {
+  __shared__ double part[kThreads / 32][kRowsPerCta];
+  const int n_kept = p.st->counts[2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const long long i = (long long)blockIdx.x * kRowsPerCta + lane * 4;
+  double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
+  if (i < p.N) {
+    for (int a = warp; a < n_kept; a += kThreads / 32) {
+      const double d = p.dbeta64[a];
+      if (d == 0.0) continue;
+      const float4 xv = __ldg(reinterpret_cast<const float4*>(p.xv + (long long)kept[a] * p.ld + i));
+      s0 += (double)xv.x * d; s1 += (double)xv.y * d; s2 += (double)xv.z * d; s3 += (double)xv.w * d;
+    }
+  }
+  part[warp][lane * 4 + 0] = s0; part[warp][lane * 4 + 1] = s1;
+  part[warp][lane * 4 + 2] = s2; part[warp][lane * 4 + 3] = s3;
+  __syncthreads();
+  if (threadIdx.x < kRowsPerCta) {
+    const long long r = (long long)blockIdx.x * kRowsPerCta + threadIdx.x;
+    if (r < p.N) {
+      double s = 0.0;
+#pragma unroll
+      for (int w = 0; w < kThreads / 32; ++w) s += part[w][threadIdx.x];
+      if (s != 0.0) p.resid[r] = (float)((double)p.resid[r] - s);
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
+    DeviceState* st = p.st;
+    st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
+    st->round += 1;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// CSC
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kThreads) k_dot_csc(Problem p, const int* __restrict__ kept) {
+  const int lane = threadIdx.x & 31;
+  const int a = (blockIdx.x * kThreads + threadIdx.x) >> 5;
+  if (a >= p.n_keep) return;
+  if (a >= p.st->counts[2]) {
+    if (lane == 0) p.dbeta[a] = 0.f;
+    return;
+  }
+  const int j = kept[a];
+  double acc = 0.0;
+  for (long long q = p.xptr[j] + lane; q < p.xptr[j + 1]; q += 32)
+    acc += (double)__ldg(p.xv + q) * (double)p.resid[__ldg(p.xrow + q)];
+  acc = warp_sum(acc);
+  if (lane == 0) finish_coefficient(p, a, j, acc);
+}
+
+constexpr int kMaxRowsCsc = 4096;      // rows owned by one CTA (64-bit accumulators in shared memory)
+
+__global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, const int* __restrict__ kept, int rows_per_cta,
+                                                         int advance) {
+  __shared__ long long acc[kMaxRowsCsc];
+  __shared__ double wmax[kThreads / 32];
+  __shared__ int s_shift;
+  const int n_kept = p.st->counts[2];
+  const long long r0 = (long long)blockIdx.x * rows_per_cta;
+  const long long r1 = min(p.N, r0 + rows_per_cta);
+  // scale: every row sum is below n_kept * max|x| * max|dbeta| < 2^e, stored in units of 2^-(61 - e)
+  double dmax = 0.0;
+  for (int a = threadIdx.x; a < n_kept; a += kThreads) dmax = fmax(dmax, fabs(p.dbeta64[a]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) dmax = fmax(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = dmax;
+  for (int r = threadIdx.x; r < rows_per_cta; r += kThreads) acc[r] = 0;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double m = 0.0;
+    for (int w = 0; w < kThreads / 32; ++w) m = fmax(m, wmax[w]);
+    int e = 0;
+    if (m > 0.0 && isfinite(m)) frexp(m * (double)p.st->x_abs_max * (double)max(n_kept, 1), &e);
+    s_shift = (m > 0.0 && isfinite(m)) ? 61 - e : INT_MIN;
+  }
+  __syncthreads();
+  const int shift = s_shift;
+  if (shift != INT_MIN && r0 < p.N) {
+    for (int a = threadIdx.x; a < n_kept; a += kThreads) {
+      const double d = p.dbeta64[a];
+      if (d == 0.0) continue;
+      const int j = kept[a];
+      long long lo = p.xptr[j], hi = p.xptr[j + 1];
+      const long long end = hi;
+      while (lo < hi) {                                    // first entry with row >= r0
+        const long long mid = (lo + hi) >> 1;
+        if (__ldg(p.xrow + mid) < r0) lo = mid + 1; else hi = mid;
+      }
+      for (long long q = lo; q < end; ++q) {
+        const long long r = __ldg(p.xrow + q);
+        if (r >= r1) break;
+        const long long fx = __double2ll_rn(ldexp((double)__ldg(p.xv + q) * d, shift));
+        atomicAdd(reinterpret_cast<unsigned long long*>(&acc[r - r0]), (unsigned long long)fx);
+      }
+    }
+    __syncthreads();
+    for (long long r = r0 + threadIdx.x; r < r1; r += kThreads) {
+      const long long v = acc[r - r0];
+      if (v != 0) p.resid[r] = (float)((double)p.resid[r] - ldexp((double)v, -shift));
+    }
+  }
+  if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
+    DeviceState* st = p.st;
+    st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
+    st->round += 1;
+  }
+}
+
+__global__ void k_set_counts(Problem p, int n_cand, int n_examined, int n_kept) {
+  p.st->counts[0] = n_cand; p.st->counts[1] = n_examined; p.st->counts[2] = n_kept; p.st->counts[3] = 0;
+}
+
+__global__ void k_clear_nonzero(Problem p) { p.st->counts[3] = 0; }
+
+__global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out) {
+  const int n_kept = p.st->counts[2];
+  for (int a = blockIdx.x * blockDim.x + threadIdx.x; a < p.n_keep; a += gridDim.x * blockDim.x) {
+    if (kept_out != nullptr) kept_out[a] = a < n_kept ? kept[a] : -1;
+    if (dbeta_out != nullptr) dbeta_out[a] = a < n_kept ? p.dbeta[a] : 0.f;
+  }
+  if (counts_out != nullptr && blockIdx.x == 0 && threadIdx.x < 4) counts_out[threadIdx.x] = p.st->counts[threadIdx.x];
+}
+
+}  // namespace
+
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s) {
+  k_clear_nonzero<<<1, 1, 0, s>>>(p);
+  if (p.layout == STRADS_DENSE_COLMAJOR) {
+    k_dot_dense<<<dim3(p.dot_parts, p.n_keep), kThreads, 0, s>>>(p, kept);
+    k_apply_dense<<<(unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s>>>(p, kept, advance);
+  } else {
+    k_dot_csc<<<(p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(p, kept);
+    long long grid = (long long)p.sm_count * 2;
+    const long long need = (p.N + kMaxRowsCsc - 1) / kMaxRowsCsc;
+    if (grid < need) grid = need;
+    const int rows_per_cta = (int)((p.N + grid - 1) / grid);
+    k_apply_csc<<<(unsigned)grid, kThreads, 0, s>>>(p, kept, rows_per_cta, advance);
+  }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s) {
+  k_set_counts<<<1, 1, 0, s>>>(p, n_cand, n_examined, n_kept);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,
+                          cudaStream_t s) {
+  k_export<<<(p.n_keep + 255) / 256, 256, 0, s>>>(p, kept, kept_out, dbeta_out, counts_out);
+  return cudaGetLastError();
+}
+
+}  // namespace strads

@@ -1,0 +1,359 @@
+"""Parity of the CUDA library with the FP64 CPU oracle, element by element, through the C ABI.
+
+Three levels, as the round has three kinds of output:
+  1. candidates: bit-exact ordered lists from identical (delta, seed, t);
+  2. one round from identical (beta, r, delta): same kept list (decisions within 1e-6 of rho are
+     replayed by the oracle and must then agree), dbeta within 1e-5 relative + 1e-7 max|beta|;
+  3. free-running objective within 1e-4 relative after a fixed number of rounds.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1312_5766_b200 import workloads as wl
+from helpers import oracle_matrix
+
+pytestmark = pytest.mark.gpu
+
+RTOL_DBETA = 1e-5        # relative tolerance on a coefficient change (FP64 accumulation on both sides)
+ATOL_DBETA = 1e-7        # times max|beta|: beta is stored in FP32 on the device (2^-24 = 6e-8 rounding)
+RHO_EXCUSE = 1e-6        # |corr| this close to rho may fall either way (FP32 Gram vs FP64 oracle)
+RTOL_OBJ = 1e-4
+
+
+def _binding():
+    from paper_1312_5766_b200 import binding
+    return binding
+
+
+def _solver(p, **kw):
+    return _binding().StradsLasso.from_problem(p, device="cuda", **kw)
+
+
+# --------------------------------------------------------------------------------------------------
+# level 1: sampler
+# --------------------------------------------------------------------------------------------------
+def _delta_cases(J, rng):
+    C = 1e4
+    sweep = np.full(J, C, dtype=np.float32)
+    part = sweep.copy()
+    part[rng.random(J) < 0.7] = 0.0
+    late = (rng.random(J) < 0.05) * rng.exponential(0.05, J)
+    mixed = np.where(rng.random(J) < 0.1, C, late)
+    wide = 10.0 ** rng.uniform(-8, 3, J)
+    return {"sweep": sweep, "partial_sweep": part, "late": late.astype(np.float32),
+            "mixed": mixed.astype(np.float32), "wide": wide.astype(np.float32),
+            "zeros": np.zeros(J, dtype=np.float32)}
+
+
+@pytest.mark.parametrize("J,n_cand", [(10_000, 200), (100_000, 2048), (99_997, 1000), (1_000_003, 8192),
+                                      (37, 37), (5, 1), (4096, 4096), (2_000_001, 16384)])
+def test_candidates_bit_exact(J, n_cand):
+    rng = np.random.default_rng(J)
+    p = wl.make_problem(dict(kind="csc_uniform", n_rows=64, n_cols=J, n_true=1, lam_frac=0.1, nnz_col=2,
+                             n_candidates=n_cand, n_keep=1, rho=0.1), seed=0)
+    cases = _delta_cases(J, rng)
+    names = list(cases) if J <= 100_000 else ["sweep", "mixed", "late"]
+    for seed, t in [(0, 0), ((0xABCDEF01 << 32) | 0x2345, 7), (42, (1 << 32) + 5)]:
+        p.seed = seed
+        s = _solver(p)
+        s.set_round(t)
+        for name in names:
+            d = cases[name]
+            s.delta.copy_(torch.from_numpy(d))
+            got = s.sample().cpu().numpy()
+            want = oracle.sample(d.astype(np.float64), p.eta, seed, t, n_cand)
+            assert np.array_equal(got, want), (name, seed, t, np.flatnonzero(got != want)[:5])
+        assert s.status()[0] == 0
+        s.close()
+
+
+def test_sampler_refinement_path_is_exact():
+    # every race time is exactly 0 for the coefficients with infinite priority: one histogram bin
+    # holds far more keys than the boundary buffer, so the select must refine down to the index bits
+    J, n_cand = 200_000, 300
+    p = wl.make_problem(dict(kind="csc_uniform", n_rows=64, n_cols=J, n_true=1, lam_frac=0.1, nnz_col=2,
+                             n_candidates=n_cand, n_keep=1, rho=0.1), seed=0)
+    d = np.zeros(J, dtype=np.float32)
+    d[1000:150_000] = np.inf
+    s = _solver(p)
+    s.delta.copy_(torch.from_numpy(d))
+    got = s.sample().cpu().numpy()
+    want = oracle.sample(d.astype(np.float64), p.eta, 0, 0, n_cand)
+    assert np.array_equal(got, want) and want.tolist() == list(range(1000, 1300))
+    rc, bits = s.status()
+    assert rc == 0 and bits & 1                      # informational "refined" bit
+    # and the next ordinary draw is unaffected by the detour
+    d2 = np.full(J, 1e4, dtype=np.float32)
+    s.delta.copy_(torch.from_numpy(d2))
+    assert np.array_equal(s.sample().cpu().numpy(), oracle.sample(d2.astype(np.float64), p.eta, 0, 0, n_cand))
+
+
+def test_uniform_draw_flag_ignores_delta():
+    b = _binding()
+    J, n_cand = 50_000, 500
+    p = wl.make_problem(dict(kind="csc_uniform", n_rows=64, n_cols=J, n_true=1, lam_frac=0.1, nnz_col=2,
+                             n_candidates=n_cand, n_keep=1, rho=0.1), seed=3)
+    s = _solver(p, flags=b.FLAG_UNIFORM_DRAW)
+    s.delta.copy_(torch.rand(J, device="cuda"))
+    got = s.sample().cpu().numpy()
+    # uniform weights = any constant delta with eta chosen so that w = 1 exactly
+    want = oracle.sample(np.ones(J), 0.0, 3, 0, n_cand)
+    assert np.array_equal(got, want)
+
+
+# --------------------------------------------------------------------------------------------------
+# init
+# --------------------------------------------------------------------------------------------------
+def _small_problems():
+    return {
+        "dense": dict(kind="dense_iid", n_rows=1000, n_cols=3000, n_true=30, lam_frac=0.05,
+                      n_candidates=300, n_keep=48, rho=0.1),
+        "dense_grouped": dict(kind="dense_grouped", n_rows=2000, n_cols=2000, n_true=20, lam_frac=0.02,
+                              n_candidates=400, n_keep=64, rho=0.1, group=20),
+        "csc": dict(kind="csc_uniform", n_rows=5000, n_cols=20000, n_true=100, lam_frac=0.01, nnz_col=50,
+                    n_candidates=1000, n_keep=128, rho=0.1),
+        "csc_zipf": dict(kind="csc_zipf", n_rows=20000, n_cols=50000, n_true=100, lam_frac=0.01, nnz_col=20,
+                         n_candidates=1500, n_keep=400, rho=0.05),
+    }
+
+
+@pytest.mark.parametrize("name", list(_small_problems()))
+def test_init_state(name):
+    p = wl.make_problem(_small_problems()[name], seed=1)
+    X = oracle_matrix(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.numpy(), 1e4)
+    s = _solver(p)
+    assert np.allclose(s.colnorm2().cpu().numpy(), n2, rtol=1e-13, atol=0)
+    assert np.array_equal(s.resid.cpu().numpy(), p.y.numpy())
+    assert np.all(s.delta.cpu().numpy() == np.float32(1e4)) and np.all(s.beta.cpu().numpy() == 0)
+    f = s.objective()
+    assert abs(f - oracle.objective(resid, beta, p.lam)) < 1e-12 * f
+    assert s.get_round() == 0
+
+
+@pytest.mark.parametrize("name", ["dense", "csc"])
+def test_init_from_nonzero_beta(name):
+    p = wl.make_problem(_small_problems()[name], seed=2)
+    X = oracle_matrix(p)
+    b0 = torch.zeros(p.n_cols)
+    idx = torch.randperm(p.n_cols, generator=torch.Generator().manual_seed(0))[:40]
+    b0[idx] = torch.randn(40, generator=torch.Generator().manual_seed(1))
+    s = _solver(p, beta0=b0)
+    f_want, r_want = oracle.objective_from_scratch(X, p.y.numpy(), b0.numpy().astype(np.float64), p.lam)
+    assert np.allclose(s.resid.cpu().numpy(), r_want, rtol=0, atol=2e-7 * np.abs(r_want).max())
+    assert abs(s.objective() - f_want) < 1e-6 * f_want
+
+
+# --------------------------------------------------------------------------------------------------
+# level 2: filter and update from identical state
+# --------------------------------------------------------------------------------------------------
+def _assert_kept_matches(X, n2, cand, n_keep, rho, got_kept, got_examined):
+    want, ne, mm = oracle.filter(X, n2, cand, n_keep, rho)
+    if not np.array_equal(got_kept, want):
+        assert mm <= RHO_EXCUSE, ("kept differs without a borderline pair", mm)
+        want, ne, _ = oracle.filter(X, n2, cand, n_keep, rho, follow=got_kept, tol=RHO_EXCUSE)
+        assert np.array_equal(got_kept, want)
+    assert got_examined == ne
+    return want
+
+
+@pytest.mark.parametrize("name", list(_small_problems()))
+def test_filter_matches_oracle(name):
+    cfg = _small_problems()[name]
+    p = wl.make_problem(cfg, seed=3)
+    X = oracle_matrix(p)
+    n2 = oracle.colnorm2(X)
+    s = _solver(p)
+    rho = float(np.float32(p.rho))
+    rng = np.random.default_rng(0)
+    rejected = 0
+    for trial in range(4):
+        n_cand = [p.n_candidates, p.n_candidates, 33, 1][trial]
+        cand = rng.permutation(p.n_cols)[:n_cand].astype(np.int32)
+        if name == "dense_grouped" and trial == 0:
+            cand = np.arange(n_cand, dtype=np.int32)          # whole groups side by side: many rejections
+        kept_d, counts_d, gram = s.filter(torch.from_numpy(cand).cuda(), want_gram=True)
+        counts = counts_d.cpu().numpy()
+        kept = kept_d.cpu().numpy()
+        nk = int(counts[2])
+        assert np.all(kept[nk:] == -1) and counts[0] == n_cand
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept[:nk], int(counts[1]))
+        rejected += int(counts[1]) - nk
+        # the Gram itself against FP64 dot products on sampled pairs
+        g = gram.cpu().numpy()
+        for a, b in rng.integers(0, n_cand, size=(300, 2)):
+            want = oracle.corr(X, n2, cand[a], cand[b]) * np.sqrt(n2[cand[a]] * n2[cand[b]])
+            assert abs(g[a, b] - want) < 2e-6 + 4e-6 * abs(want), (a, b, g[a, b], want)
+    if name in ("dense_grouped", "csc_zipf", "dense"):
+        assert rejected > 0
+
+
+@pytest.mark.parametrize("name", list(_small_problems()))
+def test_update_matches_oracle(name):
+    p = wl.make_problem(_small_problems()[name], seed=4)
+    X = oracle_matrix(p)
+    s = _solver(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.numpy(), 1e4)
+    rng = np.random.default_rng(1)
+    lam = float(np.float32(p.lam))
+    for step in range(6):
+        n_kept = [p.n_keep, p.n_keep, 1, 0, p.n_keep // 2, p.n_keep][step]
+        kept = rng.permutation(p.n_cols)[:n_kept].astype(np.int32)
+        # identical state on both sides
+        beta[:] = s.beta.cpu().numpy(); resid[:] = s.resid.cpu().numpy(); delta[:] = s.delta.cpu().numpy()
+        d_got = s.update(torch.from_numpy(kept).cuda()).cpu().numpy()
+        d_want = oracle.update(X, n2, lam, kept, beta, resid, delta)
+        bmax = max(np.abs(beta).max(), 1e-30)
+        assert np.all(np.abs(d_got[:n_kept] - d_want) <= RTOL_DBETA * np.abs(d_want) + ATOL_DBETA * bmax)
+        assert np.all(d_got[n_kept:] == 0)
+        assert np.allclose(s.beta.cpu().numpy(), beta, rtol=0, atol=1.2e-7 * bmax)
+        assert np.allclose(s.resid.cpu().numpy(), resid, rtol=0, atol=2e-7 * np.abs(resid).max() + 1e-7 * bmax)
+        dl = s.delta.cpu().numpy()
+        assert np.allclose(dl[kept], np.abs(d_want), rtol=RTOL_DBETA, atol=ATOL_DBETA * bmax)
+        untouched = np.ones(p.n_cols, bool); untouched[kept] = False
+        assert np.all(dl[untouched] == delta[untouched].astype(np.float32))
+    assert s.get_round() == 0                      # split-phase calls do not advance t
+
+
+@pytest.mark.parametrize("name", list(_small_problems()))
+def test_rounds_teacher_forced(name):
+    """Whole rounds; before each one the oracle is given the device's state, so every round is checked
+    from identical inputs (candidates exact, kept equal, dbeta within tolerance)."""
+    p = wl.make_problem(_small_problems()[name], seed=5)
+    X = oracle_matrix(p)
+    s = _solver(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.numpy(), 1e4)
+    lam, eta, rho = float(np.float32(p.lam)), float(np.float32(p.eta)), float(np.float32(p.rho))
+    n_rounds = 40
+    for t in range(n_rounds):
+        beta[:] = s.beta.cpu().numpy(); resid[:] = s.resid.cpu().numpy(); delta[:] = s.delta.cpu().numpy()
+        cand_d, kept_d, dbeta_d, counts_d = s.round()
+        counts = counts_d.cpu().numpy(); nk = int(counts[2])
+        cand = cand_d.cpu().numpy(); kept = kept_d.cpu().numpy()[:nk]; d_got = dbeta_d.cpu().numpy()[:nk]
+        want_cand = oracle.sample(delta, eta, p.seed, t, p.n_candidates)
+        assert np.array_equal(cand, want_cand), t
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept, int(counts[1]))
+        d_want = oracle.update(X, n2, lam, kept, beta, resid, delta)
+        bmax = max(np.abs(beta).max(), 1e-30)
+        assert np.all(np.abs(d_got - d_want) <= RTOL_DBETA * np.abs(d_want) + ATOL_DBETA * bmax), t
+        assert int(counts[3]) == int(np.count_nonzero(d_got))
+    assert s.get_round() == n_rounds
+    tot = s.totals()
+    assert tot["rounds"] == n_rounds and tot["kept"] > 0
+    assert s.status() == (0, 0)
+
+
+# --------------------------------------------------------------------------------------------------
+# level 3: free-running objective
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,rounds", [("dense", 600), ("csc", 900), ("dense_grouped", 500)])
+def test_objective_after_fixed_rounds(name, rounds):
+    p = wl.make_problem(_small_problems()[name], seed=6)
+    X = oracle_matrix(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.numpy(), 1e4)
+    lam, eta, rho = float(np.float32(p.lam)), float(np.float32(p.eta)), float(np.float32(p.rho))
+    for t in range(rounds):
+        oracle.round(X, n2, lam, eta, rho, p.n_candidates, p.n_keep, p.seed, t, beta, resid, delta)
+    f_want = oracle.objective(resid, beta, lam)
+    s = _solver(p)
+    s.run(rounds)
+    f_got = s.objective()
+    assert abs(f_got - f_want) <= RTOL_OBJ * f_want, (f_got, f_want)
+    # the maintained FP32 residual has not drifted from y - X beta
+    f_scratch, r_scratch = oracle.objective_from_scratch(X, p.y.numpy(), s.beta.cpu().numpy().astype(np.float64), lam)
+    assert abs(f_scratch - f_got) <= 1e-5 * f_want
+    assert np.abs(s.resid.cpu().numpy() - r_scratch).max() <= 1e-4 * np.abs(r_scratch).max()
+
+
+def test_same_seed_gives_identical_bits():
+    for name in ("dense", "csc_zipf"):
+        p = wl.make_problem(_small_problems()[name], seed=7)
+        outs = []
+        for rep in range(2):
+            s = _solver(p)
+            s.run(60)
+            outs.append((s.beta.cpu().numpy().copy(), s.resid.cpu().numpy().copy(), s.delta.cpu().numpy().copy()))
+        for a, b in zip(*outs):
+            assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_round_on_host_state_equals_round_on_device_state():
+    p = wl.make_problem(_small_problems()["dense"], seed=8)
+    a, b = _solver(p), _solver(p)
+    beta_h = torch.zeros(p.n_cols).pin_memory(); resid_h = p.y.clone().pin_memory()
+    delta_h = torch.full((p.n_cols,), 1e4).pin_memory()
+    kept_h = torch.zeros(p.n_keep, dtype=torch.int32).pin_memory()
+    dbeta_h = torch.zeros(p.n_keep).pin_memory(); counts_h = torch.zeros(4, dtype=torch.int32).pin_memory()
+    for t in range(5):
+        cand, kept, dbeta, counts = a.round()
+        b.round_host(beta_h, resid_h, delta_h, kept_h, dbeta_h, counts_h)
+        assert torch.equal(kept.cpu(), kept_h) and torch.equal(dbeta.cpu(), dbeta_h) and torch.equal(counts.cpu(), counts_h)
+        assert torch.equal(a.beta.cpu(), beta_h) and torch.equal(a.resid.cpu(), resid_h) and torch.equal(a.delta.cpu(), delta_h)
+
+
+def test_resume_from_saved_state():
+    p = wl.make_problem(_small_problems()["csc"], seed=9)
+    a = _solver(p)
+    a.run(10)
+    saved = (a.beta.clone(), a.resid.clone(), a.delta.clone(), a.get_round())
+    a.run(10)
+    b = _solver(p)
+    b.beta.copy_(saved[0]); b.resid.copy_(saved[1]); b.delta.copy_(saved[2]); b.set_round(saved[3])
+    b.run(10)
+    assert torch.equal(a.beta, b.beta) and torch.equal(a.resid, b.resid) and torch.equal(a.delta, b.delta)
+
+
+def test_no_filter_flag_keeps_first_candidates():
+    b = _binding()
+    p = wl.make_problem(_small_problems()["dense_grouped"], seed=10)
+    s = _solver(p, flags=b.FLAG_NO_FILTER)
+    cand, kept, dbeta, counts = s.round()
+    assert torch.equal(kept, cand[: p.n_keep]) and counts.cpu().tolist()[1:3] == [p.n_keep, p.n_keep]
+
+
+def test_ragged_rows_and_padding():
+    # N not a multiple of 4 or of any tile, ld > N with NaN in the padding: nothing may leak in
+    cfg = dict(kind="dense_iid", n_rows=1003, n_cols=777, n_true=10, lam_frac=0.05, n_candidates=131, n_keep=19,
+               rho=0.1)
+    p = wl.make_problem(cfg, seed=11)
+    ld = 1008
+    vals = torch.full((p.n_cols, ld), float("nan"))
+    vals[:, : p.n_rows] = p.values
+    b = _binding()
+    s = b.StradsLasso(wl.DENSE, p.n_rows, p.n_cols, vals.cuda(), p.y.cuda(), p.lam, p.eta, p.rho, p.n_candidates,
+                      p.n_keep, seed=p.seed)
+    X = oracle_matrix(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.numpy(), 1e4)
+    lam, eta, rho = float(np.float32(p.lam)), float(np.float32(p.eta)), float(np.float32(p.rho))
+    assert np.allclose(s.colnorm2().cpu().numpy(), n2, rtol=1e-13)
+    for t in range(12):
+        beta[:] = s.beta.cpu().numpy(); resid[:] = s.resid.cpu().numpy(); delta[:] = s.delta.cpu().numpy()
+        cand_d, kept_d, dbeta_d, counts_d = s.round()
+        counts = counts_d.cpu().numpy(); nk = int(counts[2])
+        cand = cand_d.cpu().numpy(); kept = kept_d.cpu().numpy()[:nk]
+        assert np.array_equal(cand, oracle.sample(delta, eta, p.seed, t, p.n_candidates))
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept, int(counts[1]))
+        d_want = oracle.update(X, n2, lam, kept, beta, resid, delta)
+        assert np.all(np.abs(dbeta_d.cpu().numpy()[:nk] - d_want) <= RTOL_DBETA * np.abs(d_want) + ATOL_DBETA)
+    assert torch.isfinite(s.resid).all() and s.status() == (0, 0)
+
+
+def test_degenerate_sizes():
+    # P' = P = J = 1 and a single row
+    b = _binding()
+    vals = torch.tensor([[2.0, 0.0, 0.0, 0.0]]).cuda()
+    y = torch.tensor([3.0]).cuda()
+    s = b.StradsLasso(wl.DENSE, 1, 1, vals, y, lam=1.0, eta=1e-6, rho=0.1, n_candidates=1, n_keep=1)
+    cand, kept, dbeta, counts = s.round()
+    # n = 4, g = 6: beta = S(6/4, 1/4) = 1.25, r = 3 - 2*1.25 = 0.5
+    assert cand.tolist() == [0] and kept.tolist() == [0] and abs(float(dbeta[0]) - 1.25) < 1e-7
+    assert abs(float(s.resid[0]) - 0.5) < 1e-7 and abs(s.objective() - (0.125 + 1.25)) < 1e-7
+    # an all-zero column never moves and never conflicts
+    vals = torch.zeros((3, 8)); vals[1, :4] = 0.5
+    s = b.StradsLasso(wl.DENSE, 8, 3, vals.cuda(), torch.ones(8).cuda(), lam=0.1, eta=1e-6, rho=0.1,
+                      n_candidates=3, n_keep=3)
+    cand, kept, dbeta, counts = s.round()
+    assert counts.cpu().tolist() == [3, 3, 3, 1] and sorted(kept.tolist()) == [0, 1, 2]
+    assert s.beta.cpu().tolist()[0] == 0.0 and s.beta.cpu().tolist()[2] == 0.0 and s.status() == (0, 0)
