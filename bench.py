@@ -1,0 +1,322 @@
+#!/usr/bin/env python
+"""Benchmark of the scheduled-Lasso round on B200: coordinate updates per second.
+
+A step is one whole round (sample -> Gram -> greedy filter -> update) of the dense 10,000 x 100,000
+configuration ("c2"), on synthetic data generated on the device from a seed.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2] [--impl ours|reference]
+
+Prints ONE JSON line.  `--impl reference` times the FP64 CPU oracle instead (rank 0 only).
+With N > 1 (under torchrun) every rank runs an independent replica: the round has no inter-GPU step.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_1312_5766_b200 import workloads as wl  # noqa: E402
+
+METRIC = "coordinate updates/sec and % of HBM roofline per STRADS round (1xB200)"
+UNIT = "coordinate updates/s"
+SM_COUNT, FMA_LANES_PER_SM = 148, 128
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                "sm_max_mhz": d.get("sm_max_mhz", 1965.0), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(gpu_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self) -> dict:
+        if self.p is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        for line in self.f.read().splitlines():
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                sm.append(float(c[1])); mx.append(float(c[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        self.f.close()
+        os.unlink(self.f.name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+def oracle_inputs(p: wl.LassoProblem):
+    """Host copies of the device arrays for the CPU oracle (the same FP32 bits)."""
+    import oracle
+    if p.layout == wl.DENSE:
+        X = oracle.Matrix.dense(p.values.cpu().numpy(), n_rows=p.n_rows)
+    else:
+        X = oracle.Matrix.csc(p.n_rows, p.n_cols, p.values.cpu().numpy(), p.row_idx.cpu().numpy(),
+                              p.col_ptr.cpu().numpy())
+    return X
+
+
+def time_oracle_rounds(p, X, n2, state, t0, n_cand, n_keep, budget_s, min_rounds=3, max_rounds=10**9):
+    """Runs oracle rounds from `state` until the time budget is used; returns (updates, seconds, rounds)."""
+    import oracle
+    beta, resid, delta = state
+    lam, eta, rho = float(np.float32(p.lam)), float(np.float32(p.eta)), float(np.float32(p.rho))
+    kept_total, rounds = 0, 0
+    start = time.perf_counter()
+    while rounds < max_rounds and (rounds < min_rounds or time.perf_counter() - start < budget_s):
+        out = oracle.round(X, n2, lam, eta, rho, n_cand, n_keep, p.seed, t0 + rounds, beta, resid, delta)
+        kept_total += int(out["counts"][2])
+        rounds += 1
+    return kept_total, time.perf_counter() - start, rounds
+
+
+def run_reference(args, device):
+    """The reference arm: the FP64 oracle, as it stands, on the host cores (single thread)."""
+    import oracle
+    p = wl.make_problem(args.workload, seed=0, device=device)
+    X = oracle_inputs(p)
+    n2, beta, resid, delta = oracle.init(X, p.y.cpu().numpy(), 1e4)
+    # size the per-step sample so that the whole run ends within a few minutes
+    n_cand, n_keep = p.n_candidates, p.n_keep
+    budget = 150.0
+    probe = (beta.copy(), resid.copy(), delta.copy())
+    while True:
+        _, sec, _ = time_oracle_rounds(p, X, n2, tuple(a.copy() for a in probe), 0, n_cand, n_keep, 0.0, min_rounds=1,
+                                       max_rounds=1)
+        if sec * (args.steps + args.warmup) <= budget or n_keep == 1:
+            break
+        n_keep = max(1, n_keep // 2)
+        n_cand = max(n_keep, n_cand // 2)
+    time_oracle_rounds(p, X, n2, (beta, resid, delta), 0, n_cand, n_keep, 0.0, min_rounds=args.warmup,
+                       max_rounds=args.warmup)
+    kept, sec, rounds = time_oracle_rounds(p, X, n2, (beta, resid, delta), args.warmup, n_cand, n_keep, 0.0,
+                                           min_rounds=args.steps, max_rounds=args.steps)
+    value = kept / sec
+    sample = (f"{rounds} oracle rounds of {args.workload} with P'={n_cand}, P={n_keep} per step "
+              f"(full round is P'={p.n_candidates}, P={p.n_keep})")
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * sec / rounds, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "n_rows": p.n_rows, "n_cols": p.n_cols, "n_candidates": n_cand,
+                   "n_keep": n_keep},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+def aggregate(units_local: float, ms_local: float, dist_ok: bool, device):
+    """Whole-job numbers: units summed over ranks, time = max over ranks."""
+    if not dist_ok:
+        return units_local, ms_local
+    import torch.distributed as dist
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    m = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    dist.all_reduce(m, op=dist.ReduceOp.MAX)
+    return float(u.item()), float(m.item())
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default="c2")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=200)
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
+    ap.add_argument("--n-cols", type=int, default=0,
+                    help="profiling aid: same workload with fewer columns J (keeps N, P', P), so that a "
+                         "multi-pass ncu capture holds less device memory")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        device = f"cuda:{local_rank}" if torch.cuda.is_available() else "cpu"
+        print(json.dumps(run_reference(args, device)), flush=True)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    torch.cuda.set_device(local_rank)
+    device = f"cuda:{local_rank}"
+    dist_ok = world > 1
+    if dist_ok:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(device))
+
+    from paper_1312_5766_b200 import binding
+    cfg = dict(wl.CONFIGS[args.workload], name=args.workload)
+    if args.n_cols:
+        cfg["n_cols"] = args.n_cols
+        cfg["n_true"] = max(1, cfg["n_true"] * args.n_cols // wl.CONFIGS[args.workload]["n_cols"])
+    p = wl.make_problem(cfg, seed=0, device=device)                # every rank: the same problem, own replica
+    p.seed = rank                                                   # ... with its own random stream
+    s = binding.StradsLasso.from_problem(p, device=device)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist_ok:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: K rounds after W warm-up rounds -------------------------------------
+    s.run(args.warmup)
+    kept_before = s.totals()["kept"]
+    s.profile_begin(args.steps)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    clocks = ClockSampler(local_rank)
+    ev0.record()
+    s.run(args.steps)
+    ev1.record()
+    barrier()
+    clk = clocks.stop()
+    ms_local = ev0.elapsed_time(ev1)
+    prof = s.profile_end()
+    tot = s.totals()
+    kept_local = tot["kept"] - kept_before
+    kept_all, ms = aggregate(kept_local, ms_local, dist_ok, device)
+    value = kept_all / (ms * 1e-3)
+    objective = s.objective()
+    rc, status_bits = s.status()
+
+    # ---- roofline of the dominant kernel (dense: the candidate Gram, an FP32 contraction) ----------
+    peaks = measured_peaks()
+    step_ms = {k: prof[k] / max(prof["rounds"], 1) for k in ("sample_ms", "gram_ms", "filter_ms", "update_ms")}
+    if p.layout == wl.DENSE:
+        flops = float(p.n_candidates) * (p.n_candidates - 1) * p.n_rows          # U'(U'-1) N, upper triangle
+        achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
+        peak = SM_COUNT * FMA_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+        roofline = {"kernel": "k_gram_dense_simt", "bound": "alu", "achieved": achieved, "peak": peak,
+                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
+                    "peak_source": "148 SMs x 128 FP32 FMA lanes x 2 flop x max SM clock (derived)"}
+    else:
+        nnz_col = p.nnz / p.n_cols
+        byts = 8.0 * nnz_col * p.n_candidates
+        achieved = byts / (step_ms["gram_ms"] * 1e-3) / 1e9
+        roofline = {"kernel": "k_gram_csc", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
+                    "peak_source": peaks["source"]}
+    # the update kernels against the HBM roofline (bytes: kept columns once + r read and written)
+    kept_per_round = kept_local / args.steps
+    if p.layout == wl.DENSE:
+        upd_bytes = 4.0 * p.n_rows * kept_per_round + 8.0 * p.n_rows + 16.0 * kept_per_round
+    else:
+        upd_bytes = 8.0 * (p.nnz / p.n_cols) * kept_per_round + 8.0 * p.n_rows
+    upd_gbs = upd_bytes / (step_ms["update_ms"] * 1e-3) / 1e9
+
+    # ---- end to end: state in pinned host memory, copied in and out every step ---------------------
+    e2e_steps = min(args.e2e_steps, args.steps)
+    beta_h = s.beta.cpu().pin_memory(); resid_h = s.resid.cpu().pin_memory(); delta_h = s.delta.cpu().pin_memory()
+    kept_h = torch.zeros(p.n_keep, dtype=torch.int32).pin_memory()
+    dbeta_h = torch.zeros(p.n_keep).pin_memory(); counts_h = torch.zeros(4, dtype=torch.int32).pin_memory()
+    for _ in range(3):
+        s.round_host(beta_h, resid_h, delta_h, kept_h, dbeta_h, counts_h)
+    barrier()
+    e2e_kept = 0
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        s.round_host(beta_h, resid_h, delta_h, kept_h, dbeta_h, counts_h)
+        e2e_kept += int(counts_h[2])
+    torch.cuda.synchronize()
+    e2e_ms_local = (time.perf_counter() - t0) * 1e3
+    e2e_kept_all, e2e_ms = aggregate(e2e_kept, e2e_ms_local, dist_ok, device)
+    h2d = 4 * (2 * p.n_cols + p.n_rows)
+    d2h = h2d + 4 * (2 * p.n_keep + 4)
+
+    # ---- CPU baseline: the oracle on a bounded sample of the same workload (rank 0, N = 1 only) ----
+    cpu_baseline = None
+    if rank == 0 and world == 1 and args.cpu_baseline_seconds > 0:
+        import oracle
+        X = oracle_inputs(p)
+        n2 = s.colnorm2().cpu().numpy().copy()
+        state = (s.beta.cpu().numpy().astype(np.float64), s.resid.cpu().numpy().astype(np.float64),
+                 s.delta.cpu().numpy().astype(np.float64))
+        k, sec, rounds = time_oracle_rounds(p, X, n2, state, s.get_round(), p.n_candidates, p.n_keep,
+                                            args.cpu_baseline_seconds)
+        cpu_baseline = {"value": k / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"{rounds} full oracle rounds of {args.workload} from the state after the timed "
+                                  f"region ({sec:.1f} s, single thread; host has {os.cpu_count()} cores)"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload + (f" with J={args.n_cols}" if args.n_cols else ""), "layout": "dense" if p.layout == wl.DENSE else "csc",
+                       "n_rows": p.n_rows, "n_cols": p.n_cols, "n_candidates": p.n_candidates, "n_keep": p.n_keep,
+                       "rho": p.rho, "eta": p.eta, "lambda": p.lam, "parallelism": f"replicas x{world}",
+                       "l2": "design matrix (4 GB for c2) far exceeds L2; every round draws a fresh candidate set"},
+            "rounds_per_s": world * args.steps / (ms * 1e-3),
+            "kept_per_round": kept_per_round,
+            "objective": objective, "status_bits": status_bits,
+            "step_ms": step_ms,
+            "roofline": roofline,
+            "update_hbm": {"achieved": upd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                           "frac": upd_gbs / peaks["hbm_gbs"], "bytes_per_round": upd_bytes},
+            "cpu_baseline": cpu_baseline,
+            "e2e": {"value": e2e_kept_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "steps": e2e_steps},
+            "gpu_launches": 7 * args.steps,
+            "clocks": clk,
+        }
+        print(json.dumps(line), flush=True)
+    if dist_ok:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

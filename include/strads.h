@@ -161,6 +161,14 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out);
 /* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);
 
+/* Optional step timing with CUDA events on the handle's stream.  After strads_profile_begin the next
+ * max_rounds rounds (strads_round / strads_run / strads_round_host) record an event at every step
+ * boundary; strads_profile_end waits for the stream and returns the summed device time in
+ * milliseconds of ms[0] sampling, ms[1] Gram, ms[2] greedy filter, ms[3] update over *rounds rounds.
+ * Events are host-side driver objects; no device memory is allocated. */
+int strads_profile_begin(strads_handle_t h, int64_t max_rounds);
+int strads_profile_end(strads_handle_t h, double* ms_host_out /* [4] */, int64_t* rounds_host_out);
+
 int strads_destroy(strads_handle_t h);
 
 const char* strads_error_string(int code);

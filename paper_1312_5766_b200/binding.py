@@ -25,7 +25,7 @@ EXPORTS = [
     "strads_workspace_bytes", "strads_lasso_init", "strads_round", "strads_run", "strads_round_host",
     "strads_objective", "strads_sample", "strads_filter", "strads_update", "strads_get_round",
     "strads_set_round", "strads_totals", "strads_status", "strads_colnorm2", "strads_destroy",
-    "strads_error_string", "strads_last_cuda_error",
+    "strads_error_string", "strads_last_cuda_error", "strads_profile_begin", "strads_profile_end",
 ]
 
 
@@ -78,6 +78,8 @@ def load() -> C.CDLL:
         lib.strads_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
         lib.strads_colnorm2.argtypes = [C.c_void_p, C.POINTER(C.c_void_p)]
         lib.strads_destroy.argtypes = [C.c_void_p]
+        lib.strads_profile_begin.argtypes = [C.c_void_p, C.c_int64]
+        lib.strads_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = lib
     return _lib
 
@@ -233,6 +235,15 @@ class StradsLasso:
         _check(load().strads_colnorm2(self._h, C.byref(ptr)), "strads_colnorm2")
         off = ptr.value - self.workspace.data_ptr()
         return self.workspace[off:off + 8 * self.J].view(torch.float64)
+
+    def profile_begin(self, max_rounds: int) -> None:
+        _check(load().strads_profile_begin(self._h, int(max_rounds)), "strads_profile_begin")
+
+    def profile_end(self) -> dict:
+        ms = (C.c_double * 4)()
+        n = C.c_int64(0)
+        _check(load().strads_profile_end(self._h, ms, C.byref(n)), "strads_profile_end")
+        return {"rounds": int(n.value), "sample_ms": ms[0], "gram_ms": ms[1], "filter_ms": ms[2], "update_ms": ms[3]}
 
     def close(self) -> None:
         if self._h:

@@ -15,6 +15,9 @@ struct strads_lasso_s {
   cudaStream_t stream;
   int device;
   long long round_host;     // mirrors DeviceState::round (every round adds exactly one)
+  // optional step timing: 5 events per round (start, after sample, Gram, filter, update)
+  cudaEvent_t* prof_events;
+  long long prof_cap, prof_rounds;
 };
 
 namespace {
@@ -95,10 +98,19 @@ int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_
 
 int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
   const Problem& p = h->p;
+  cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + 5 * h->prof_rounds : nullptr;
+  if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
-  int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr);
-  if (rc) return rc;
+  if (ev) CK(cudaEventRecord(ev[1], h->stream));
+  if (!(p.flags & STRADS_FLAG_NO_FILTER)) {
+    if (p.layout == STRADS_DENSE_COLMAJOR) CK(launch_gram_dense_simt(p, p.cand, p.n_cand, out ? out->gram : nullptr, h->stream));
+    else CK(launch_gram_csc(p, p.cand, p.n_cand, out ? out->gram : nullptr, h->stream));
+  }
+  if (ev) CK(cudaEventRecord(ev[2], h->stream));
+  CK(launch_filter(p, p.cand, p.n_cand, p.kept, h->stream));
+  if (ev) CK(cudaEventRecord(ev[3], h->stream));
   CK(launch_update(p, p.kept, 1, h->stream));
+  if (ev) { CK(cudaEventRecord(ev[4], h->stream)); h->prof_rounds += 1; }
   h->round_host += 1;
   if (out != nullptr) {
     if (out->cand) CK(cudaMemcpyAsync(out->cand, p.cand, sizeof(int) * p.n_cand, cudaMemcpyDeviceToDevice, h->stream));
@@ -161,6 +173,7 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   p.obj_partial = reinterpret_cast<double*>(ws + L.off_obj);
   h->stream = static_cast<cudaStream_t>(c->stream);
   h->round_host = 0;
+  h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
 
   auto fail = [&](int code) { delete h; return code; };
   cudaError_t e = cudaGetDevice(&h->device);
@@ -286,9 +299,53 @@ int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out) {
   return STRADS_OK;
 }
 
+int strads_profile_begin(strads_handle_t h, int64_t max_rounds) {
+  if (h == nullptr || max_rounds < 1 || max_rounds > (1 << 20)) return STRADS_ERR_INVALID_ARG;
+  if (h->prof_events != nullptr) return STRADS_ERR_INVALID_ARG;
+  h->prof_events = new (std::nothrow) cudaEvent_t[5 * max_rounds];
+  if (h->prof_events == nullptr) return STRADS_ERR_INVALID_ARG;
+  for (long long i = 0; i < 5 * max_rounds; ++i) {
+    cudaError_t e = cudaEventCreate(&h->prof_events[i]);
+    if (e != cudaSuccess) {
+      for (long long k = 0; k < i; ++k) cudaEventDestroy(h->prof_events[k]);
+      delete[] h->prof_events;
+      h->prof_events = nullptr;
+      return cuda_fail(e, "cudaEventCreate");
+    }
+  }
+  h->prof_cap = max_rounds;
+  h->prof_rounds = 0;
+  return STRADS_OK;
+}
+
+int strads_profile_end(strads_handle_t h, double* ms_host_out, int64_t* rounds_host_out) {
+  if (h == nullptr || h->prof_events == nullptr) return STRADS_ERR_INVALID_ARG;
+  int rc = STRADS_OK;
+  cudaError_t e = cudaStreamSynchronize(h->stream);
+  if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
+  double ms[4] = {0, 0, 0, 0};
+  for (long long r = 0; r < h->prof_rounds && rc == STRADS_OK; ++r)
+    for (int k = 0; k < 4; ++k) {
+      float v = 0.f;
+      e = cudaEventElapsedTime(&v, h->prof_events[5 * r + k], h->prof_events[5 * r + k + 1]);
+      if (e != cudaSuccess) { rc = cuda_fail(e, "cudaEventElapsedTime"); break; }
+      ms[k] += v;
+    }
+  if (ms_host_out) for (int k = 0; k < 4; ++k) ms_host_out[k] = ms[k];
+  if (rounds_host_out) *rounds_host_out = h->prof_rounds;
+  for (long long i = 0; i < 5 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
+  delete[] h->prof_events;
+  h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
+  return rc;
+}
+
 int strads_destroy(strads_handle_t h) {
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
   cudaStreamSynchronize(h->stream);
+  if (h->prof_events != nullptr) {
+    for (long long i = 0; i < 5 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
+    delete[] h->prof_events;
+  }
   delete h;
   return STRADS_OK;
 }

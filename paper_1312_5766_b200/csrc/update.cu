@@ -216,8 +216,6 @@ __global__ void k_set_counts(Problem p, int n_cand, int n_examined, int n_kept) 
   p.st->counts[0] = n_cand; p.st->counts[1] = n_examined; p.st->counts[2] = n_kept; p.st->counts[3] = 0;
 }
 
-__global__ void k_clear_nonzero(Problem p) { p.st->counts[3] = 0; }
-
 __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out) {
   const int n_kept = p.st->counts[2];
   for (int a = blockIdx.x * blockDim.x + threadIdx.x; a < p.n_keep; a += gridDim.x * blockDim.x) {
@@ -230,7 +228,6 @@ __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta
 }  // namespace
 
 cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s) {
-  k_clear_nonzero<<<1, 1, 0, s>>>(p);
   if (p.layout == STRADS_DENSE_COLMAJOR) {
     k_dot_dense<<<dim3(p.dot_parts, p.n_keep), kThreads, 0, s>>>(p, kept);
     k_apply_dense<<<(unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s>>>(p, kept, advance);
