@@ -113,8 +113,10 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
 
 size_t filter_smem_bytes(const Problem& p) { return (size_t)(kBatch + 1) * p.mask_words * sizeof(unsigned int); }
 
-cudaError_t prepare_filter(const Problem& p) {
-  return cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)filter_smem_bytes(p));
+// Kernel-wide attribute: the largest size any handle can need (see prepare_sample).
+cudaError_t prepare_filter(const Problem&) {
+  return cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)((kBatch + 1) * (STRADS_MAX_CANDIDATES / 32) * sizeof(unsigned int)));
 }
 
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s) {

@@ -210,8 +210,11 @@ static size_t sort_smem_bytes(const Problem& p) {
   return (size_t)n * sizeof(unsigned long long);
 }
 
-cudaError_t prepare_sample(const Problem& p) {
-  return cudaFuncSetAttribute(k_sample_sort, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_smem_bytes(p));
+// The attribute belongs to the kernel, not to a handle: always ask for the largest size any handle can
+// need, so that a later handle with fewer candidates does not lower the limit under an earlier one.
+cudaError_t prepare_sample(const Problem&) {
+  return cudaFuncSetAttribute(k_sample_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)(STRADS_MAX_CANDIDATES * sizeof(unsigned long long)));
 }
 
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
