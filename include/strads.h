@@ -171,6 +171,25 @@ int strads_profile_end(strads_handle_t h, double* ms_host_out /* [4] */, int64_t
 
 int strads_destroy(strads_handle_t h);
 
+/* (No counterpart in the paper: a packaging variant of SAP step 1.)
+ * The candidate draw of strads_sample for callers that must not allocate device memory -- code that
+ * runs inside another component's memory pool, plugins whose host forbids cudaMalloc after start-up,
+ * latency-critical loops.  It needs no handle and no workspace: the scratch memory of the select
+ * passes lives in a fixed array inside the library (about 65 KB on every GPU that loads it, until the
+ * process exits), which limits it to n_candidates <= STRADS_STATIC_MAX_CANDIDATES; larger requests
+ * return STRADS_ERR_UNSUPPORTED.  The call allocates nothing (no cudaMalloc / cudaFree, no allocating
+ * library routine).
+ *   delta_dev [n_cols] device, 16-byte aligned; cand_dev [n_candidates] device: the same ordered list
+ *   strads_sample gives for the same (delta, eta, seed, t, flags); stream: cudaStream_t.
+ * Asynchronous on `stream`.  The first call on a device looks up the array's device address (with
+ * that device current); make that first call before any stream capture begins.  All calls on one
+ * device share the array and it keeps the previous call's contents (the call clears what must start
+ * at zero), so two calls that overlap on the GPU -- different streams, or different threads -- race:
+ * serialise them. */
+#define STRADS_STATIC_MAX_CANDIDATES 4096
+int strads_sample_static(const float* delta_dev, int64_t n_cols, float eta, uint64_t seed, uint64_t t,
+                         int32_t n_candidates, uint32_t flags, int32_t* cand_dev, void* stream);
+
 const char* strads_error_string(int code);
 /* Text of the last CUDA error seen by this library on the calling thread ("" if none). */
 const char* strads_last_cuda_error(void);

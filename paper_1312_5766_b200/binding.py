@@ -26,6 +26,7 @@ EXPORTS = [
     "strads_objective", "strads_sample", "strads_filter", "strads_update", "strads_get_round",
     "strads_set_round", "strads_totals", "strads_status", "strads_colnorm2", "strads_destroy",
     "strads_error_string", "strads_last_cuda_error", "strads_profile_begin", "strads_profile_end",
+    "strads_sample_static",
 ]
 
 
@@ -79,6 +80,8 @@ def load() -> C.CDLL:
         lib.strads_colnorm2.argtypes = [C.c_void_p, C.POINTER(C.c_void_p)]
         lib.strads_destroy.argtypes = [C.c_void_p]
         lib.strads_profile_begin.argtypes = [C.c_void_p, C.c_int64]
+        lib.strads_sample_static.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_uint64, C.c_uint64, C.c_int32,
+                                             C.c_uint32, C.c_void_p, C.c_void_p]
         lib.strads_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
         _lib = lib
     return _lib
@@ -110,6 +113,24 @@ def workspace_bytes(layout, n_rows, n_cols, n_candidates, n_keep, nnz=0, ld=None
     out = C.c_size_t(0)
     _check(load().strads_workspace_bytes(C.byref(cfg), C.byref(out)), "strads_workspace_bytes")
     return int(out.value)
+
+
+STATIC_MAX_CANDIDATES = 4096
+
+
+def sample_static(delta: torch.Tensor, eta: float, seed: int, t: int, n_candidates: int, flags: int = 0,
+                  out: torch.Tensor | None = None) -> torch.Tensor:
+    """Candidate draw without a handle or workspace (strads_sample_static): for callers that cannot
+    allocate device memory.  `out` (int32 [n_candidates], device) is allocated here only if not given."""
+    assert delta.is_cuda and delta.dtype == torch.float32 and delta.is_contiguous()
+    if out is None:
+        out = torch.empty(n_candidates, dtype=torch.int32, device=delta.device)
+    with torch.cuda.device(delta.device):
+        stream = torch.cuda.current_stream().cuda_stream
+        _check(load().strads_sample_static(_ptr(delta), int(delta.numel()), float(eta), int(seed), int(t),
+                                           int(n_candidates), int(flags), _ptr(out), C.c_void_p(stream)),
+               "strads_sample_static")
+    return out
 
 
 class StradsLasso:

@@ -13,6 +13,9 @@
 //                    that CTA alone refines the boundary over further 12-bit digits (rare, exact).
 //   k_sample_collect pass 2: appends "sure" and "boundary" keys to two small buffers.
 //   k_sample_sort    one CTA: bitonic sort of both buffers in shared memory, writes cand[P'].
+#include <cstddef>
+#include <mutex>
+
 #include "strads_internal.cuh"
 
 namespace strads {
@@ -230,3 +233,84 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
 }
 
 }  // namespace strads
+
+// ------------------------------------------------------------------------------------------------
+// strads_sample_static: the same candidate draw for callers that cannot allocate device memory.
+//
+// The select passes need scratch memory (a 4096-bin histogram, two key buffers, a few counters).
+// The handle-based path carves it out of the caller's workspace; here it lives in one file-scope
+// device array of fixed size, so a caller that may not call cudaMalloc -- code running inside
+// somebody else's memory pool, a plugin whose host forbids allocation after start-up, a real-time
+// loop -- still gets the draw.  Every GPU that loads the library holds these ~65 KB until exit.
+// ------------------------------------------------------------------------------------------------
+namespace strads {
+namespace {
+
+struct StaticSampleScratch {
+  DeviceState st;
+  unsigned int hist[kHistBins];
+  unsigned long long sure[STRADS_STATIC_MAX_CANDIDATES];
+  unsigned long long boundary[STRADS_STATIC_MAX_CANDIDATES / 2];
+};
+
+static __device__ __align__(256) unsigned char g_static_sample_scratch[sizeof(StaticSampleScratch)];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+StaticSampleScratch* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device
+int g_static_sms[kMaxDevices] = {};
+
+__global__ void k_static_set_round(StaticSampleScratch* sc, unsigned long long t) { sc->st.round = t; }
+
+}  // namespace
+}  // namespace strads
+
+extern "C" int strads_sample_static(const float* delta_dev, int64_t n_cols, float eta, uint64_t seed, uint64_t t,
+                                    int32_t n_candidates, uint32_t flags, int32_t* cand_dev, void* stream) {
+  using namespace strads;
+  if (delta_dev == nullptr || cand_dev == nullptr) return STRADS_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(delta_dev) & 15) != 0) return STRADS_ERR_INVALID_ARG;
+  if (n_cols < 1 || n_cols >= (1ll << 31) || n_candidates < 1 || n_candidates > n_cols) return STRADS_ERR_INVALID_ARG;
+  if (!(eta > 0.f) && !(flags & STRADS_FLAG_UNIFORM_DRAW)) return STRADS_ERR_INVALID_ARG;
+  if (n_candidates > STRADS_STATIC_MAX_CANDIDATES) return STRADS_ERR_UNSUPPORTED;   // scratch array is fixed-size
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return STRADS_ERR_CUDA;
+  StaticSampleScratch* sc = nullptr;
+  int sms = 0;
+  {
+    // once per device, with that device current: in host code the array's name is only a stand-in,
+    // the address a kernel can use comes from cudaGetSymbolAddress
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_ptr[dev] == nullptr) {
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_sample_scratch) != cudaSuccess || ptr == nullptr) return STRADS_ERR_CUDA;
+      if (cudaDeviceGetAttribute(&g_static_sms[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+        return STRADS_ERR_CUDA;
+      g_static_ptr[dev] = static_cast<StaticSampleScratch*>(ptr);
+    }
+    sc = g_static_ptr[dev];
+    sms = g_static_sms[dev];
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the last call left: counters, tickets and histogram must start at zero
+  if (cudaMemsetAsync(sc, 0, offsetof(StaticSampleScratch, sure), s) != cudaSuccess) return STRADS_ERR_CUDA;
+  k_static_set_round<<<1, 1, 0, s>>>(sc, t);
+
+  Problem p = {};
+  p.J = n_cols;
+  p.delta = const_cast<float*>(delta_dev);
+  p.eta = eta;
+  p.seed = seed;
+  p.flags = flags;
+  p.n_cand = n_candidates;
+  p.n_keep = 1;
+  p.st = &sc->st;
+  p.hist = sc->hist;
+  p.sure = sc->sure;
+  p.boundary = sc->boundary;
+  p.cap_sure = n_candidates;
+  p.cap_boundary = STRADS_STATIC_MAX_CANDIDATES / 2;
+  p.sm_count = sms;
+  return launch_sample(p, cand_dev, s) == cudaSuccess ? STRADS_OK : STRADS_ERR_CUDA;
+}
