@@ -237,12 +237,15 @@ def main():
     peaks = measured_peaks()
     step_ms = {k: prof[k] / max(prof["rounds"], 1) for k in ("sample_ms", "gram_ms", "filter_ms", "update_ms")}
     if p.layout == wl.DENSE:
-        flops = float(p.n_candidates) * (p.n_candidates - 1) * p.n_rows          # U'(U'-1) N, upper triangle
+        # algorithmic flops P'(P'-1)N (upper triangle, 2 flop per multiply-add); the kernel issues 3 TF32 MMAs per
+        # product (3xTF32), so the tensor pipe does 3x this -- `achieved` counts the algorithmic flops only
+        flops = float(p.n_candidates) * (p.n_candidates - 1) * p.n_rows
         achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
-        peak = SM_COUNT * FMA_LANES_PER_SM * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
-        roofline = {"kernel": "k_gram_dense_simt", "bound": "alu", "achieved": achieved, "peak": peak,
+        peak = peaks["bf16_tflops_sustained"] * 0.5          # TF32 dense = half the BF16 rate (nominal 1.1 vs 2.25 PF)
+        roofline = {"kernel": "k_gram_dense_tc", "bound": "tensor", "achieved": achieved, "peak": peak,
                     "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                    "peak_source": "148 SMs x 128 FP32 FMA lanes x 2 flop x max SM clock (derived)"}
+                    "tensor_issue_factor": 3,
+                    "peak_source": f"{peaks['source']} BF16 sustained x 0.5 (nominal TF32:BF16 ratio)"}
     else:
         nnz_col = p.nnz / p.n_cols
         byts = 8.0 * nnz_col * p.n_candidates

@@ -57,6 +57,11 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
 #define STRADS_FLAG_UNIFORM_DRAW  1u   /* p(j) uniform instead of delta_j^2 + eta (the random
                                           scheduler the paper compares with, Section 5.1)      */
 #define STRADS_FLAG_NO_FILTER     2u   /* skip the rho test: keep the first P candidates       */
+#define STRADS_FLAG_SIMT_GRAM     4u   /* dense Gram on the FP32 SIMT kernel instead of the
+                                          tensor-core kernels                                  */
+#define STRADS_FLAG_GRAM_3XTF32   8u   /* dense Gram always by the 3xTF32 tensor-core kernel
+                                          (default: TF32 screen + exact recheck of the pairs
+                                          within 2^-8 of rho; 3xTF32 only if those overflow)   */
 
 /* limits */
 #define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (one CTA sorts the winners in shared memory) */
@@ -92,8 +97,9 @@ typedef struct {
   int32_t* kept;      /* [P]  coefficients that passed the rho test, in walk order; -1 after n_kept */
   float*   dbeta;     /* [P]  signed change beta_j^(t_j) - beta_j^(t_j - 1) per kept entry; 0 after n_kept */
   int32_t* counts;    /* [4]  n_candidates, n_examined, n_kept, n_nonzero_changes          */
-  float*   gram;      /* [P'*P'] x_a^T x_b of all candidate pairs in candidate order;
-                         (debug aid: costs 4 P'^2 bytes of traffic per round)               */
+  float*   gram;      /* [P'*P'] x_a^T x_b of all candidate pairs in candidate order (debug aid:
+                         costs 4 P'^2 bytes of traffic per round; dense X then takes the FP32
+                         SIMT Gram kernel, which is the one that can export its values)      */
 } strads_round_out_t;
 
 /* Bytes of device workspace that `cfg` needs (pointer fields of cfg are not read). */
@@ -156,6 +162,8 @@ int strads_totals(strads_handle_t h, int64_t* totals_host_out /* [4] */);
 #define STRADS_STATUS_SAMPLER_REFINED 1u   /* informational: the sampler needed extra select passes */
 #define STRADS_STATUS_NONFINITE       2u   /* a gradient x_j^T r was NaN or Inf                     */
 #define STRADS_STATUS_WAIT_EXPIRED    4u   /* a bounded wait in a kernel gave up                     */
+#define STRADS_STATUS_GRAM_FALLBACK   8u   /* informational: the dense Gram's TF32 screen left more
+                                              borderline pairs than its list holds; 3xTF32 was used  */
 int strads_status(strads_handle_t h, uint32_t* bits_host_out);
 
 /* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */

@@ -19,6 +19,8 @@ LIB_PATH = os.path.join(_HERE, "libstrads_b200.so")
 OK = 0
 FLAG_UNIFORM_DRAW = 1
 FLAG_NO_FILTER = 2
+FLAG_SIMT_GRAM = 4
+FLAG_GRAM_3XTF32 = 8
 MAX_CANDIDATES = 16384
 
 EXPORTS = [

@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (no_filter) {
     const int nk = min(n_cand, p.n_keep);
     for (int i = tid; i < p.n_keep; i += kThreads) kept_out[i] = i < nk ? cand[i] : -1;
-    if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; }
+    if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; }
     return;
   }
 
@@ -106,7 +106,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   __syncthreads();
   const int nk = s_kept;
   for (int i = nk + tid; i < p.n_keep; i += kThreads) kept_out[i] = -1;
-  if (tid == 0) { p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; }
+  if (tid == 0) { p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; }
 }
 
 }  // namespace

@@ -1,0 +1,370 @@
+// SAP step 2, dense X, on the 5th-generation tensor cores: conflict bits of all candidate pairs from
+// G = X_C^T X_C, a genuine dense contraction (M = N' = P', K = the N samples).
+//
+// One CTA per 128 x 128 output tile of the upper triangle of tile pairs.  Accumulator: 128 lanes x 128
+// FP32 columns of tensor memory.  Operands: the candidate columns themselves, gathered through the
+// candidate list by four producer warps with 16-byte cp.async copies (zero-filled past N) straight
+// into the K-major 128-byte-swizzled layout tcgen05.mma reads: 128 bytes of K per row per stage, a ring
+// of stages handed back and forth with mbarriers (producers -> MMA: "full"; tcgen05.commit ->
+// producers: "empty").  A fifth warp's elected lane issues the MMAs.
+//
+// Two precisions of the same kernel:
+//   screen (default): one TF32 MMA per product on the raw FP32 bits (the tensor core uses the top 11
+//       significand bits of each input), 6 stages of 32 KB.  |G_tf32 - G| <= 2^-9 ||x_a|| ||x_b||
+//       whatever the data, so a pair whose |corr| is further than 2^-8 from rho is decided for
+//       certain; the few pairs inside that band are appended to a list and decided exactly by
+//       k_gram_recheck (FP64 dot product).  The decisions equal those of an exact Gram.
+//   3xTF32 (fallback, runs only if that list overflows): the producers also split every operand into
+//       hi + lo TF32 parts, G ~= lo.hi + hi.lo + hi.hi, 3 stages of 64 KB.
+// Epilogue: the producer warps read the accumulator back with tcgen05.ld, threshold in FP64 and write
+// one 32-bit mask word per row and 32 columns.
+//
+// Every wait has an iteration limit; on expiry the CTA raises STRADS_STATUS_WAIT_EXPIRED, stops issuing
+// work, and still frees its tensor memory.
+#include "strads_internal.cuh"
+
+namespace strads {
+namespace {
+
+constexpr int kTile = 128;                 // rows and columns of the output tile
+constexpr int kBlockK = 32;                // floats of K per stage = one 128-byte swizzle row
+constexpr int kTileBytes = kTile * 128;    // 16 KB: 128 rows x 128 bytes
+constexpr int kProducerWarps = 4;
+constexpr int kThreads = 32 * (kProducerWarps + 1);
+constexpr uint32_t kWaitLimit = 1u << 24;
+constexpr uint32_t kTmemCols = 128;
+constexpr size_t kRingBytes = 192 * 1024;
+constexpr size_t kDynSmem = kRingBytes + 1024;
+// Half-width of the "too close to call" band of the screen, relative to ||x_a|| ||x_b||: input
+// truncation costs at most 2^-9 (two operands, 11 significand bits each, Cauchy-Schwarz on the sum),
+// the N/8 FP32 accumulator updates at most 2^-23 each; doubled for margin.
+__device__ __forceinline__ double screen_band(long long N) { return 1.0 / 256.0 + (double)N * (1.0 / 33554432.0); }
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait for the phase with the given parity; false = gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    if (ok) return true;
+  }
+  return false;
+}
+
+// Shared-memory matrix descriptor: K-major, 128-byte swizzle, rows of 128 bytes, 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4)        // start address / 16
+         | ((uint64_t)1 << 16)                       // leading byte offset / 16 (unused for swizzled K-major)
+         | ((uint64_t)(1024 >> 4) << 32)             // stride byte offset / 16
+         | ((uint64_t)1 << 46)                       // descriptor version of this architecture
+         | ((uint64_t)2 << 61);                      // 128-byte swizzle
+}
+
+// D[tmem] (+)= A[smem] * B[smem]^T, TF32 inputs, FP32 accumulate, M = N = 128, K = 8.
+__device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_load32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// 16 bytes global -> shared, asynchronously; only the first `bytes` (0, 4, 8, 12 or 16) are read, the rest is zero.
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, uint32_t bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// x = hi + lo with hi the top 11 significand bits of x (what a TF32 MMA reads of x); lo again cut to TF32.
+__device__ __forceinline__ float tf32_lo(float x) {
+  const float hi = __uint_as_float(__float_as_uint(x) & 0xffffe000u);
+  return __uint_as_float(__float_as_uint(x - hi) & 0xffffe000u);
+}
+
+template <bool k3x>
+__global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const int* __restrict__ cand, int n_cand,
+                                                                int n_tiles) {
+  constexpr int kStageBytes = (k3x ? 4 : 2) * kTileBytes;       // raw A, raw B [, lo A, lo B]
+  constexpr int kStages = (int)(kRingBytes / kStageBytes);      // 3 or 6
+  constexpr int kAhead = kStages - 1;                           // k-blocks in flight per producer thread
+
+  extern __shared__ unsigned char dyn_smem[];
+  __shared__ __align__(8) unsigned long long bars[2 * kStages + 1];   // full[], empty[], accumulator done
+  __shared__ uint32_t s_tmem_base;
+  __shared__ volatile int s_abort;
+  __shared__ int idxA[kTile], idxB[kTile];
+  __shared__ double n2B[kTile];
+
+  // as a fallback the 3xTF32 variant runs only when the screen's list overflowed
+  if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && p.st->amb_count <= (unsigned)p.cap_amb) return;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && blockIdx.x == 0 && tid == 0)
+    atomicOr(&p.st->status, STRADS_STATUS_GRAM_FALLBACK);
+  int ti = 0, rem = blockIdx.x;                        // linear index -> (ti, tj), ti <= tj
+  while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
+  const int tj = ti + rem;
+
+  const uint32_t tiles0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;      // swizzle atoms need 1024-byte alignment
+  unsigned char* tiles_ptr = dyn_smem + (tiles0 - smem_u32(dyn_smem));
+  const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[kStages]), done_bar = smem_u32(&bars[2 * kStages]);
+
+  if (tid < kTile) {
+    const int ga = ti * kTile + tid, gb = tj * kTile + tid;
+    idxA[tid] = ga < n_cand ? cand[ga] : -1;
+    idxB[tid] = gb < n_cand ? cand[gb] : -1;
+    n2B[tid] = gb < n_cand ? p.n2[cand[gb]] : 0.0;
+  }
+  if (tid == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, kProducerWarps); mbar_init(empty0 + 8 * s, 1); }
+    mbar_init(done_bar, 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == kProducerWarps) {                        // the MMA warp owns the tensor-memory allocation
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
+                 "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = s_tmem_base;
+
+  const long long N = p.N;
+  const int n_kb = (int)((N + kBlockK - 1) / kBlockK);
+
+  if (warp < kProducerWarps) {
+    // ------------------------------ producers ------------------------------
+    const int chunk = lane & 7;                        // which 16 bytes of the 128-byte row
+    const int rsub = lane >> 3;                        // 4 rows per warp-wide copy
+    // per thread: 8 rows of A and the same 8 rows of B, always the same chunk
+    const float* srcA[8];
+    const float* srcB[8];
+    uint32_t dst_off[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int row = warp * 32 + i * 4 + rsub;
+      srcA[i] = idxA[row] >= 0 ? p.xv + (long long)idxA[row] * p.ld : nullptr;
+      srcB[i] = idxB[row] >= 0 ? p.xv + (long long)idxB[row] * p.ld : nullptr;
+      dst_off[i] = (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
+    }
+    auto issue = [&](int kb) {                         // all copies of one k-block, one commit group
+      const int s = kb % kStages;
+      const long long k = (long long)kb * kBlockK + chunk * 4;
+      const long long left = N - k;                    // floats of this chunk that exist
+      const uint32_t bytes = left >= 4 ? 16u : (left > 0 ? (uint32_t)left * 4u : 0u);
+      const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        cp_async16(sb + dst_off[i], srcA[i] ? (const void*)(srcA[i] + (bytes ? k : 0)) : (const void*)p.xv,
+                   srcA[i] ? bytes : 0u);
+        cp_async16(sb + kTileBytes + dst_off[i], srcB[i] ? (const void*)(srcB[i] + (bytes ? k : 0)) : (const void*)p.xv,
+                   srcB[i] ? bytes : 0u);
+      }
+    };
+    // prologue: the ring is empty, fill kAhead stages
+    for (int kb = 0; kb < kAhead; ++kb) {
+      if (kb < n_kb) issue(kb);
+      cp_async_commit();
+    }
+    for (int kb = 0; kb < n_kb; ++kb) {
+      const int s = kb % kStages;
+      cp_async_wait<kAhead - 1>();                     // this thread's copies of k-block kb have landed
+      if (k3x) {                                       // split: the raw tile stays as "hi", write the "lo" tiles
+        unsigned char* st = tiles_ptr + (size_t)s * kStageBytes;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          float4 a = *reinterpret_cast<const float4*>(st + dst_off[i]);
+          float4 b = *reinterpret_cast<const float4*>(st + kTileBytes + dst_off[i]);
+          a.x = tf32_lo(a.x); a.y = tf32_lo(a.y); a.z = tf32_lo(a.z); a.w = tf32_lo(a.w);
+          b.x = tf32_lo(b.x); b.y = tf32_lo(b.y); b.z = tf32_lo(b.z); b.w = tf32_lo(b.w);
+          *reinterpret_cast<float4*>(st + 2 * kTileBytes + dst_off[i]) = a;
+          *reinterpret_cast<float4*>(st + 3 * kTileBytes + dst_off[i]) = b;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes -> visible to the MMA's reads
+      __syncwarp();
+      if (lane == 0) mbar_arrive(full0 + 8 * s);
+      // refill: k-block kb + kAhead goes into the stage that k-block kb - 1 used
+      const int nxt = kb + kAhead;
+      if (nxt < n_kb) {
+        bool got = !s_abort;
+        if (got && nxt >= kStages) got = mbar_wait(empty0 + 8 * (nxt % kStages), (uint32_t)(nxt / kStages - 1) & 1u);
+        if (!__all_sync(0xffffffffu, got)) {
+          if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+          break;
+        }
+        issue(nxt);
+      }
+      cp_async_commit();
+    }
+    cp_async_wait<0>();
+  } else {
+    // ------------------------------ MMA issuer (whole warp waits, one lane issues) ------------------------------
+    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+    uint32_t acc = 0;
+    for (int kb = 0; kb < n_kb; ++kb) {
+      const int s = kb % kStages;
+      const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+      const bool got = !s_abort && mbar_wait(full0 + 8 * s, ph);
+      if (!__all_sync(0xffffffffu, got)) {
+        if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+        break;
+      }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (lane == 0) {
+        const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes;
+        const uint64_t a_hi = umma_desc(sb), b_hi = umma_desc(sb + kTileBytes);
+#pragma unroll
+        for (int k8 = 0; k8 < kBlockK / 8; ++k8) {     // K = 8 per instruction: 32 bytes along the swizzled row
+          const uint64_t o = (uint64_t)(k8 * 2);
+          if (k3x) {
+            const uint64_t a_lo = umma_desc(sb + 2 * kTileBytes), b_lo = umma_desc(sb + 3 * kTileBytes);
+            umma_tf32(tmem_base, a_lo + o, b_hi + o, idesc, acc);
+            umma_tf32(tmem_base, a_hi + o, b_lo + o, idesc, 1u);
+            umma_tf32(tmem_base, a_hi + o, b_hi + o, idesc, 1u);
+          } else {
+            umma_tf32(tmem_base, a_hi + o, b_hi + o, idesc, acc);
+          }
+          acc = 1;
+        }
+        umma_commit(empty0 + 8 * s);                   // frees the stage when these MMAs have read it
+      }
+      __syncwarp();
+    }
+    if (lane == 0) umma_commit(done_bar);              // accumulator complete
+    __syncwarp();
+  }
+
+  // ------------------------------ epilogue (warps 0..3: TMEM lanes 32 w .. 32 w + 31) ------------------------------
+  if (warp < kProducerWarps) {
+    bool ok = !s_abort && mbar_wait(done_bar, 0u);
+    ok = __all_sync(0xffffffffu, ok);
+    if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (ok) {
+      const int la = warp * 32 + lane;
+      const int a = ti * kTile + la;
+      const double n2a = a < n_cand ? p.n2[idxA[la]] : 0.0;
+      const double rho = (double)p.rho;
+      const double band = screen_band(N);
+#pragma unroll 1
+      for (int c = 0; c < kTile / 32; ++c) {
+        uint32_t v[32];
+        tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
+        uint32_t word = 0u;
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const int lb = c * 32 + j;
+          const int b = tj * kTile + lb;
+          const double den = sqrt(n2a * n2B[lb]);
+          const double g = fabs((double)__uint_as_float(v[j]));
+          const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
+          bool hit = live && g >= rho * den;
+          if (!k3x && live && b > a && fabs(g - rho * den) <= band * den) {
+            // too close to call in TF32: leave the bit clear and let k_gram_recheck decide exactly
+            hit = false;
+            const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
+            if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
+          }
+          word |= (uint32_t)hit << j;
+        }
+        const int widx = tj * (kTile / 32) + c;
+        if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+      }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  }
+  __syncthreads();
+  if (warp == kProducerWarps) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product.
+// Setting a bit is idempotent and order-independent, so the result is deterministic.
+__global__ void __launch_bounds__(256) k_gram_recheck(Problem p, const int* __restrict__ cand) {
+  const unsigned int n = p.st->amb_count;
+  if (n > (unsigned)p.cap_amb) return;                 // overflow: the 3xTF32 kernel redoes every bit instead
+  const int lane = threadIdx.x & 31;
+  const unsigned int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const unsigned int n_warps = (gridDim.x * blockDim.x) >> 5;
+  const long long n4 = (p.N + 3) >> 2;
+  for (unsigned int e = warp; e < n; e += n_warps) {
+    const unsigned int pr = p.amb_pairs[e];
+    const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
+    const int ja = cand[a], jb = cand[b];
+    const float4* xa = reinterpret_cast<const float4*>(p.xv + (long long)ja * p.ld);
+    const float4* xb = reinterpret_cast<const float4*>(p.xv + (long long)jb * p.ld);
+    double acc = 0.0;
+    for (long long g = lane; g < n4; g += 32) {
+      const float4 u = __ldg(xa + g), w = __ldg(xb + g);
+      const long long i = g << 2;
+      acc += (double)u.x * w.x;
+      if (i + 1 < p.N) acc += (double)u.y * w.y;
+      if (i + 2 < p.N) acc += (double)u.z * w.z;
+      if (i + 3 < p.N) acc += (double)u.w * w.w;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+    if (lane == 0) {
+      const double den = sqrt(p.n2[ja] * p.n2[jb]);
+      if (den > 0.0 && fabs(acc) >= (double)p.rho * den)
+        atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+    }
+  }
+}
+
+}  // namespace
+
+cudaError_t prepare_gram_dense_tc() {
+  cudaError_t e = cudaFuncSetAttribute(k_gram_dense_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+}
+
+// screen -> exact recheck of the borderline pairs -> (only if their list overflowed) 3xTF32 over everything
+cudaError_t launch_gram_dense_tc(const Problem& p, const int* cand, int n_cand, cudaStream_t s) {
+  const int n_tiles = (n_cand + kTile - 1) / kTile;
+  const int blocks = n_tiles * (n_tiles + 1) / 2;
+  if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
+    k_gram_dense_tc<false><<<blocks, kThreads, kDynSmem, s>>>(p, cand, n_cand, n_tiles);
+    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(p, cand);
+  }
+  k_gram_dense_tc<true><<<blocks, kThreads, kDynSmem, s>>>(p, cand, n_cand, n_tiles);
+  return cudaGetLastError();
+}
+
+}  // namespace strads

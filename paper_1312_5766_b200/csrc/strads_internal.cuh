@@ -29,6 +29,8 @@ struct DeviceState {
   double objective;             // result slot of the objective reduction
   float x_abs_max;              // max |x_ij| (CSC: bounds the fixed-point residual update)
   int beta0_nonzero;            // set at init when the starting beta has a non-zero entry
+  unsigned int amb_count;       // pairs the TF32 screen of the dense Gram left to the exact recheck
+  unsigned int pad[3];
 };
 
 static constexpr int kHistBits = 12;
@@ -66,6 +68,8 @@ struct Problem {
   unsigned int* dot_ticket;     // [n_keep]
   int dot_parts;
   double* obj_partial;          // [2 * kObjBlocks]
+  unsigned int* amb_pairs;      // [cap_amb] (a << 16 | b), positions in the candidate list
+  int cap_amb;
   int sm_count;
 };
 static constexpr int kObjBlocks = 296;
@@ -145,6 +149,8 @@ cudaError_t launch_objective(const Problem& p, cudaStream_t s);
 cudaError_t prepare_sample(const Problem& p);
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
+cudaError_t prepare_gram_dense_tc();
+cudaError_t launch_gram_dense_tc(const Problem& p, const int* cand, int n_cand, cudaStream_t s);
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s);

@@ -357,3 +357,66 @@ def test_degenerate_sizes():
     cand, kept, dbeta, counts = s.round()
     assert counts.cpu().tolist() == [3, 3, 3, 1] and sorted(kept.tolist()) == [0, 1, 2]
     assert s.beta.cpu().tolist()[0] == 0.0 and s.beta.cpu().tolist()[2] == 0.0 and s.status() == (0, 0)
+
+
+# --------------------------------------------------------------------------------------------------
+# tensor-core Gram (3xTF32, tcgen05) against the oracle and against the FP32 SIMT kernel
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("cfg", [
+    dict(kind="dense_iid", n_rows=1000, n_cols=3000, n_true=30, lam_frac=0.05, n_candidates=300, n_keep=300, rho=0.1),
+    dict(kind="dense_grouped", n_rows=2000, n_cols=2000, n_true=20, lam_frac=0.02, n_candidates=640, n_keep=640,
+         rho=0.1, group=20),
+    dict(kind="dense_iid", n_rows=1003, n_cols=900, n_true=10, lam_frac=0.05, n_candidates=131, n_keep=131, rho=0.05),
+    dict(kind="dense_iid", n_rows=24, n_cols=600, n_true=5, lam_frac=0.05, n_candidates=513, n_keep=513, rho=0.3),
+])
+def test_tensor_core_gram_decisions(cfg):
+    b = _binding()
+    p = wl.make_problem(cfg, seed=12)
+    ld = (p.n_rows + 3) // 4 * 4
+    vals = torch.full((p.n_cols, ld), float("nan"))
+    vals[:, : p.n_rows] = p.values
+    X = oracle_matrix(p)
+    n2 = oracle.colnorm2(X)
+    rho = float(np.float32(p.rho))
+    mk = lambda flags: b.StradsLasso(wl.DENSE, p.n_rows, p.n_cols, vals.cuda(), p.y.cuda(), p.lam, p.eta, p.rho,
+                                     p.n_candidates, p.n_keep, seed=p.seed, flags=flags)
+    tc, simt, tc3 = mk(0), mk(b.FLAG_SIMT_GRAM), mk(b.FLAG_GRAM_3XTF32)
+    rng = np.random.default_rng(5)
+    for trial in range(3):
+        cand = rng.permutation(p.n_cols)[: p.n_candidates].astype(np.int32)
+        if cfg["kind"] == "dense_grouped" and trial == 0:
+            cand = np.arange(p.n_candidates, dtype=np.int32)
+        cd = torch.from_numpy(cand).cuda()
+        kept_tc, counts_tc = tc.filter(cd)
+        c = counts_tc.cpu().numpy(); nk = int(c[2])
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept_tc.cpu().numpy()[:nk], int(c[1]))
+        kept_s, counts_s = simt.filter(cd)
+        assert torch.equal(kept_tc, kept_s) and torch.equal(counts_tc, counts_s)
+        kept_3, counts_3 = tc3.filter(cd)
+        assert torch.equal(kept_tc, kept_3) and torch.equal(counts_tc, counts_3)
+    assert tc.status() == (0, 0) and tc3.status() == (0, 0)
+
+
+def test_tensor_core_screen_overflow_falls_back_to_3xtf32():
+    # every pair correlates at ~rho: x_j = sqrt(rho) z + sqrt(1 - rho) e_j, so hundreds of thousands of pairs
+    # fall inside the screen's "too close to call" band and its list overflows
+    b = _binding()
+    N, J, rho = 12_000, 1536, 0.25
+    g = torch.Generator().manual_seed(3)
+    z = torch.randn(N, generator=g)
+    x = (rho ** 0.5) * z[None, :] + ((1 - rho) ** 0.5) * torch.randn((J, N), generator=g)
+    x -= x.mean(dim=1, keepdim=True)
+    x /= x.norm(dim=1, keepdim=True)
+    y = torch.randn(N, generator=g)
+    mk = lambda flags: b.StradsLasso(wl.DENSE, N, J, x.cuda(), y.cuda(), 0.1, 1e-6, rho, J, 64, seed=0, flags=flags)
+    tc, simt = mk(0), mk(b.FLAG_SIMT_GRAM)
+    cand = torch.randperm(J, generator=g).to(torch.int32).cuda()
+    kept_tc, counts_tc = tc.filter(cand)
+    kept_s, counts_s = simt.filter(cand)
+    X = oracle.Matrix.dense(x.numpy())
+    n2 = oracle.colnorm2(X)
+    c = counts_tc.cpu().numpy(); nk = int(c[2])
+    _assert_kept_matches(X, n2, cand.cpu().numpy(), 64, float(np.float32(rho)), kept_tc.cpu().numpy()[:nk], int(c[1]))
+    # the two FP32-accurate kernels may differ only on pairs within 1e-6 of rho; on this data they agree
+    assert torch.equal(kept_tc, kept_s) and torch.equal(counts_tc, counts_s)
+    assert tc.status() == (0, 8)                     # informational bit: the fallback did run
