@@ -11,6 +11,7 @@
 using namespace strads;
 
 struct strads_lasso_s {
+  alignas(64) unsigned char gram_tmap[128];   // tensor map over the packed candidate buffer (dense layouts)
   Problem p;
   cudaStream_t stream;
   int device;
@@ -39,8 +40,9 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_dbeta, off_dbeta64,
-      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, total;
+      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb;
+  long long ldc;
 };
 
 // Checks everything about cfg that does not need its pointers.
@@ -82,6 +84,8 @@ Layout carve(const strads_lasso_config_t* c) {
   L.off_obj = take(sizeof(double) * 2 * kObjBlocks);
   L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // borderline pairs of the TF32 screen (1 MB)
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
+  L.ldc = (c->n_rows + 3) / 4 * 4;
+  L.off_xc = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(float) * (size_t)c->n_candidates * L.ldc : 0);
   L.total = o;
   return L;
 }
@@ -90,16 +94,18 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
-cudaError_t launch_gram(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s) {
+cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg) {
+  const Problem& p = h->p;
+  cudaStream_t s = h->stream;
   if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, cand, n_cand, s);
+  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, s);
 }
 
 int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg) {
   const Problem& p = h->p;
   if (!(p.flags & STRADS_FLAG_NO_FILTER)) {
-    CK(launch_gram(p, cand, n_cand, gram_dbg, h->stream));
+    CK(launch_gram(h, cand, n_cand, gram_dbg));
   }
   CK(launch_filter(p, cand, n_cand, p.kept, h->stream));
   return STRADS_OK;
@@ -111,7 +117,7 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
   if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
   if (ev) CK(cudaEventRecord(ev[1], h->stream));
-  if (!(p.flags & STRADS_FLAG_NO_FILTER)) CK(launch_gram(p, p.cand, p.n_cand, out ? out->gram : nullptr, h->stream));
+  if (!(p.flags & STRADS_FLAG_NO_FILTER)) CK(launch_gram(h, p.cand, p.n_cand, out ? out->gram : nullptr));
   if (ev) CK(cudaEventRecord(ev[2], h->stream));
   CK(launch_filter(p, p.cand, p.n_cand, p.kept, h->stream));
   if (ev) CK(cudaEventRecord(ev[3], h->stream));
@@ -179,6 +185,9 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   p.obj_partial = reinterpret_cast<double*>(ws + L.off_obj);
   p.amb_pairs = reinterpret_cast<unsigned int*>(ws + L.off_amb);
   p.cap_amb = L.cap_amb;
+  p.xc = reinterpret_cast<float*>(ws + L.off_xc);
+  p.ldc = L.ldc;
+  p.cand_cur = nullptr;
   h->stream = static_cast<cudaStream_t>(c->stream);
   h->round_host = 0;
   h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
@@ -191,6 +200,8 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   if ((e = prepare_sample(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_sample"));
   if ((e = prepare_filter(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_filter"));
   if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
+  if (p.layout == STRADS_DENSE_COLMAJOR && (e = encode_gram_tensor_map(p, h->gram_tmap)) != cudaSuccess)
+    return fail(cuda_fail(e, "encode_gram_tensor_map"));
   if ((e = launch_init(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
   if ((e = launch_resid_from_beta(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
   *out_handle = h;

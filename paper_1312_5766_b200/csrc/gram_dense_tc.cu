@@ -1,36 +1,39 @@
 // SAP step 2, dense X, on the 5th-generation tensor cores: conflict bits of all candidate pairs from
 // G = X_C^T X_C, a genuine dense contraction (M = N' = P', K = the N samples).
 //
-// One CTA per 128 x 128 output tile of the upper triangle of tile pairs.  Accumulator: 128 lanes x 128
-// FP32 columns of tensor memory.  Operands: the candidate columns themselves, gathered through the
-// candidate list by four producer warps with 16-byte cp.async copies (zero-filled past N) straight
-// into the K-major 128-byte-swizzled layout tcgen05.mma reads: 128 bytes of K per row per stage, a ring
-// of stages handed back and forth with mbarriers (producers -> MMA: "full"; tcgen05.commit ->
-// producers: "empty").  A fifth warp's elected lane issues the MMAs.
-//
-// Two precisions of the same kernel:
-//   screen (default): one TF32 MMA per product on the raw FP32 bits (the tensor core uses the top 11
-//       significand bits of each input), 6 stages of 32 KB.  |G_tf32 - G| <= 2^-9 ||x_a|| ||x_b||
-//       whatever the data, so a pair whose |corr| is further than 2^-8 from rho is decided for
-//       certain; the few pairs inside that band are appended to a list and decided exactly by
-//       k_gram_recheck (FP64 dot product).  The decisions equal those of an exact Gram.
-//   3xTF32 (fallback, runs only if that list overflows): the producers also split every operand into
-//       hi + lo TF32 parts, G ~= lo.hi + hi.lo + hi.hi, 3 stages of 64 KB.
-// Epilogue: the producer warps read the accumulator back with tcgen05.ld, threshold in FP64 and write
-// one 32-bit mask word per row and 32 columns.
+//   k_pack_candidates   copies the P' candidate columns into one contiguous [P'][ldc] buffer.  The
+//                       candidates are scattered over the whole design matrix (one 2 MB page each for a
+//                       4 GB X); gathering them once makes every later access TLB- and TMA-friendly
+//                       (measured: the same GEMM runs 2x slower straight from scattered columns).
+//   k_gram_dense_tc<0>  "screen": one CTA per 128 x 128 tile of the upper triangle of tile pairs; one
+//                       thread feeds a 3-stage ring of 64 KB stages with TMA tile loads (128-byte
+//                       swizzle, zero fill past N and P'), one thread issues tcgen05.mma kind::tf32
+//                       on the raw FP32 bits into a 128 x 128 FP32 accumulator in tensor memory, four
+//                       warps read it back with tcgen05.ld, threshold in FP64 and write mask words.
+//                       A single-pass TF32 correlation is within 2^-9 of the exact one whatever the
+//                       data, so pairs further than the band from rho are decided for certain; the few
+//                       inside the band go to a list ...
+//   k_gram_recheck      ... and are decided exactly (FP64 dot product), so the decisions equal those of
+//                       an exact Gram.
+//   k_gram_dense_tc<1>  3xTF32 fallback, runs only if that list overflows (or on request): producer
+//                       warps copy with cp.async and split every operand into hi + lo TF32 parts,
+//                       G ~= lo.hi + hi.lo + hi.hi.
 //
 // Every wait has an iteration limit; on expiry the CTA raises STRADS_STATUS_WAIT_EXPIRED, stops issuing
-// work, and still frees its tensor memory.
+// work, and still frees its tensor memory.  No multicast anywhere.
+#include <cuda.h>
+
 #include "strads_internal.cuh"
 
 namespace strads {
 namespace {
 
 constexpr int kTile = 128;                 // rows and columns of the output tile
-constexpr int kBlockK = 32;                // floats of K per stage = one 128-byte swizzle row
+constexpr int kBlockK = 32;                // floats of K per sub-block = one 128-byte swizzle row
 constexpr int kTileBytes = kTile * 128;    // 16 KB: 128 rows x 128 bytes
-constexpr int kProducerWarps = 4;
-constexpr int kThreads = 32 * (kProducerWarps + 1);
+constexpr int kProducerWarps = 4;          // epilogue warps; also the cp.async producers of the 3xTF32 variant
+constexpr int kMmaWarp = 4, kTmaWarp = 5;
+constexpr int kThreads = 32 * 6;
 constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr uint32_t kTmemCols = 128;
 constexpr size_t kRingBytes = 192 * 1024;
@@ -47,6 +50,15 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+// One TMA tile load: box {32 floats, 128 rows} at element coordinates (x = k, y = row) -> shared memory.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 // Bounded wait for the phase with the given parity; false = gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
@@ -111,19 +123,31 @@ __device__ __forceinline__ float tf32_lo(float x) {
   return __uint_as_float(__float_as_uint(x - hi) & 0xffffe000u);
 }
 
+// One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).
+__global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand) {
+  const int a = blockIdx.x;
+  if (a >= n_cand) return;
+  const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)cand[a] * p.ld);
+  float4* dst = reinterpret_cast<float4*>(p.xc + (long long)a * p.ldc);
+  const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
+  for (long long g = threadIdx.x; g < n4; g += blockDim.x) dst[g] = __ldg(src + g);
+}
+
 template <bool k3x>
-__global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const int* __restrict__ cand, int n_cand,
-                                                                int n_tiles) {
-  constexpr int kStageBytes = (k3x ? 4 : 2) * kTileBytes;       // raw A, raw B [, lo A, lo B]
-  constexpr int kStages = (int)(kRingBytes / kStageBytes);      // 3 or 6
-  constexpr int kAhead = kStages - 1;                           // k-blocks in flight per producer thread
+__global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const __grid_constant__ CUtensorMap tmap,
+                                                                int n_cand, int n_tiles) {
+  // A stage holds kSub sub-blocks of 32 floats of K for A, the same for B [3xTF32: plus the two lo tiles].
+  constexpr int kSub = k3x ? 1 : 2;
+  constexpr int kStageBytes = (k3x ? 4 : 2 * kSub) * kTileBytes;       // 64 KB either way
+  constexpr int kStages = (int)(kRingBytes / kStageBytes);             // 3
+  constexpr int kAhead = kStages - 1;                                  // 3xTF32: stages in flight per producer thread
+  constexpr uint32_t kFullCount = k3x ? kProducerWarps : 1;            // arrivals that complete "full"
 
   extern __shared__ unsigned char dyn_smem[];
   __shared__ __align__(8) unsigned long long bars[2 * kStages + 1];   // full[], empty[], accumulator done
   __shared__ uint32_t s_tmem_base;
   __shared__ volatile int s_abort;
-  __shared__ int idxA[kTile], idxB[kTile];
-  __shared__ double n2B[kTile];
+  __shared__ double normA[kTile], normB[kTile];                        // ||x|| of the tile's rows / columns
 
   // as a fallback the 3xTF32 variant runs only when the screen's list overflowed
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && p.st->amb_count <= (unsigned)p.cap_amb) return;
@@ -141,17 +165,16 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 
   if (tid < kTile) {
     const int ga = ti * kTile + tid, gb = tj * kTile + tid;
-    idxA[tid] = ga < n_cand ? cand[ga] : -1;
-    idxB[tid] = gb < n_cand ? cand[gb] : -1;
-    n2B[tid] = gb < n_cand ? p.n2[cand[gb]] : 0.0;
+    normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
+    normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
   }
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, kProducerWarps); mbar_init(empty0 + 8 * s, 1); }
+    for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, kFullCount); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(done_bar, 1);
     s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == kProducerWarps) {                        // the MMA warp owns the tensor-memory allocation
+  if (warp == kMmaWarp) {                              // the MMA warp owns the tensor-memory allocation
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&s_tmem_base)),
                  "r"(kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -162,63 +185,79 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const uint32_t tmem_base = s_tmem_base;
 
   const long long N = p.N;
-  const int n_kb = (int)((N + kBlockK - 1) / kBlockK);
+  const int n_st = (int)((N + (long long)kBlockK * kSub - 1) / ((long long)kBlockK * kSub));   // stages of K
 
-  if (warp < kProducerWarps) {
-    // ------------------------------ producers ------------------------------
+  if (!k3x && warp == kTmaWarp) {
+    // ------------------------------ screen: TMA producer (one lane) ------------------------------
+    for (int st = 0; st < n_st; ++st) {
+      const int s = st % kStages;
+      bool got = !s_abort;
+      if (got && st >= kStages) got = mbar_wait(empty0 + 8 * s, (uint32_t)(st / kStages - 1) & 1u);
+      if (!__all_sync(0xffffffffu, got)) {
+        if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+        break;
+      }
+      if (lane == 0) {
+        const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes, bar = full0 + 8 * s;
+        mbar_arrive_expect_tx(bar, (uint32_t)kStageBytes);
+#pragma unroll
+        for (int sub = 0; sub < kSub; ++sub) {
+          const int k = (st * kSub + sub) * kBlockK;    // past N the whole box is zero-filled
+          tma_load_2d(sb + sub * kTileBytes, &tmap, k, ti * kTile, bar);
+          tma_load_2d(sb + (kSub + sub) * kTileBytes, &tmap, k, tj * kTile, bar);
+        }
+      }
+      __syncwarp();
+    }
+  } else if (k3x && warp < kProducerWarps) {
+    // ------------------------------ 3xTF32: cp.async producers that also split hi / lo ------------------------------
     const int chunk = lane & 7;                        // which 16 bytes of the 128-byte row
     const int rsub = lane >> 3;                        // 4 rows per warp-wide copy
-    // per thread: 8 rows of A and the same 8 rows of B, always the same chunk
     const float* srcA[8];
     const float* srcB[8];
     uint32_t dst_off[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int row = warp * 32 + i * 4 + rsub;
-      srcA[i] = idxA[row] >= 0 ? p.xv + (long long)idxA[row] * p.ld : nullptr;
-      srcB[i] = idxB[row] >= 0 ? p.xv + (long long)idxB[row] * p.ld : nullptr;
+      const int ga = ti * kTile + row, gb = tj * kTile + row;
+      srcA[i] = ga < n_cand ? p.xc + (long long)ga * p.ldc : nullptr;
+      srcB[i] = gb < n_cand ? p.xc + (long long)gb * p.ldc : nullptr;
       dst_off[i] = (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
     }
-    auto issue = [&](int kb) {                         // all copies of one k-block, one commit group
-      const int s = kb % kStages;
-      const long long k = (long long)kb * kBlockK + chunk * 4;
+    auto issue = [&](int st) {                         // all copies of one stage
+      const uint32_t sb = tiles0 + (uint32_t)(st % kStages) * kStageBytes;
+      const long long k = (long long)st * kBlockK + chunk * 4;
       const long long left = N - k;                    // floats of this chunk that exist
       const uint32_t bytes = left >= 4 ? 16u : (left > 0 ? (uint32_t)left * 4u : 0u);
-      const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        cp_async16(sb + dst_off[i], srcA[i] ? (const void*)(srcA[i] + (bytes ? k : 0)) : (const void*)p.xv,
+        cp_async16(sb + dst_off[i], srcA[i] ? (const void*)(srcA[i] + (bytes ? k : 0)) : (const void*)p.xc,
                    srcA[i] ? bytes : 0u);
-        cp_async16(sb + kTileBytes + dst_off[i], srcB[i] ? (const void*)(srcB[i] + (bytes ? k : 0)) : (const void*)p.xv,
+        cp_async16(sb + kTileBytes + dst_off[i], srcB[i] ? (const void*)(srcB[i] + (bytes ? k : 0)) : (const void*)p.xc,
                    srcB[i] ? bytes : 0u);
       }
     };
-    // prologue: the ring is empty, fill kAhead stages
-    for (int kb = 0; kb < kAhead; ++kb) {
-      if (kb < n_kb) issue(kb);
+    for (int st = 0; st < kAhead; ++st) {              // prologue: the ring is empty, fill kAhead stages
+      if (st < n_st) issue(st);
       cp_async_commit();
     }
-    for (int kb = 0; kb < n_kb; ++kb) {
-      const int s = kb % kStages;
-      cp_async_wait<kAhead - 1>();                     // this thread's copies of k-block kb have landed
-      if (k3x) {                                       // split: the raw tile stays as "hi", write the "lo" tiles
-        unsigned char* st = tiles_ptr + (size_t)s * kStageBytes;
+    for (int st = 0; st < n_st; ++st) {
+      const int s = st % kStages;
+      cp_async_wait<kAhead - 1>();                     // this thread's copies of stage st have landed
+      unsigned char* sp = tiles_ptr + (size_t)s * kStageBytes;
 #pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          float4 a = *reinterpret_cast<const float4*>(st + dst_off[i]);
-          float4 b = *reinterpret_cast<const float4*>(st + kTileBytes + dst_off[i]);
-          a.x = tf32_lo(a.x); a.y = tf32_lo(a.y); a.z = tf32_lo(a.z); a.w = tf32_lo(a.w);
-          b.x = tf32_lo(b.x); b.y = tf32_lo(b.y); b.z = tf32_lo(b.z); b.w = tf32_lo(b.w);
-          *reinterpret_cast<float4*>(st + 2 * kTileBytes + dst_off[i]) = a;
-          *reinterpret_cast<float4*>(st + 3 * kTileBytes + dst_off[i]) = b;
-        }
+      for (int i = 0; i < 8; ++i) {                    // the raw tile stays as "hi", write the "lo" tiles
+        float4 a = *reinterpret_cast<const float4*>(sp + dst_off[i]);
+        float4 b = *reinterpret_cast<const float4*>(sp + kTileBytes + dst_off[i]);
+        a.x = tf32_lo(a.x); a.y = tf32_lo(a.y); a.z = tf32_lo(a.z); a.w = tf32_lo(a.w);
+        b.x = tf32_lo(b.x); b.y = tf32_lo(b.y); b.z = tf32_lo(b.z); b.w = tf32_lo(b.w);
+        *reinterpret_cast<float4*>(sp + 2 * kTileBytes + dst_off[i]) = a;
+        *reinterpret_cast<float4*>(sp + 3 * kTileBytes + dst_off[i]) = b;
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // these writes -> visible to the MMA's reads
       __syncwarp();
-      if (lane == 0) mbar_arrive(full0 + 8 * s);
-      // refill: k-block kb + kAhead goes into the stage that k-block kb - 1 used
-      const int nxt = kb + kAhead;
-      if (nxt < n_kb) {
+      if (lane == 0) mbar_arrive(full0 + 8 * s);      // release: this warp's part of the stage is ready
+      const int nxt = st + kAhead;                     // refill the stage that st - 1 used
+      if (nxt < n_st) {
         bool got = !s_abort;
         if (got && nxt >= kStages) got = mbar_wait(empty0 + 8 * (nxt % kStages), (uint32_t)(nxt / kStages - 1) & 1u);
         if (!__all_sync(0xffffffffu, got)) {
@@ -230,25 +269,30 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       cp_async_commit();
     }
     cp_async_wait<0>();
-  } else {
+  } else if (warp == kMmaWarp) {
     // ------------------------------ MMA issuer (whole warp waits, one lane issues) ------------------------------
     const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
     uint32_t acc = 0;
-    for (int kb = 0; kb < n_kb; ++kb) {
-      const int s = kb % kStages;
-      const uint32_t ph = (uint32_t)(kb / kStages) & 1u;
+    for (int st = 0; st < n_st; ++st) {
+      const int s = st % kStages;
+      const uint32_t ph = (uint32_t)(st / kStages) & 1u;
       const bool got = !s_abort && mbar_wait(full0 + 8 * s, ph);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
         break;
       }
+      // 3xTF32 only: its tiles were written through the generic proxy (cp.async, st.shared) by the producers;
+      // the acquire above made them visible to this thread, this fence orders them before the MMA's reads.
+      // (Fencing here and not in the producers: a producer's fence would also wait for its copies in flight.)
+      if (k3x) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       if (lane == 0) {
         const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes;
-        const uint64_t a_hi = umma_desc(sb), b_hi = umma_desc(sb + kTileBytes);
 #pragma unroll
-        for (int k8 = 0; k8 < kBlockK / 8; ++k8) {     // K = 8 per instruction: 32 bytes along the swizzled row
-          const uint64_t o = (uint64_t)(k8 * 2);
+        for (int k8 = 0; k8 < kSub * kBlockK / 8; ++k8) {   // K = 8 per instruction: 32 bytes along the swizzled row
+          const int sub = k8 / (kBlockK / 8);
+          const uint64_t a_hi = umma_desc(sb + sub * kTileBytes), b_hi = umma_desc(sb + (kSub + sub) * kTileBytes);
+          const uint64_t o = (uint64_t)((k8 % (kBlockK / 8)) * 2);
           if (k3x) {
             const uint64_t a_lo = umma_desc(sb + 2 * kTileBytes), b_lo = umma_desc(sb + 3 * kTileBytes);
             umma_tf32(tmem_base, a_lo + o, b_hi + o, idesc, acc);
@@ -276,7 +320,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     if (ok) {
       const int la = warp * 32 + lane;
       const int a = ti * kTile + la;
-      const double n2a = a < n_cand ? p.n2[idxA[la]] : 0.0;
+      const double norm_a = normA[la];
       const double rho = (double)p.rho;
       const double band = screen_band(N);
 #pragma unroll 1
@@ -288,7 +332,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
         for (int j = 0; j < 32; ++j) {
           const int lb = c * 32 + j;
           const int b = tj * kTile + lb;
-          const double den = sqrt(n2a * n2B[lb]);
+          const double den = norm_a * normB[lb];
           const double g = fabs((double)__uint_as_float(v[j]));
           const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
           bool hit = live && g >= rho * den;
@@ -307,15 +351,15 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
-  if (warp == kProducerWarps) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
-// Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product.
-// Setting a bit is idempotent and order-independent, so the result is deterministic.
-__global__ void __launch_bounds__(256) k_gram_recheck(Problem p, const int* __restrict__ cand) {
+// Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product of the
+// packed columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
+__global__ void __launch_bounds__(256) k_gram_recheck(Problem p) {
   const unsigned int n = p.st->amb_count;
   if (n > (unsigned)p.cap_amb) return;                 // overflow: the 3xTF32 kernel redoes every bit instead
   const int lane = threadIdx.x & 31;
@@ -325,12 +369,11 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, const int* __re
   for (unsigned int e = warp; e < n; e += n_warps) {
     const unsigned int pr = p.amb_pairs[e];
     const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
-    const int ja = cand[a], jb = cand[b];
-    const float4* xa = reinterpret_cast<const float4*>(p.xv + (long long)ja * p.ld);
-    const float4* xb = reinterpret_cast<const float4*>(p.xv + (long long)jb * p.ld);
+    const float4* xa = reinterpret_cast<const float4*>(p.xc + (long long)a * p.ldc);
+    const float4* xb = reinterpret_cast<const float4*>(p.xc + (long long)b * p.ldc);
     double acc = 0.0;
     for (long long g = lane; g < n4; g += 32) {
-      const float4 u = __ldg(xa + g), w = __ldg(xb + g);
+      const float4 u = xa[g], w = xb[g];
       const long long i = g << 2;
       acc += (double)u.x * w.x;
       if (i + 1 < p.N) acc += (double)u.y * w.y;
@@ -340,7 +383,7 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, const int* __re
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) {
-      const double den = sqrt(p.n2[ja] * p.n2[jb]);
+      const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
       if (den > 0.0 && fabs(acc) >= (double)p.rho * den)
         atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
     }
@@ -355,15 +398,42 @@ cudaError_t prepare_gram_dense_tc() {
   return cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
 }
 
-// screen -> exact recheck of the borderline pairs -> (only if their list overflowed) 3xTF32 over everything
-cudaError_t launch_gram_dense_tc(const Problem& p, const int* cand, int n_cand, cudaStream_t s) {
+// Tensor map over the packed candidate buffer: [n_cand rows][N floats], row pitch ldc, box 32 x 128, 128-byte
+// swizzle, zero fill outside.  `out` is 128 bytes, 64-byte aligned (a CUtensorMap).
+cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+  if (e != cudaSuccess) return e;
+  if (fn == nullptr || qres != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+  using EncodeFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+  const cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.n_cand};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.ldc * sizeof(float)};
+  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTile};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeFn>(fn)(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, p.xc,
+                                                    dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// pack -> screen -> exact recheck of the borderline pairs -> (only if their list overflowed) 3xTF32 over everything
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, cudaStream_t s) {
   const int n_tiles = (n_cand + kTile - 1) / kTile;
   const int blocks = n_tiles * (n_tiles + 1) / 2;
+  Problem q = p;
+  q.cand_cur = cand;
+  const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
+  k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand);
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
-    k_gram_dense_tc<false><<<blocks, kThreads, kDynSmem, s>>>(p, cand, n_cand, n_tiles);
-    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(p, cand);
+    k_gram_dense_tc<false><<<blocks, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles);
+    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q);
   }
-  k_gram_dense_tc<true><<<blocks, kThreads, kDynSmem, s>>>(p, cand, n_cand, n_tiles);
+  k_gram_dense_tc<true><<<blocks, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles);
   return cudaGetLastError();
 }
 

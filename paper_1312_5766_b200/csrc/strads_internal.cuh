@@ -70,6 +70,9 @@ struct Problem {
   double* obj_partial;          // [2 * kObjBlocks]
   unsigned int* amb_pairs;      // [cap_amb] (a << 16 | b), positions in the candidate list
   int cap_amb;
+  float* xc;                    // dense: packed copy of the candidate columns, [n_cand][ldc]
+  long long ldc;                // N rounded up to a multiple of 4
+  const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
   int sm_count;
 };
 static constexpr int kObjBlocks = 296;
@@ -150,7 +153,8 @@ cudaError_t prepare_sample(const Problem& p);
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_gram_dense_tc();
-cudaError_t launch_gram_dense_tc(const Problem& p, const int* cand, int n_cand, cudaStream_t s);
+cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, cudaStream_t s);
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s);
