@@ -3,9 +3,11 @@
 //
 // The walk is a serial chain (whether candidate i is kept depends on every earlier decision), and each
 // keep needs the conflict row of the kept candidate: a dependent memory access.  To take that latency
-// off the chain, one CTA prefetches the rows of the next 32 still-unblocked candidates together into
-// shared memory (they are the only ones that can be kept next), and one warp then resolves those 32
-// in order against the running `blocked` mask entirely in shared memory.
+// off the chain, one CTA works in batches of 32: the next 32 still-unblocked candidates (the only ones
+// that can be kept next) are found with a warp scan, their conflict rows are fetched together into
+// shared memory, each lane extracts its candidate's conflicts with the other 31 into one 32-bit word,
+// and the greedy decision inside the batch is then 32 steps of register arithmetic.  The rows of the
+// newly kept candidates are OR-ed into the running `blocked` mask by the whole CTA.
 #include "strads_internal.cuh"
 
 namespace strads {
@@ -18,18 +20,20 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
                                                       int* __restrict__ kept_out) {
   extern __shared__ unsigned int sm[];
   const int W = p.mask_words;
+  const int Ws = W | 1;                          // odd row pitch: column reads of `rows` hit 32 different banks
   unsigned int* blocked = sm;                    // [W]
-  unsigned int* rows = sm + W;                   // [kBatch][W]
-  __shared__ int pos[kBatch];
+  unsigned int* rows = sm + W;                   // [kBatch][Ws]
+  __shared__ int pos[kBatch];                    // positions (in the candidate list) of the batch
+  __shared__ int cval[kBatch];                   // cand[pos[.]]
   __shared__ int s_m, s_cursor, s_kept, s_examined, s_done;
+  __shared__ unsigned int s_keepmask;
   const int tid = threadIdx.x, lane = tid & 31;
-  const bool no_filter = (p.flags & STRADS_FLAG_NO_FILTER) != 0;
 
   for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
   if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = 0; s_done = 0; }
   __syncthreads();
 
-  if (no_filter) {
+  if (p.flags & STRADS_FLAG_NO_FILTER) {
     const int nk = min(n_cand, p.n_keep);
     for (int i = tid; i < p.n_keep; i += kThreads) kept_out[i] = i < nk ? cand[i] : -1;
     if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; }
@@ -37,30 +41,35 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   }
 
   while (true) {
-    // 1. the next <= kBatch candidates that are not blocked yet
+    // 1. the next <= kBatch candidates at or after the cursor that are not blocked yet (warp 0)
     if (tid < 32) {
       int m = 0;
       int cur = s_cursor;
       while (cur < n_cand && m < kBatch) {
-        const int wbase = (cur >> 5) + lane;           // 32 mask words at a time
+        const int wbase = (cur >> 5) + lane;           // 32 mask words at a time, one per lane
         unsigned int freew = 0u;
         if (wbase < W) {
           freew = ~blocked[wbase];
           const int first = wbase << 5;
-          if (first < cur) freew &= (cur - first >= 32) ? 0u : (0xffffffffu << (cur - first));
-          if (first + 32 > n_cand) freew &= (n_cand - first <= 0) ? 0u : (0xffffffffu >> (first + 32 - n_cand));
+          if (first < cur) freew &= 0xffffffffu << (cur - first);                         // only lane 0 can be cut
+          if (first + 32 > n_cand) freew &= first >= n_cand ? 0u : (0xffffffffu >> (first + 32 - n_cand));
         }
-        // lanes in order append their free positions
-        for (int l = 0; l < 32 && m < kBatch; ++l) {
-          unsigned int fw = __shfl_sync(0xffffffffu, freew, l);
-          const int base = ((cur >> 5) + l) << 5;
-          while (fw && m < kBatch) {
-            const int b = __ffs(fw) - 1;
-            fw &= fw - 1;
-            if (lane == 0) pos[m] = base + b;
-            ++m;
-          }
+        const int cnt = __popc(freew);
+        int incl = cnt;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
         }
+        const int total = __shfl_sync(0xffffffffu, incl, 31);
+        int slot = m + incl - cnt;                     // where this lane's first free position goes
+        unsigned int fw = freew;
+        while (fw && slot < kBatch) {
+          const int b = __ffs(fw) - 1;
+          fw &= fw - 1;
+          pos[slot++] = (wbase << 5) + b;
+        }
+        m = min(kBatch, m + total);
         if (m < kBatch) cur = ((cur >> 5) + 32) << 5;  // all 32 words consumed
       }
       if (lane == 0) s_m = m;
@@ -71,37 +80,87 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
       if (tid == 0) s_examined = n_cand;
       break;
     }
-    // 2. fetch their conflict rows together
-    for (int e = tid; e < m * W; e += kThreads) {
-      const int r = e / W, w = e - r * W;
-      rows[r * W + w] = __ldcg(&p.conflict[(long long)pos[r] * W + w]);
-    }
-    __syncthreads();
-    // 3. resolve in order
-    if (tid < 32) {
-      int nk = s_kept;
-      int last = -1;
-      bool full = false;
-      for (int q = 0; q < m; ++q) {
-        const int i = pos[q];
-        const bool is_blocked = (blocked[i >> 5] >> (i & 31)) & 1u;
-        last = i;
-        if (!is_blocked) {
-          if (lane == 0) kept_out[nk] = cand[i];
-          ++nk;
-          for (int w = (i >> 5) + lane; w < W; w += 32) blocked[w] |= rows[q * W + w];
-          __syncwarp();
-          if (nk == p.n_keep) { full = true; break; }
+    // 2. fetch their conflict rows (and their coefficient indices) together.  Loads first, stores after:
+    //    a store to `rows` between two loads would order them and cost one memory round trip per word.
+    if (tid < m) cval[tid] = cand[pos[tid]];
+    {
+      const int warp = tid >> 5;                       // warp w fetches rows w, w + 8, w + 16, w + 24
+      const unsigned int* src[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) src[u] = p.conflict + (long long)pos[min(warp + 8 * u, m - 1)] * W;
+      for (int w0 = lane; w0 < W; w0 += 64) {
+        unsigned int v[8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          v[u] = __ldcg(src[u] + w0);
+          v[4 + u] = w0 + 32 < W ? __ldcg(src[u] + w0 + 32) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int r = warp + 8 * u;
+          if (r < m) {
+            rows[r * Ws + w0] = v[u];
+            if (w0 + 32 < W) rows[r * Ws + w0 + 32] = v[4 + u];
+          }
         }
       }
+    }
+    __syncthreads();
+    // 3. decide the batch in order (warp 0, registers only)
+    if (tid < 32) {
+      // lane q: bit b set <=> candidate q conflicts with the LATER batch member b (row q is valid from its own word on)
+      // (fixed trip counts, so that the 32 reads / shuffles are independent and overlap)
+      const unsigned int valid = m >= 32 ? 0xffffffffu : ((1u << m) - 1u);
+      const int my_row = min(lane, m - 1) * Ws;
+      unsigned int mine = 0u;
+#pragma unroll
+      for (int b = 0; b < kBatch; ++b) {
+        const int pb = pos[min(b, m - 1)];
+        mine |= ((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << b;
+      }
+      mine &= valid & ~((2u << lane) - 1u);            // later members only (lane 31: none)
+      if (lane >= m) mine = 0u;
+      unsigned int cq[kBatch];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q) cq[q] = __shfl_sync(0xffffffffu, mine, q);
+      unsigned int alive = valid;
+      unsigned int keep = 0u;
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+        if ((alive >> q) & 1u) { keep |= 1u << q; alive &= ~cq[q]; }
+      const int nk = s_kept;
+      const int room = p.n_keep - nk;
+      bool full = false;
+      if (__popc(keep) >= room) {                      // stop exactly at P: drop the surplus from the back
+        while (__popc(keep) > room) keep &= ~(1u << (31 - __clz(keep)));
+        full = true;
+      }
+      if ((keep >> lane) & 1u) kept_out[nk + __popc(keep & ((1u << lane) - 1u))] = cval[lane];
       if (lane == 0) {
-        s_kept = nk;
-        s_cursor = last + 1;
-        if (full) { s_examined = last + 1; s_done = 1; }
+        s_keepmask = keep;
+        s_kept = nk + __popc(keep);
+        if (full) { s_examined = pos[31 - __clz(keep)] + 1; s_done = 1; }
+        else s_cursor = pos[m - 1] + 1;
       }
     }
     __syncthreads();
     if (s_done) break;
+    // 4. OR the rows of the newly kept candidates into the mask (a row is valid from its own word on)
+    //    Four threads share a word, each takes 8 of the 32 batch members; reads are unconditional so that they overlap.
+    const unsigned int keep = s_keepmask;
+    for (int u = tid; u < 4 * W; u += kThreads) {
+      const int w = u >> 2, q0 = (u & 3) * 8;
+      unsigned int acc = 0u;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const int q = q0 + i;
+        const unsigned int v = rows[min(q, m - 1) * Ws + w];
+        const bool use = ((keep >> q) & 1u) && w >= (pos[min(q, m - 1)] >> 5);
+        acc |= use ? v : 0u;
+      }
+      if (acc) atomicOr(&blocked[w], acc);
+    }
+    __syncthreads();
   }
   __syncthreads();
   const int nk = s_kept;
@@ -111,12 +170,15 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
 
 }  // namespace
 
-size_t filter_smem_bytes(const Problem& p) { return (size_t)(kBatch + 1) * p.mask_words * sizeof(unsigned int); }
+size_t filter_smem_bytes(const Problem& p) {
+  return ((size_t)p.mask_words + (size_t)kBatch * (p.mask_words | 1)) * sizeof(unsigned int);
+}
 
 // Kernel-wide attribute: the largest size any handle can need (see prepare_sample).
 cudaError_t prepare_filter(const Problem&) {
+  constexpr int kMaxWords = STRADS_MAX_CANDIDATES / 32;
   return cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)((kBatch + 1) * (STRADS_MAX_CANDIDATES / 32) * sizeof(unsigned int)));
+                              (int)((kMaxWords + kBatch * (kMaxWords | 1)) * sizeof(unsigned int)));
 }
 
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s) {
