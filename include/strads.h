@@ -63,6 +63,10 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
                                           (default: TF32 screen + exact recheck of the pairs
                                           within 2^-8 of rho; 3xTF32 only if those overflow)   */
 
+#define STRADS_FLAG_FULL_GRAM    16u   /* form the conflict bits of ALL P' candidates before the
+                                          walk (default: of a leading window of 1.5 P + 128 first,
+                                          of all P' only if the walk runs out of the window)    */
+
 /* limits */
 #define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (one CTA sorts the winners in shared memory) */
 
@@ -172,7 +176,9 @@ int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);
 /* Optional step timing with CUDA events on the handle's stream.  After strads_profile_begin the next
  * max_rounds rounds (strads_round / strads_run / strads_round_host) record an event at every step
  * boundary; strads_profile_end waits for the stream and returns the summed device time in
- * milliseconds of ms[0] sampling, ms[1] Gram, ms[2] greedy filter, ms[3] update over *rounds rounds.
+ * milliseconds of ms[0] sampling, ms[1] Gram (of the candidate window, or of all candidates when no window is
+ * used), ms[2] greedy walk (plus the whole-list retry when the window was too short), ms[3] update over
+ * *rounds rounds.
  * Events are host-side driver objects; no device memory is allocated. */
 int strads_profile_begin(strads_handle_t h, int64_t max_rounds);
 int strads_profile_end(strads_handle_t h, double* ms_host_out /* [4] */, int64_t* rounds_host_out);

@@ -21,6 +21,7 @@ FLAG_UNIFORM_DRAW = 1
 FLAG_NO_FILTER = 2
 FLAG_SIMT_GRAM = 4
 FLAG_GRAM_3XTF32 = 8
+FLAG_FULL_GRAM = 16
 MAX_CANDIDATES = 16384
 
 EXPORTS = [

@@ -40,8 +40,8 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_dbeta, off_dbeta64,
-      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, total;
-  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb;
+      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, total;
+  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles;
   long long ldc;
 };
 
@@ -86,6 +86,8 @@ Layout carve(const strads_lasso_config_t* c) {
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
   L.ldc = (c->n_rows + 3) / 4 * 4;
   L.off_xc = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(float) * (size_t)c->n_candidates * L.ldc : 0);
+  L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)
+  L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
   L.total = o;
   return L;
 }
@@ -94,20 +96,39 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
-cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg) {
+cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, bool only_if_short) {
   const Problem& p = h->p;
   cudaStream_t s = h->stream;
-  if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, s);
+  if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, s);
+  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, s);
 }
 
-int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg) {
+// The greedy walk stops at P kept, so it normally looks at little more than the first P candidates: form the
+// conflict bits of a leading window only (1.5 P + 128, rounded to the Gram tile) and walk that.  The result is
+// final when P are kept inside the window; otherwise the filter raises window_short and the whole-list
+// Gram + walk, enqueued behind it, runs (it is a no-op otherwise).  Same kept set either way.
+int window_of(const Problem& p, int n_cand) {
+  if (p.flags & (STRADS_FLAG_FULL_GRAM | STRADS_FLAG_SIMT_GRAM)) return n_cand;
+  const long long w = ((long long)p.n_keep + p.n_keep / 2 + 128 + 127) / 128 * 128;
+  return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
+}
+
+int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, cudaEvent_t after_gram = nullptr) {
   const Problem& p = h->p;
-  if (!(p.flags & STRADS_FLAG_NO_FILTER)) {
-    CK(launch_gram(h, cand, n_cand, gram_dbg));
+  if (p.flags & STRADS_FLAG_NO_FILTER) {
+    if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
+    CK(launch_filter(p, cand, n_cand, n_cand, false, p.kept, h->stream));
+    return STRADS_OK;
   }
-  CK(launch_filter(p, cand, n_cand, p.kept, h->stream));
+  const int window = gram_dbg != nullptr ? n_cand : window_of(p, n_cand);
+  CK(launch_gram(h, cand, window, gram_dbg, false));
+  if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
+  CK(launch_filter(p, cand, window, n_cand, false, p.kept, h->stream));
+  if (window < n_cand) {
+    CK(launch_gram(h, cand, n_cand, nullptr, true));
+    CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, h->stream));
+  }
   return STRADS_OK;
 }
 
@@ -117,9 +138,10 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
   if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
   if (ev) CK(cudaEventRecord(ev[1], h->stream));
-  if (!(p.flags & STRADS_FLAG_NO_FILTER)) CK(launch_gram(h, p.cand, p.n_cand, out ? out->gram : nullptr));
-  if (ev) CK(cudaEventRecord(ev[2], h->stream));
-  CK(launch_filter(p, p.cand, p.n_cand, p.kept, h->stream));
+  {
+    const int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr);
+    if (rc) return rc;
+  }
   if (ev) CK(cudaEventRecord(ev[3], h->stream));
   CK(launch_update(p, p.kept, 1, h->stream));
   if (ev) { CK(cudaEventRecord(ev[4], h->stream)); h->prof_rounds += 1; }
@@ -188,6 +210,8 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   p.xc = reinterpret_cast<float*>(ws + L.off_xc);
   p.ldc = L.ldc;
   p.cand_cur = nullptr;
+  p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
+  p.partial_tiles = L.partial_tiles;
   h->stream = static_cast<cudaStream_t>(c->stream);
   h->round_host = 0;
   h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;

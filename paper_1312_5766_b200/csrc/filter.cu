@@ -16,8 +16,12 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kBatch = 32;
 
-__global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand,
-                                                      int* __restrict__ kept_out) {
+// n_cand < n_total: the list is only a leading window of the candidates.  If P are kept inside it the result
+// is final (the walk never looks further); otherwise window_short is raised and the caller's retry over
+// the whole list (launched with only_if_short) replaces the result.
+__global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
+                                                      int only_if_short, int* __restrict__ kept_out) {
+  if (only_if_short && !p.st->window_short) return;
   extern __shared__ unsigned int sm[];
   const int W = p.mask_words;
   const int Ws = W | 1;                          // odd row pitch: column reads of `rows` hit 32 different banks
@@ -36,7 +40,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (p.flags & STRADS_FLAG_NO_FILTER) {
     const int nk = min(n_cand, p.n_keep);
     for (int i = tid; i < p.n_keep; i += kThreads) kept_out[i] = i < nk ? cand[i] : -1;
-    if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; }
+    if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; p.st->window_short = 0; }
     return;
   }
 
@@ -165,7 +169,10 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   __syncthreads();
   const int nk = s_kept;
   for (int i = nk + tid; i < p.n_keep; i += kThreads) kept_out[i] = -1;
-  if (tid == 0) { p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; }
+  if (tid == 0) {
+    p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0;
+    p.st->window_short = (!only_if_short && nk < p.n_keep && n_cand < n_total) ? 1 : 0;
+  }
 }
 
 }  // namespace
@@ -181,8 +188,9 @@ cudaError_t prepare_filter(const Problem&) {
                               (int)((kMaxWords + kBatch * (kMaxWords | 1)) * sizeof(unsigned int)));
 }
 
-cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s) {
-  k_filter<<<1, kThreads, filter_smem_bytes(p), s>>>(p, cand, n_cand, kept_out);
+cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
+                          cudaStream_t s) {
+  k_filter<<<1, kThreads, filter_smem_bytes(p), s>>>(p, cand, n_cand, n_total, only_if_short ? 1 : 0, kept_out);
   return cudaGetLastError();
 }
 

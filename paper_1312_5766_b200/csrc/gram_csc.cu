@@ -12,7 +12,8 @@ constexpr int kThreads = 256;
 constexpr int kStage = 1024;          // entries of column a staged in shared memory (longer columns: global)
 
 __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __restrict__ cand, int n_cand,
-                                                        float* __restrict__ gram_dbg) {
+                                                        float* __restrict__ gram_dbg, int only_if_short) {
+  if (only_if_short && !p.st->window_short) return;
   __shared__ int arow[kStage];
   __shared__ float aval[kStage];
   const int a = blockIdx.x;
@@ -71,8 +72,9 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
 
 }  // namespace
 
-cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s) {
-  k_gram_csc<<<n_cand, kThreads, 0, s>>>(p, cand, n_cand, gram_dbg);
+cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
+                            cudaStream_t s) {
+  k_gram_csc<<<n_cand, kThreads, 0, s>>>(p, cand, n_cand, gram_dbg, only_if_short ? 1 : 0);
   return cudaGetLastError();
 }
 

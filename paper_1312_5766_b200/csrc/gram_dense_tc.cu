@@ -123,10 +123,34 @@ __device__ __forceinline__ float tf32_lo(float x) {
   return __uint_as_float(__float_as_uint(x - hi) & 0xffffe000u);
 }
 
+// 32 Gram values of row a against columns b0 .. b0 + 31 -> conflict bits.  Screen mode leaves the pairs
+// inside the band undecided (bit clear) and appends them to the list k_gram_recheck works through.
+template <bool kScreen>
+__device__ __forceinline__ uint32_t decide_word(const Problem& p, const uint32_t (&v)[32], int a, int b0, int n_cand,
+                                                double norm_a, const double* norm_b, double rho, double band) {
+  uint32_t word = 0u;
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    const int b = b0 + j;
+    const double den = norm_a * norm_b[j];
+    const double g = fabs((double)__uint_as_float(v[j]));
+    const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
+    bool hit = live && g >= rho * den;
+    if (kScreen && live && b > a && fabs(g - rho * den) <= band * den) {
+      hit = false;
+      const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
+      if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
+    }
+    word |= (uint32_t)hit << j;
+  }
+  return word;
+}
+
 // One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).
-__global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand) {
+__global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
+                                                         int only_if_short) {
   const int a = blockIdx.x;
-  if (a >= n_cand) return;
+  if (a >= n_cand || (only_if_short && !p.st->window_short)) return;
   const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)cand[a] * p.ld);
   float4* dst = reinterpret_cast<float4*>(p.xc + (long long)a * p.ldc);
   const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
@@ -135,7 +159,7 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
 
 template <bool k3x>
 __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const __grid_constant__ CUtensorMap tmap,
-                                                                int n_cand, int n_tiles) {
+                                                                int n_cand, int n_tiles, int n_split, int only_if_short) {
   // A stage holds kSub sub-blocks of 32 floats of K for A, the same for B [3xTF32: plus the two lo tiles].
   constexpr int kSub = k3x ? 1 : 2;
   constexpr int kStageBytes = (k3x ? 4 : 2 * kSub) * kTileBytes;       // 64 KB either way
@@ -149,13 +173,17 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   __shared__ volatile int s_abort;
   __shared__ double normA[kTile], normB[kTile];                        // ||x|| of the tile's rows / columns
 
+  if (only_if_short && !p.st->window_short) return;
   // as a fallback the 3xTF32 variant runs only when the screen's list overflowed
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && p.st->amb_count <= (unsigned)p.cap_amb) return;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && blockIdx.x == 0 && tid == 0)
     atomicOr(&p.st->status, STRADS_STATUS_GRAM_FALLBACK);
-  int ti = 0, rem = blockIdx.x;                        // linear index -> (ti, tj), ti <= tj
+  // With n_split > 1 the K range of a tile is shared by n_split CTAs, each leaving an FP32 partial tile that
+  // k_gram_reduce sums in split order (a window of few tiles would otherwise use few SMs).
+  const int tile = blockIdx.x / n_split, split = blockIdx.x - tile * n_split;
+  int ti = 0, rem = tile;                              // linear index -> (ti, tj), ti <= tj
   while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
   const int tj = ti + rem;
 
@@ -185,7 +213,10 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const uint32_t tmem_base = s_tmem_base;
 
   const long long N = p.N;
-  const int n_st = (int)((N + (long long)kBlockK * kSub - 1) / ((long long)kBlockK * kSub));   // stages of K
+  const int n_st_all = (int)((N + (long long)kBlockK * kSub - 1) / ((long long)kBlockK * kSub));   // stages of K
+  const int per_split = (n_st_all + n_split - 1) / n_split;
+  const int st_first = min(n_st_all, split * per_split);
+  const int n_st = min(n_st_all, st_first + per_split) - st_first;     // this CTA's stages (may be 0)
 
   if (!k3x && warp == kTmaWarp) {
     // ------------------------------ screen: TMA producer (one lane) ------------------------------
@@ -202,7 +233,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
         mbar_arrive_expect_tx(bar, (uint32_t)kStageBytes);
 #pragma unroll
         for (int sub = 0; sub < kSub; ++sub) {
-          const int k = (st * kSub + sub) * kBlockK;    // past N the whole box is zero-filled
+          const int k = ((st_first + st) * kSub + sub) * kBlockK;    // past N the whole box is zero-filled
           tma_load_2d(sb + sub * kTileBytes, &tmap, k, ti * kTile, bar);
           tma_load_2d(sb + (kSub + sub) * kTileBytes, &tmap, k, tj * kTile, bar);
         }
@@ -226,7 +257,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     }
     auto issue = [&](int st) {                         // all copies of one stage
       const uint32_t sb = tiles0 + (uint32_t)(st % kStages) * kStageBytes;
-      const long long k = (long long)st * kBlockK + chunk * 4;
+      const long long k = (long long)(st_first + st) * kBlockK + chunk * 4;
       const long long left = N - k;                    // floats of this chunk that exist
       const uint32_t bytes = left >= 4 ? 16u : (left > 0 ? (uint32_t)left * 4u : 0u);
 #pragma unroll
@@ -326,24 +357,19 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 #pragma unroll 1
       for (int c = 0; c < kTile / 32; ++c) {
         uint32_t v[32];
-        tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
-        uint32_t word = 0u;
+        if (n_st > 0) {
+          tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
+        } else {                                       // a split with no K of its own contributes zero
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int lb = c * 32 + j;
-          const int b = tj * kTile + lb;
-          const double den = norm_a * normB[lb];
-          const double g = fabs((double)__uint_as_float(v[j]));
-          const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
-          bool hit = live && g >= rho * den;
-          if (!k3x && live && b > a && fabs(g - rho * den) <= band * den) {
-            // too close to call in TF32: leave the bit clear and let k_gram_recheck decide exactly
-            hit = false;
-            const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
-            if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
-          }
-          word |= (uint32_t)hit << j;
+          for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
+        if (n_split > 1) {
+          uint4* dst = reinterpret_cast<uint4*>(p.gram_partial + (((size_t)tile * n_split + split) * kTile + la) * kTile + c * 32);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+          continue;
+        }
+        const uint32_t word = decide_word<!k3x>(p, v, a, tj * kTile + c * 32, n_cand, norm_a, normB + c * 32, rho, band);
         const int widx = tj * (kTile / 32) + c;
         if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
       }
@@ -357,9 +383,47 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   }
 }
 
+// Split-K: sums the partial tiles of one output tile in split order and thresholds (screen rules).
+// One CTA per (tile, 32 rows); thread = (row, 32-column chunk).
+__global__ void __launch_bounds__(128) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short) {
+  if (only_if_short && !p.st->window_short) return;
+  __shared__ double normB[kTile];
+  const int tile = blockIdx.x >> 2, rgroup = blockIdx.x & 3;
+  int ti = 0, rem = tile;
+  while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
+  const int tj = ti + rem;
+  {
+    const int gb = tj * kTile + threadIdx.x;
+    normB[threadIdx.x] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
+  }
+  __syncthreads();
+  const int la = rgroup * 32 + (threadIdx.x >> 2), c = threadIdx.x & 3;
+  const int a = ti * kTile + la;
+  float acc[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) acc[j] = 0.f;
+  for (int s = 0; s < n_split; ++s) {
+    const float4* src = reinterpret_cast<const float4*>(p.gram_partial + (((size_t)tile * n_split + s) * kTile + la) * kTile + c * 32);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float4 u = __ldcg(src + j);
+      acc[4 * j] += u.x; acc[4 * j + 1] += u.y; acc[4 * j + 2] += u.z; acc[4 * j + 3] += u.w;
+    }
+  }
+  uint32_t v[32];
+#pragma unroll
+  for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+  const double norm_a = a < n_cand ? sqrt(p.n2[p.cand_cur[a]]) : 0.0;
+  const uint32_t word = decide_word<true>(p, v, a, tj * kTile + c * 32, n_cand, norm_a, normB + c * 32, (double)p.rho,
+                                          screen_band(p.N));
+  const int widx = tj * (kTile / 32) + c;
+  if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+}
+
 // Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product of the
 // packed columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
-__global__ void __launch_bounds__(256) k_gram_recheck(Problem p) {
+__global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_short) {
+  if (only_if_short && !p.st->window_short) return;
   const unsigned int n = p.st->amb_count;
   if (n > (unsigned)p.cap_amb) return;                 // overflow: the 3xTF32 kernel redoes every bit instead
   const int lane = threadIdx.x & 31;
@@ -421,19 +485,32 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-// pack -> screen -> exact recheck of the borderline pairs -> (only if their list overflowed) 3xTF32 over everything
-cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, cudaStream_t s) {
+// pack -> screen [-> split-K reduce] -> exact recheck of the borderline pairs -> (only if their list overflowed)
+// 3xTF32 over everything
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
+                                 cudaStream_t s) {
   const int n_tiles = (n_cand + kTile - 1) / kTile;
-  const int blocks = n_tiles * (n_tiles + 1) / 2;
+  const int tiles = n_tiles * (n_tiles + 1) / 2;
+  const int ois = only_if_short ? 1 : 0;
+  // few tiles (a candidate window): share each tile's K range among CTAs so that all SMs work
+  int n_split = 1;
+  if (tiles * 2 <= p.sm_count) {
+    const int n_st = (int)((p.N + 2 * kBlockK - 1) / (2 * kBlockK));
+    n_split = p.sm_count / tiles;
+    if (n_split > n_st) n_split = n_st;
+    if (n_split > p.partial_tiles / tiles) n_split = p.partial_tiles / tiles;
+    if (n_split < 1) n_split = 1;
+  }
   Problem q = p;
   q.cand_cur = cand;
   const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
-  k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand);
+  k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand, ois);
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
-    k_gram_dense_tc<false><<<blocks, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles);
-    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q);
+    k_gram_dense_tc<false><<<tiles * n_split, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, n_split, ois);
+    if (n_split > 1) k_gram_reduce<<<tiles * 4, 128, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
+    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q, ois);
   }
-  k_gram_dense_tc<true><<<blocks, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles);
+  k_gram_dense_tc<true><<<tiles, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, 1, ois);
   return cudaGetLastError();
 }
 

@@ -30,7 +30,8 @@ struct DeviceState {
   float x_abs_max;              // max |x_ij| (CSC: bounds the fixed-point residual update)
   int beta0_nonzero;            // set at init when the starting beta has a non-zero entry
   unsigned int amb_count;       // pairs the TF32 screen of the dense Gram left to the exact recheck
-  unsigned int pad[3];
+  int window_short;             // the filter ran out of its candidate window before P were kept: redo on all P'
+  unsigned int pad[2];
 };
 
 static constexpr int kHistBits = 12;
@@ -73,6 +74,8 @@ struct Problem {
   float* xc;                    // dense: packed copy of the candidate columns, [n_cand][ldc]
   long long ldc;                // N rounded up to a multiple of 4
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
+  float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
+  int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles
   int sm_count;
 };
 static constexpr int kObjBlocks = 296;
@@ -154,10 +157,16 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_gram_dense_tc();
 cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
-cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, cudaStream_t s);
-cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
+// `only_if_short`: the launch is the whole-list retry of a windowed round and does nothing unless the
+// window's filter set DeviceState::window_short.
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
+                                 cudaStream_t s);
+cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
+                            cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);
-cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int* kept_out, cudaStream_t s);
+// Walks cand[0 .. n_cand); n_total >= n_cand is the length of the whole list (n_cand < n_total: a window).
+cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
+                          cudaStream_t s);
 cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s);
 cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s);
 cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,

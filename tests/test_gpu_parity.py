@@ -420,3 +420,36 @@ def test_tensor_core_screen_overflow_falls_back_to_3xtf32():
     # the two FP32-accurate kernels may differ only on pairs within 1e-6 of rho; on this data they agree
     assert torch.equal(kept_tc, kept_s) and torch.equal(counts_tc, counts_s)
     assert tc.status() == (0, 8)                     # informational bit: the fallback did run
+
+
+# --------------------------------------------------------------------------------------------------
+# candidate window: the default (window first, whole list only if the walk runs out) against the
+# whole-list Gram, on data where the window suffices and on data where it does not
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,n_keep", [("dense", 24), ("dense_grouped", 24), ("dense_grouped", 120), ("csc", 100),
+                                         ("csc_zipf", 60), ("csc_zipf", 300)])
+def test_window_equals_full_gram(name, n_keep):
+    b = _binding()
+    cfg = dict(_small_problems()[name], n_keep=n_keep)
+    cfg["n_candidates"] = 1024 if "dense" in name else cfg["n_candidates"]
+    p = wl.make_problem(cfg, seed=13)
+    X = oracle_matrix(p)
+    n2 = oracle.colnorm2(X)
+    rho = float(np.float32(p.rho))
+    lazy, full = _solver(p), _solver(p, flags=b.FLAG_FULL_GRAM)
+    rng = np.random.default_rng(6)
+    shorts = 0
+    for trial in range(4):
+        cand = rng.permutation(p.n_cols)[: p.n_candidates].astype(np.int32)
+        if name == "dense_grouped" and trial % 2 == 0:
+            cand = np.arange(p.n_candidates, dtype=np.int32)       # whole groups side by side: the window runs short
+        cd = torch.from_numpy(cand).cuda()
+        kept_l, counts_l = lazy.filter(cd)
+        kept_f, counts_f = full.filter(cd)
+        assert torch.equal(kept_l, kept_f) and torch.equal(counts_l, counts_f), (name, trial)
+        c = counts_l.cpu().numpy(); nk = int(c[2])
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept_l.cpu().numpy()[:nk], int(c[1]))
+        shorts += nk < p.n_keep
+    if (name, n_keep) in (("dense_grouped", 120), ("csc_zipf", 300)):
+        assert shorts > 0                        # these did exercise the whole-list retry
+    assert lazy.status()[0] == 0
