@@ -215,19 +215,22 @@ def main():
     # ---- device-resident timing: K rounds after W warm-up rounds -------------------------------------
     s.run(args.warmup)
     kept_before = s.totals()["kept"]
-    s.profile_begin(args.steps)
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     clocks = ClockSampler(local_rank)
     ev0.record()
-    s.run(args.steps)
+    s.run(args.steps)                      # strads_run: one captured round replayed K times
     ev1.record()
     barrier()
-    clk = clocks.stop()
     ms_local = ev0.elapsed_time(ev1)
-    prof = s.profile_end()
     tot = s.totals()
     kept_local = tot["kept"] - kept_before
+    # per-step device times: the next rounds of the same run, launched kernel by kernel with events between the steps
+    prof_rounds = min(args.steps, 500)
+    s.profile_begin(prof_rounds)
+    s.run(prof_rounds)
+    prof = s.profile_end()
+    clk = clocks.stop()
     kept_all, ms = aggregate(kept_local, ms_local, dist_ok, device)
     value = kept_all / (ms * 1e-3)
     objective = s.objective()
@@ -294,6 +297,9 @@ def main():
                         "sample": f"{rounds} full oracle rounds of {args.workload} from the state after the timed "
                                   f"region ({sec:.1f} s, single thread; host has {os.cpu_count()} cores)"}
 
+    # kernels per round: sampler 3, window Gram (dense: pack, screen, split-K reduce, recheck, 3xTF32 gate = 5;
+    # CSC: 1), walk 1, whole-list retry (dense 4 + 1, CSC 1 + 1; they return at once when not needed), update 2
+    launches_per_round = 3 + (5 + 1 + 5 if p.layout == wl.DENSE else 1 + 1 + 2) + 2
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -306,14 +312,16 @@ def main():
             "rounds_per_s": world * args.steps / (ms * 1e-3),
             "kept_per_round": kept_per_round,
             "objective": objective, "status_bits": status_bits,
-            "step_ms": step_ms,
+            "step_ms": step_ms, "step_ms_rounds": prof["rounds"],
+            "step_ms_note": "device time per step over the rounds right after the timed region, launched kernel by "
+                            "kernel with CUDA events between steps (the timed region itself replays a CUDA graph)",
             "roofline": roofline,
             "update_hbm": {"achieved": upd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": upd_gbs / peaks["hbm_gbs"], "bytes_per_round": upd_bytes},
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_kept_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
-            "gpu_launches": 7 * args.steps,
+            "gpu_launches": launches_per_round * args.steps,
             "clocks": clk,
         }
         print(json.dumps(line), flush=True)

@@ -19,6 +19,10 @@ struct strads_lasso_s {
   // optional step timing: 5 events per round (start, after sample, Gram, filter, update)
   cudaEvent_t* prof_events;
   long long prof_cap, prof_rounds;
+  // strads_run replays one captured round (the launch sequence of a round is fixed for a handle)
+  cudaStream_t capture_stream;
+  cudaGraph_t round_graph;
+  cudaGraphExec_t round_exec;
 };
 
 namespace {
@@ -215,6 +219,7 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   h->stream = static_cast<cudaStream_t>(c->stream);
   h->round_host = 0;
   h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
+  h->capture_stream = nullptr; h->round_graph = nullptr; h->round_exec = nullptr;
 
   auto fail = [&](int code) { delete h; return code; };
   cudaError_t e = cudaGetDevice(&h->device);
@@ -237,11 +242,42 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out) {
   return one_round(h, out);
 }
 
+// Captures the kernel sequence of one round into a graph (on a private stream: the caller's may be the legacy
+// default stream, which cannot be captured; nothing executes during capture).
+static int build_round_graph(strads_lasso_s* h) {
+  CK(cudaStreamCreateWithFlags(&h->capture_stream, cudaStreamNonBlocking));
+  cudaStream_t user = h->stream;
+  const long long round_before = h->round_host;
+  h->stream = h->capture_stream;
+  cudaError_t e = cudaStreamBeginCapture(h->capture_stream, cudaStreamCaptureModeThreadLocal);
+  int rc = STRADS_OK;
+  if (e == cudaSuccess) {
+    rc = one_round(h, nullptr);
+    e = cudaStreamEndCapture(h->capture_stream, &h->round_graph);
+  }
+  h->stream = user;
+  h->round_host = round_before;
+  if (rc) return rc;
+  if (e != cudaSuccess) return cuda_fail(e, "stream capture of a round");
+  CK(cudaGraphInstantiate(&h->round_exec, h->round_graph, 0));
+  return STRADS_OK;
+}
+
 int strads_run(strads_handle_t h, int64_t n_rounds) {
   if (h == nullptr || n_rounds < 0) return STRADS_ERR_INVALID_ARG;
-  for (int64_t i = 0; i < n_rounds; ++i) {
-    const int rc = one_round(h, nullptr);
+  const bool use_graph = h->prof_events == nullptr && n_rounds > 1;   // step timing needs events between kernels
+  if (use_graph && h->round_exec == nullptr) {
+    const int rc = build_round_graph(h);
     if (rc) return rc;
+  }
+  for (int64_t i = 0; i < n_rounds; ++i) {
+    if (use_graph) {
+      CK(cudaGraphLaunch(h->round_exec, h->stream));
+      h->round_host += 1;
+    } else {
+      const int rc = one_round(h, nullptr);
+      if (rc) return rc;
+    }
   }
   return STRADS_OK;
 }
@@ -390,6 +426,9 @@ int strads_destroy(strads_handle_t h) {
     for (long long i = 0; i < 5 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
     delete[] h->prof_events;
   }
+  if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
+  if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
+  if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
   delete h;
   return STRADS_OK;
 }
