@@ -1,0 +1,97 @@
+"""Parity at the full benchmark sizes (c2 .. c5), in the launch configuration bench.py times.
+
+The oracle cannot hold or sweep these problems whole, so each checked round is verified on what it
+touched: the candidate list bit-exactly from the device's delta (the oracle ranks all J keys), and the
+kept list, the coefficient changes and the new residual on the candidate columns alone, gathered from
+the device into a compact matrix (the oracle's filter and update only ever read those columns).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1312_5766_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+RTOL_DBETA, ATOL_DBETA, RHO_EXCUSE = 1e-5, 1e-7, 1e-6
+
+
+def _compact_matrix(p, cand):
+    """Oracle matrix whose column a is column cand[a] of X."""
+    idx = torch.from_numpy(cand.astype(np.int64)).to(p.values.device)
+    if p.layout == wl.DENSE:
+        return oracle.Matrix.dense(p.values[idx].cpu().numpy(), n_rows=p.n_rows)
+    cp = p.col_ptr
+    starts, ends = cp[idx], cp[idx + 1]
+    lens = (ends - starts).cpu().numpy()
+    new_ptr = np.concatenate([[0], np.cumsum(lens)]).astype(np.int64)
+    # all configurations here have a fixed number of entries per column
+    k = int(lens[0])
+    assert np.all(lens == k)
+    gather = (starts[:, None] + torch.arange(k, device=starts.device)[None, :]).reshape(-1)
+    return oracle.Matrix.csc(p.n_rows, len(cand), p.values[gather].cpu().numpy(), p.row_idx[gather].cpu().numpy(), new_ptr)
+
+
+def _check_round(p, s, t):
+    beta = s.beta.cpu().numpy().astype(np.float64)
+    resid = s.resid.cpu().numpy().astype(np.float64)
+    delta = s.delta.cpu().numpy().astype(np.float64)
+    cand_d, kept_d, dbeta_d, counts_d = s.round()
+    counts = counts_d.cpu().numpy(); nk = int(counts[2])
+    cand = cand_d.cpu().numpy(); kept = kept_d.cpu().numpy()[:nk]; d_got = dbeta_d.cpu().numpy()[:nk]
+    lam, eta, rho = float(np.float32(p.lam)), float(np.float32(p.eta)), float(np.float32(p.rho))
+    # level 1: candidates
+    want_cand = oracle.sample(delta, eta, p.seed, t, p.n_candidates)
+    assert np.array_equal(cand, want_cand), (t, np.flatnonzero(cand != want_cand)[:5])
+    # level 2 on the candidate columns: positions 0 .. P'-1 stand for the coefficients cand[.]
+    Xc = _compact_matrix(p, cand)
+    n2c = oracle.colnorm2(Xc)
+    assert np.allclose(s.colnorm2()[torch.from_numpy(cand.astype(np.int64)).cuda()].cpu().numpy(), n2c, rtol=1e-12)
+    order = np.arange(p.n_candidates, dtype=np.int32)
+    pos_of = {int(c): i for i, c in enumerate(cand)}
+    got_pos = np.array([pos_of[int(k)] for k in kept], dtype=np.int32)
+    want_pos, ne, mm = oracle.filter(Xc, n2c, order, p.n_keep, rho)
+    if not np.array_equal(got_pos, want_pos):
+        assert mm <= RHO_EXCUSE, ("kept differs without a borderline pair", mm)
+        want_pos, ne, _ = oracle.filter(Xc, n2c, order, p.n_keep, rho, follow=got_pos, tol=RHO_EXCUSE)
+        assert np.array_equal(got_pos, want_pos)
+    assert int(counts[1]) == ne and counts[0] == p.n_candidates
+    beta_c, delta_c = beta[cand].copy(), delta[cand].copy()
+    d_want = oracle.update(Xc, n2c, lam, got_pos, beta_c, resid, delta_c)
+    bmax = max(np.abs(beta).max(), np.abs(beta_c).max(), 1e-30)
+    assert np.all(np.abs(d_got - d_want) <= RTOL_DBETA * np.abs(d_want) + ATOL_DBETA * bmax), t
+    assert int(counts[3]) == int(np.count_nonzero(d_got))
+    r_got = s.resid.cpu().numpy()
+    assert np.abs(r_got - resid).max() <= 2e-7 * np.abs(resid).max() + 1e-7 * bmax
+    b_got = s.beta.cpu().numpy()
+    assert np.abs(b_got[cand] - beta_c).max() <= 1.2e-7 * bmax
+    untouched = np.ones(p.n_cols, bool); untouched[kept] = False
+    assert np.array_equal(b_got[untouched], beta[untouched].astype(np.float32))
+    return nk, int(counts[1])
+
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4", "c5"])
+def test_full_size_rounds(name):
+    from paper_1312_5766_b200 import binding
+    free, _ = torch.cuda.mem_get_info()
+    need = {"c2": 8e9, "c3": 26e9, "c4": 4e9, "c5": 14e9}[name]
+    if free < need:
+        pytest.skip(f"{name} needs {need / 1e9:.0f} GB of device memory")
+    p = wl.make_problem(name, seed=0, device="cuda")
+    s = binding.StradsLasso.from_problem(p, device="cuda")
+    f0 = s.objective()
+    stats = []
+    t = 0
+    for phase, (n_run, n_check) in enumerate([(0, 2), (40, 2), (150, 1)]):
+        s.run(n_run)                               # graph replay, as the benchmark does
+        t += n_run
+        for _ in range(n_check):
+            stats.append(_check_round(p, s, t))
+            t += 1
+    assert s.get_round() == t and s.status()[0] == 0
+    assert s.objective() < f0                      # and the iteration does make progress
+    tot = s.totals()
+    assert tot["rounds"] == t and tot["kept"] >= sum(k for k, _ in stats)
+    del s, p
+    torch.cuda.empty_cache()
