@@ -20,6 +20,7 @@ struct strads_lasso_s {
   cudaEvent_t* prof_events;
   long long prof_cap, prof_rounds;
   // strads_run replays one captured round (the launch sequence of a round is fixed for a handle)
+  int walk_grid;            // CTAs of the cooperative on-demand walk (CSC)
   cudaStream_t capture_stream;
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
@@ -44,7 +45,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_dbeta, off_dbeta64,
-      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, total;
+      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles;
   long long ldc;
 };
@@ -92,6 +93,10 @@ Layout carve(const strads_lasso_config_t* c) {
   L.off_xc = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(float) * (size_t)c->n_candidates * L.ldc : 0);
   L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)
   L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
+  const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
+  L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
+  L.off_walk_rows = take(csc ? sizeof(unsigned int) * 32 * (size_t)L.mask_words : 0);
+  L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
   L.total = o;
   return L;
 }
@@ -100,10 +105,11 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
-cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, bool only_if_short) {
+cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
+                        bool window = false) {
   const Problem& p = h->p;
   cudaStream_t s = h->stream;
-  if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, s);
+  if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, window, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
   return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, s);
 }
@@ -126,12 +132,17 @@ int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_
     return STRADS_OK;
   }
   const int window = gram_dbg != nullptr ? n_cand : window_of(p, n_cand);
-  CK(launch_gram(h, cand, window, gram_dbg, false));
+  CK(launch_gram(h, cand, window, gram_dbg, false, window < n_cand));
   if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
   CK(launch_filter(p, cand, window, n_cand, false, p.kept, h->stream));
   if (window < n_cand) {
-    CK(launch_gram(h, cand, n_cand, nullptr, true));
-    CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, h->stream));
+    if (p.layout == STRADS_CSC) {
+      // whole list, conflict rows formed only for the candidates the walk keeps
+      CK(launch_walk_csc(p, cand, n_cand, h->walk_grid, true, p.kept, h->stream));
+    } else {
+      CK(launch_gram(h, cand, n_cand, nullptr, true));
+      CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, h->stream));
+    }
   }
   return STRADS_OK;
 }
@@ -214,6 +225,9 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   p.xc = reinterpret_cast<float*>(ws + L.off_xc);
   p.ldc = L.ldc;
   p.cand_cur = nullptr;
+  p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
+  p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
+  p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
   p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
   p.partial_tiles = L.partial_tiles;
   h->stream = static_cast<cudaStream_t>(c->stream);
@@ -231,6 +245,12 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
   if (p.layout == STRADS_DENSE_COLMAJOR && (e = encode_gram_tensor_map(p, h->gram_tmap)) != cudaSuccess)
     return fail(cuda_fail(e, "encode_gram_tensor_map"));
+  h->walk_grid = 0;
+  if (p.layout == STRADS_CSC) {
+    if ((e = prepare_walk_csc(p, &h->walk_grid)) != cudaSuccess) return fail(cuda_fail(e, "prepare_walk_csc"));
+    if ((e = cudaMemsetAsync(p.walk_ctl, 0, sizeof(WalkControl), h->stream)) != cudaSuccess)
+      return fail(cuda_fail(e, "cudaMemsetAsync"));
+  }
   if ((e = launch_init(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
   if ((e = launch_resid_from_beta(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
   *out_handle = h;

@@ -22,6 +22,10 @@ constexpr int kBatch = 32;
 __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
                                                       int only_if_short, int* __restrict__ kept_out) {
   if (only_if_short && !p.st->window_short) return;
+  if (p.layout == STRADS_CSC && n_cand < n_total && p.st->prefer_walk && (p.st->round & 63ull) != 0) {
+    if (threadIdx.x == 0) p.st->window_short = 1;    // window attempt skipped: go straight to the whole-list walk
+    return;
+  }
   extern __shared__ unsigned int sm[];
   const int W = p.mask_words;
   const int Ws = W | 1;                          // odd row pitch: column reads of `rows` hit 32 different banks
@@ -172,6 +176,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (tid == 0) {
     p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0;
     p.st->window_short = (!only_if_short && nk < p.n_keep && n_cand < n_total) ? 1 : 0;
+    if (!only_if_short && n_cand < n_total && !p.st->window_short) p.st->prefer_walk = 0;
   }
 }
 

@@ -12,8 +12,9 @@ constexpr int kThreads = 256;
 constexpr int kStage = 1024;          // entries of column a staged in shared memory (longer columns: global)
 
 __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __restrict__ cand, int n_cand,
-                                                        float* __restrict__ gram_dbg, int only_if_short) {
+                                                        float* __restrict__ gram_dbg, int only_if_short, int window) {
   if (only_if_short && !p.st->window_short) return;
+  if (window && p.st->prefer_walk && (p.st->round & 63ull) != 0) return;   // the window attempt is being skipped
   __shared__ int arow[kStage];
   __shared__ float aval[kStage];
   const int a = blockIdx.x;
@@ -36,26 +37,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
     bool hit = false;
     if (b < n_cand && b != a) {
       const int jb = cand[b];
-      long long q = p.xptr[jb];
-      const long long qe = p.xptr[jb + 1];
-      float dot = 0.f;
-      int i = 0;
-      if (q < qe && na > 0) {
-        int rb = __ldg(p.xrow + q), ra = ar[0];
-        while (true) {
-          if (ra == rb) {
-            dot = fmaf(av[i], __ldg(p.xv + q), dot);
-            if (++i >= na || ++q >= qe) break;
-            ra = ar[i]; rb = __ldg(p.xrow + q);
-          } else if (ra < rb) {
-            if (++i >= na) break;
-            ra = ar[i];
-          } else {
-            if (++q >= qe) break;
-            rb = __ldg(p.xrow + q);
-          }
-        }
-      }
+      const float dot = sparse_dot(ar, av, na, p, jb);
       const double den = sqrt(n2a * p.n2[jb]);
       hit = den > 0.0 && fabs((double)dot) >= rho * den;
       if (gram_dbg != nullptr) {
@@ -73,8 +55,8 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
 }  // namespace
 
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
-                            cudaStream_t s) {
-  k_gram_csc<<<n_cand, kThreads, 0, s>>>(p, cand, n_cand, gram_dbg, only_if_short ? 1 : 0);
+                            bool window, cudaStream_t s) {
+  k_gram_csc<<<n_cand, kThreads, 0, s>>>(p, cand, n_cand, gram_dbg, only_if_short ? 1 : 0, window ? 1 : 0);
   return cudaGetLastError();
 }
 

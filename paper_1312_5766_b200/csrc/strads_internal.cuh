@@ -31,7 +31,16 @@ struct DeviceState {
   int beta0_nonzero;            // set at init when the starting beta has a non-zero entry
   unsigned int amb_count;       // pairs the TF32 screen of the dense Gram left to the exact recheck
   int window_short;             // the filter ran out of its candidate window before P were kept: redo on all P'
-  unsigned int pad[2];
+  int prefer_walk;              // CSC: the last round needed the whole list, so skip the window attempt for a while
+  unsigned int pad;
+};
+
+struct WalkControl {            // shared by the CTAs of the cooperative on-demand walk (CSC)
+  unsigned int bar_count, bar_gen;   // grid barrier
+  int m;                        // batch size (0: list exhausted)
+  int cursor, n_kept, examined, done, failed;
+  int pos[32];                  // positions of the batch in the candidate list
+  int cval[32];                 // their coefficient indices
 };
 
 static constexpr int kHistBits = 12;
@@ -76,6 +85,9 @@ struct Problem {
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
   float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
   int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles
+  unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words]
+  unsigned int* walk_rows;      // [32][mask_words] conflict rows of the batch in flight
+  WalkControl* walk_ctl;
   int sm_count;
 };
 static constexpr int kObjBlocks = 296;
@@ -146,6 +158,32 @@ __device__ __forceinline__ unsigned long long race_key64(float delta_j, float et
   return ((unsigned long long)__float_as_uint(T) << 32) | j;
 }
 
+// x_a^T x_b of two CSC columns (ascending rows): a given as arrays (possibly staged in shared memory), b read
+// from X.  Products are added in row order, so every kernel that uses this gets the same bits.
+__device__ __forceinline__ float sparse_dot(const int* ar, const float* av, int na, const Problem& p, int jb) {
+  long long q = p.xptr[jb];
+  const long long qe = p.xptr[jb + 1];
+  float dot = 0.f;
+  int i = 0;
+  if (q < qe && na > 0) {
+    int rb = __ldg(p.xrow + q), ra = ar[0];
+    while (true) {
+      if (ra == rb) {
+        dot = fmaf(av[i], __ldg(p.xv + q), dot);
+        if (++i >= na || ++q >= qe) break;
+        ra = ar[i]; rb = __ldg(p.xrow + q);
+      } else if (ra < rb) {
+        if (++i >= na) break;
+        ra = ar[i];
+      } else {
+        if (++q >= qe) break;
+        rb = __ldg(p.xrow + q);
+      }
+    }
+  }
+  return dot;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Launchers (one per step; all enqueue on `s` and return a cudaError_t).
 // ---------------------------------------------------------------------------------------------
@@ -162,9 +200,13 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
 cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
                                  cudaStream_t s);
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
-                            cudaStream_t s);
+                            bool window, cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);
 // Walks cand[0 .. n_cand); n_total >= n_cand is the length of the whole list (n_cand < n_total: a window).
+// CSC: greedy walk that forms conflict rows only for the candidates it is about to keep (cooperative kernel).
+cudaError_t prepare_walk_csc(const Problem& p, int* grid_out);
+cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int grid, bool only_if_short, int* kept_out,
+                            cudaStream_t s);
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s);
 cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s);
