@@ -297,10 +297,10 @@ def main():
                         "sample": f"{rounds} full oracle rounds of {args.workload} from the state after the timed "
                                   f"region ({sec:.1f} s, single thread; host has {os.cpu_count()} cores)"}
 
-    # kernels per round: sampler 3, window Gram (dense: pack, screen, split-K reduce, recheck, 3xTF32 gate = 5;
+    # kernels per round: sampler 4, window Gram (dense: pack, screen, split-K reduce, recheck, 3xTF32 gate = 5;
     # CSC: 1), walk 1, whole-list retry (dense 4 + 1, CSC: the on-demand walk, 1; they return at once when not
     # needed), update 2
-    launches_per_round = 3 + (5 + 1 + 5 if p.layout == wl.DENSE else 1 + 1 + 1) + 2
+    launches_per_round = 4 + (5 + 1 + 5 if p.layout == wl.DENSE else 1 + 1 + 1) + 2
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

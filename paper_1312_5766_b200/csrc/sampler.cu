@@ -12,7 +12,8 @@
 //                    expectation whatever the weights are; if it ever exceeds the boundary buffer,
 //                    that CTA alone refines the boundary over further 12-bit digits (rare, exact).
 //   k_sample_collect pass 2: appends "sure" and "boundary" keys to two small buffers.
-//   k_sample_sort    one CTA: bitonic sort of both buffers in shared memory, writes cand[P'].
+//   k_sample_sort_chunks / k_sample_rank   order the winners: 1024-key chunks sorted in shared memory by
+//                    one CTA each, then every key's rank by binary search in the other chunks.
 #include <cstddef>
 #include <mutex>
 
@@ -110,6 +111,8 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
   find_bin(sh, kHistBins, p.n_cand, &s_bin, &s_before);
   if (tid == 0) {
     p.st->hist_ticket = 0;
+    p.st->sure_count = 0;                             // append cursors of the collect pass that follows
+    p.st->boundary_count = 0;
     s_sel.prefix = (unsigned long long)s_bin;
     s_sel.bits = kHistBits;
     s_sel.n_sure = (int)s_before;
@@ -180,45 +183,79 @@ __device__ void bitonic_sort(unsigned long long* a, int n) {
 
 __device__ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
-__global__ void __launch_bounds__(1024) k_sample_sort(Problem p, int* cand_out) {
-  extern __shared__ unsigned long long keys[];
+constexpr int kChunk = 1024;             // keys sorted by one CTA
+
+// Which slice of which buffer CTA `c` owns: sure chunks first, then boundary chunks.
+struct ChunkRef { unsigned long long* base; int n; int first; bool is_sure; };
+__device__ __forceinline__ ChunkRef chunk_of(const Problem& p, const SelectState& sel, int c) {
+  const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
+  const int sure_chunks = (p.cap_sure + kChunk - 1) / kChunk;
+  ChunkRef r;
+  r.is_sure = c < sure_chunks;
+  const int ci = r.is_sure ? c : c - sure_chunks;
+  const int total = r.is_sure ? n_sure : n_bnd;
+  r.first = ci * kChunk;
+  r.n = max(0, min(kChunk, total - r.first));
+  r.base = (r.is_sure ? p.sure : p.boundary) + r.first;
+  return r;
+}
+
+// Step 1 of the final ordering: every CTA sorts one chunk of up to 1024 collected keys in shared memory
+// (bitonic) and writes it back in place.  One CTA sorting all P' keys would be bound by its own shared-memory
+// bandwidth (~100 us for 16,384 keys); chunks run on as many SMs as there are chunks.
+__global__ void __launch_bounds__(512) k_sample_sort_chunks(Problem p) {
+  __shared__ unsigned long long keys[kChunk];
   const SelectState sel = p.st->sel;
-  const int n_sure = min(sel.n_sure, p.cap_sure);
-  const int n_bnd = min(sel.n_boundary, p.cap_boundary);
-  const int need = p.n_cand - n_sure;              // winners taken from the boundary set
-  int n = pow2_ceil(max(n_sure, 1));
-  for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = i < n_sure ? p.sure[i] : ~0ull;
+  const ChunkRef ch = chunk_of(p, sel, blockIdx.x);
+  if (ch.n == 0) return;
+  const int n = pow2_ceil(ch.n);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = i < ch.n ? ch.base[i] : ~0ull;
   __syncthreads();
   bitonic_sort(keys, n);
-  for (int i = threadIdx.x; i < n_sure; i += blockDim.x) cand_out[i] = (int)(keys[i] & 0xffffffffull);
-  __syncthreads();
-  n = pow2_ceil(max(n_bnd, 1));
-  for (int i = threadIdx.x; i < n; i += blockDim.x) keys[i] = i < n_bnd ? p.boundary[i] : ~0ull;
-  __syncthreads();
-  bitonic_sort(keys, n);
-  for (int i = threadIdx.x; i < need && i < n_bnd; i += blockDim.x)
-    cand_out[n_sure + i] = (int)(keys[i] & 0xffffffffull);
-  if (threadIdx.x == 0) {
-    p.st->sure_count = 0;
-    p.st->boundary_count = 0;
-    p.st->counts[0] = p.n_cand;
+  for (int i = threadIdx.x; i < ch.n; i += blockDim.x) ch.base[i] = keys[i];
+}
+
+// Number of keys < key in a sorted array (keys are distinct).
+__device__ __forceinline__ int count_less(const unsigned long long* a, int n, unsigned long long key) {
+  int lo = 0, hi = n;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (a[mid] < key) lo = mid + 1; else hi = mid;
   }
+  return lo;
+}
+
+// Step 2: the rank of a key among all collected keys = its index in its own chunk + the number of smaller
+// keys in every other chunk of its buffer (+ n_sure for boundary keys: every sure key is smaller).  The key
+// of rank r < P' is candidate r.  Each other chunk is staged in shared memory and searched there.
+__global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
+  __shared__ unsigned long long other[kChunk];
+  const SelectState sel = p.st->sel;
+  const ChunkRef ch = chunk_of(p, sel, blockIdx.x);
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
+  if (ch.n == 0) return;
+  const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
+  const unsigned long long* buf = ch.is_sure ? p.sure : p.boundary;
+  const int total = ch.is_sure ? n_sure : n_bnd;
+  const int i0 = threadIdx.x, i1 = threadIdx.x + 512;           // this thread's (up to) two keys
+  const unsigned long long k0 = i0 < ch.n ? __ldcg(ch.base + i0) : 0ull, k1 = i1 < ch.n ? __ldcg(ch.base + i1) : 0ull;
+  int r0 = i0 + (ch.is_sure ? 0 : n_sure), r1 = i1 + (ch.is_sure ? 0 : n_sure);
+  for (int o = 0; o < total; o += kChunk) {
+    if (o == ch.first) continue;
+    const int n = min(kChunk, total - o);
+    __syncthreads();
+    for (int e = threadIdx.x; e < n; e += 512) other[e] = __ldcg(buf + o + e);
+    __syncthreads();
+    r0 += count_less(other, n, k0);
+    r1 += count_less(other, n, k1);
+  }
+  if (i0 < ch.n && r0 < p.n_cand) cand_out[r0] = (int)(k0 & 0xffffffffull);
+  if (i1 < ch.n && r1 < p.n_cand) cand_out[r1] = (int)(k1 & 0xffffffffull);
 }
 
 }  // namespace
 
-static size_t sort_smem_bytes(const Problem& p) {
-  int n = 1;
-  while (n < p.cap_sure || n < p.cap_boundary) n <<= 1;
-  return (size_t)n * sizeof(unsigned long long);
-}
-
-// The attribute belongs to the kernel, not to a handle: always ask for the largest size any handle can
-// need, so that a later handle with fewer candidates does not lower the limit under an earlier one.
-cudaError_t prepare_sample(const Problem&) {
-  return cudaFuncSetAttribute(k_sample_sort, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)(STRADS_MAX_CANDIDATES * sizeof(unsigned long long)));
-}
+cudaError_t prepare_sample(const Problem&) { return cudaSuccess; }
 
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   const long long groups = (p.J + 3) >> 2;
@@ -228,7 +265,9 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   if (blocks < 1) blocks = 1;
   k_sample_hist<<<(unsigned)blocks, kThreads, 0, s>>>(p);
   k_sample_collect<<<(unsigned)blocks, kThreads, 0, s>>>(p);
-  k_sample_sort<<<1, 1024, sort_smem_bytes(p), s>>>(p, cand_out);
+  const int chunks = (p.cap_sure + kChunk - 1) / kChunk + (p.cap_boundary + kChunk - 1) / kChunk;
+  k_sample_sort_chunks<<<chunks, 512, 0, s>>>(p);
+  k_sample_rank<<<chunks, 512, 0, s>>>(p, cand_out);
   return cudaGetLastError();
 }
 
