@@ -44,7 +44,7 @@ size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
 int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
-  size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_dbeta, off_dbeta64,
+  size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles;
   long long ldc;
@@ -81,6 +81,7 @@ Layout carve(const strads_lasso_config_t* c) {
   L.off_boundary = take(sizeof(unsigned long long) * (size_t)L.cap_boundary);
   L.off_cand = take(sizeof(int) * (size_t)c->n_candidates);
   L.off_kept = take(sizeof(int) * (size_t)c->n_keep);
+  L.off_kept_pos = take(sizeof(int) * (size_t)c->n_keep);
   L.off_dbeta = take(sizeof(float) * (size_t)c->n_keep);
   L.off_dbeta64 = take(sizeof(double) * (size_t)c->n_keep);
   L.off_conflict = take(sizeof(unsigned int) * (size_t)c->n_candidates * L.mask_words);
@@ -158,7 +159,10 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
     if (rc) return rc;
   }
   if (ev) CK(cudaEventRecord(ev[3], h->stream));
-  CK(launch_update(p, p.kept, 1, h->stream));
+  // after a tensor-core Gram the kept columns are read from the packed candidate buffer
+  const bool packed = p.layout == STRADS_DENSE_COLMAJOR && !(p.flags & (STRADS_FLAG_NO_FILTER | STRADS_FLAG_SIMT_GRAM)) &&
+                      !(out && out->gram);
+  CK(launch_update(p, p.kept, 1, packed, h->stream));
   if (ev) { CK(cudaEventRecord(ev[4], h->stream)); h->prof_rounds += 1; }
   h->round_host += 1;
   if (out != nullptr) {
@@ -212,6 +216,7 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   p.cap_sure = L.cap_sure; p.cap_boundary = L.cap_boundary;
   p.cand = reinterpret_cast<int*>(ws + L.off_cand);
   p.kept = reinterpret_cast<int*>(ws + L.off_kept);
+  p.kept_pos = reinterpret_cast<int*>(ws + L.off_kept_pos);
   p.dbeta = reinterpret_cast<float*>(ws + L.off_dbeta);
   p.dbeta64 = reinterpret_cast<double*>(ws + L.off_dbeta64);
   p.conflict = reinterpret_cast<unsigned int*>(ws + L.off_conflict);
@@ -353,7 +358,7 @@ int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, fl
   CK(launch_set_counts(p, n_kept, n_kept, n_kept, h->stream));
   if (n_kept > 0)
     CK(cudaMemcpyAsync(p.kept, kept_dev, sizeof(int) * n_kept, cudaMemcpyDeviceToDevice, h->stream));
-  CK(launch_update(p, p.kept, 0, h->stream));
+  CK(launch_update(p, p.kept, 0, false, h->stream));
   if (dbeta_dev) CK(launch_export(p, p.kept, nullptr, dbeta_dev, nullptr, h->stream));
   return STRADS_OK;
 }

@@ -143,7 +143,11 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
         while (__popc(keep) > room) keep &= ~(1u << (31 - __clz(keep)));
         full = true;
       }
-      if ((keep >> lane) & 1u) kept_out[nk + __popc(keep & ((1u << lane) - 1u))] = cval[lane];
+      if ((keep >> lane) & 1u) {
+        const int slot = nk + __popc(keep & ((1u << lane) - 1u));
+        kept_out[slot] = cval[lane];
+        p.kept_pos[slot] = pos[lane];
+      }
       if (lane == 0) {
         s_keepmask = keep;
         s_kept = nk + __popc(keep);

@@ -48,7 +48,15 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
 // ------------------------------------------------------------------------------------------------
 // dense
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __restrict__ kept) {
+// Where the kept columns are read from.  After a tensor-core Gram they sit, contiguous and still in L2, in
+// the packed candidate buffer (row = position in the candidate list); otherwise in X itself.
+struct ColumnSource {
+  const float* base;
+  long long pitch;
+  const int* index;     // [n_kept]: packed: position in the candidate list; else: coefficient index
+};
+
+__global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __restrict__ kept, ColumnSource src) {
   const int a = blockIdx.y;
   if (a >= p.st->counts[2]) {
     if (blockIdx.x == 0 && threadIdx.x == 0) p.dbeta[a] = 0.f;
@@ -56,7 +64,7 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
   }
   const int part = blockIdx.x, parts = gridDim.x;
   const int j = kept[a];
-  const float* x = p.xv + (long long)j * p.ld;
+  const float* x = src.base + (long long)src.index[a] * src.pitch;
   const long long n4 = (p.N + 3) >> 2;                       // float4 groups (the last may be partial)
   const long long per = (n4 + parts - 1) / parts;
   const long long g0 = part * per, g1 = min(n4, g0 + per);
@@ -80,7 +88,6 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
     acc1 += (double)xv.y * (double)rv.y + (double)xv.w * (double)rv.w;
   }
   __shared__ double wsum[kThreads / 32];
-  __shared__ int s_last;
   double v = warp_sum(acc0 + acc1);
   if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = v;
   __syncthreads();
@@ -89,8 +96,7 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
     for (int w = 0; w < kThreads / 32; ++w) s += wsum[w];
     p.dot_partial[(long long)a * parts + part] = s;
     __threadfence();
-    s_last = atomicAdd(&p.dot_ticket[a], 1u) == (unsigned)parts - 1;
-    if (s_last) {
+    if (atomicAdd(&p.dot_ticket[a], 1u) == (unsigned)parts - 1) {   // last part of this column: finish it
       __threadfence();
       double g = 0.0;
       for (int q = 0; q < parts; ++q) g += __ldcg(&p.dot_partial[(long long)a * parts + q]);
@@ -100,31 +106,48 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
   }
 }
 
-constexpr int kRowsPerCta = 128;       // 32 lanes x float4
+// r <- r - sum_a x_a dbeta_a with every row owned by one CTA: 64 rows per CTA, a half-warp per column
+// (16 lanes x float4), so a warp reads two columns per instruction and the 16 half-warps of the CTA take the
+// kept columns round-robin, four loads in flight each.  The per-row sums of the half-warps are added in a
+// fixed order.
+constexpr int kRowsPerCta = 64;
+constexpr int kColSlots = kThreads / 16;   // half-warps per CTA
 
-__global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* __restrict__ kept, int advance) {
-  __shared__ double part[kThreads / 32][kRowsPerCta];
+__global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSource src, int advance) {
+  __shared__ double part[kColSlots][kRowsPerCta];
   const int n_kept = p.st->counts[2];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const long long i = (long long)blockIdx.x * kRowsPerCta + lane * 4;
+  const int slot = threadIdx.x >> 4, l16 = threadIdx.x & 15;
+  const long long i = (long long)blockIdx.x * kRowsPerCta + l16 * 4;
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
   if (i < p.N) {
-    for (int a = warp; a < n_kept; a += kThreads / 32) {
-      const double d = p.dbeta64[a];
-      if (d == 0.0) continue;
-      const float4 xv = __ldg(reinterpret_cast<const float4*>(p.xv + (long long)kept[a] * p.ld + i));
-      s0 += (double)xv.x * d; s1 += (double)xv.y * d; s2 += (double)xv.z * d; s3 += (double)xv.w * d;
+    for (int a0 = slot; a0 < n_kept; a0 += kColSlots * 4) {
+      float4 xv[4];
+      double d[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int a = a0 + u * kColSlots;
+        d[u] = a < n_kept ? p.dbeta64[a] : 0.0;
+        const int ai = a < n_kept ? a : a0;
+        xv[u] = __ldg(reinterpret_cast<const float4*>(src.base + (long long)src.index[ai] * src.pitch + i));
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        if (d[u] != 0.0) {
+          s0 += (double)xv[u].x * d[u]; s1 += (double)xv[u].y * d[u];
+          s2 += (double)xv[u].z * d[u]; s3 += (double)xv[u].w * d[u];
+        }
+      }
     }
   }
-  part[warp][lane * 4 + 0] = s0; part[warp][lane * 4 + 1] = s1;
-  part[warp][lane * 4 + 2] = s2; part[warp][lane * 4 + 3] = s3;
+  part[slot][l16 * 4 + 0] = s0; part[slot][l16 * 4 + 1] = s1;
+  part[slot][l16 * 4 + 2] = s2; part[slot][l16 * 4 + 3] = s3;
   __syncthreads();
   if (threadIdx.x < kRowsPerCta) {
     const long long r = (long long)blockIdx.x * kRowsPerCta + threadIdx.x;
     if (r < p.N) {
       double s = 0.0;
 #pragma unroll
-      for (int w = 0; w < kThreads / 32; ++w) s += part[w][threadIdx.x];
+      for (int w = 0; w < kColSlots; ++w) s += part[w][threadIdx.x];
       if (s != 0.0) p.resid[r] = (float)((double)p.resid[r] - s);
     }
   }
@@ -227,10 +250,15 @@ __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta
 
 }  // namespace
 
-cudaError_t launch_update(const Problem& p, const int* kept, int advance, cudaStream_t s) {
+// from_packed: the kept columns are rows p.kept_pos[.] of the packed candidate buffer (dense, after a
+// tensor-core Gram of this round); otherwise they are read from X.
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s) {
   if (p.layout == STRADS_DENSE_COLMAJOR) {
-    k_dot_dense<<<dim3(p.dot_parts, p.n_keep), kThreads, 0, s>>>(p, kept);
-    k_apply_dense<<<(unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s>>>(p, kept, advance);
+    ColumnSource src;
+    if (from_packed) { src.base = p.xc; src.pitch = p.ldc; src.index = p.kept_pos; }
+    else { src.base = p.xv; src.pitch = p.ld; src.index = kept; }
+    k_dot_dense<<<dim3(p.dot_parts, p.n_keep), kThreads, 0, s>>>(p, kept, src);
+    k_apply_dense<<<(unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s>>>(p, src, advance);
   } else {
     k_dot_csc<<<(p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(p, kept);
     long long grid = (long long)p.sm_count * 2;
