@@ -384,40 +384,55 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 }
 
 // Split-K: sums the partial tiles of one output tile in split order and thresholds (screen rules).
-// One CTA per (tile, 32 rows); thread = (row, 32-column chunk).
-__global__ void __launch_bounds__(128) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short) {
+// One CTA per (tile, 8 rows); a warp owns one row, a lane four of its 128 columns.
+__global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short) {
   if (only_if_short && !p.st->window_short) return;
-  __shared__ double normB[kTile];
-  const int tile = blockIdx.x >> 2, rgroup = blockIdx.x & 3;
+  const int tile = blockIdx.x >> 4, rgroup = blockIdx.x & 15;
   int ti = 0, rem = tile;
   while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
   const int tj = ti + rem;
-  {
-    const int gb = tj * kTile + threadIdx.x;
-    normB[threadIdx.x] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
-  }
-  __syncthreads();
-  const int la = rgroup * 32 + (threadIdx.x >> 2), c = threadIdx.x & 3;
+  const int lane = threadIdx.x & 31;
+  const int la = rgroup * 8 + (threadIdx.x >> 5);
   const int a = ti * kTile + la;
-  float acc[32];
+  const float4* src = reinterpret_cast<const float4*>(p.gram_partial + ((size_t)tile * n_split * kTile + la) * kTile) + lane;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  int s = 0;
+  for (; s + 4 <= n_split; s += 4) {                   // four loads in flight, added in split order
+    float4 u[4];
 #pragma unroll
-  for (int j = 0; j < 32; ++j) acc[j] = 0.f;
-  for (int s = 0; s < n_split; ++s) {
-    const float4* src = reinterpret_cast<const float4*>(p.gram_partial + (((size_t)tile * n_split + s) * kTile + la) * kTile + c * 32);
+    for (int k = 0; k < 4; ++k) u[k] = __ldcg(src + (size_t)(s + k) * (kTile * kTile / 4));
 #pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float4 u = __ldcg(src + j);
-      acc[4 * j] += u.x; acc[4 * j + 1] += u.y; acc[4 * j + 2] += u.z; acc[4 * j + 3] += u.w;
-    }
+    for (int k = 0; k < 4; ++k) { acc.x += u[k].x; acc.y += u[k].y; acc.z += u[k].z; acc.w += u[k].w; }
   }
-  uint32_t v[32];
-#pragma unroll
-  for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(acc[j]);
+  for (; s < n_split; ++s) {
+    const float4 u = __ldcg(src + (size_t)s * (kTile * kTile / 4));
+    acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
+  }
   const double norm_a = a < n_cand ? sqrt(p.n2[p.cand_cur[a]]) : 0.0;
-  const uint32_t word = decide_word<true>(p, v, a, tj * kTile + c * 32, n_cand, norm_a, normB + c * 32, (double)p.rho,
-                                          screen_band(p.N));
-  const int widx = tj * (kTile / 32) + c;
-  if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+  const double rho = (double)p.rho, band = screen_band(p.N);
+  const float g4[4] = {acc.x, acc.y, acc.z, acc.w};
+  unsigned int nib = 0u;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int b = tj * kTile + lane * 4 + k;
+    const double norm_b = b < n_cand ? sqrt(p.n2[p.cand_cur[b]]) : 0.0;
+    const double den = norm_a * norm_b;
+    const double g = fabs((double)g4[k]);
+    const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
+    bool hit = live && g >= rho * den;
+    if (live && b > a && fabs(g - rho * den) <= band * den) {
+      hit = false;                                     // too close to call: k_gram_recheck decides
+      const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
+      if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
+    }
+    nib |= (unsigned int)hit << k;
+  }
+  unsigned int word = nib << ((lane & 7) * 4);         // 8 lanes make one 32-column mask word
+  word |= __shfl_xor_sync(0xffffffffu, word, 1);
+  word |= __shfl_xor_sync(0xffffffffu, word, 2);
+  word |= __shfl_xor_sync(0xffffffffu, word, 4);
+  const int widx = tj * (kTile / 32) + (lane >> 3);
+  if ((lane & 7) == 0 && a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
 }
 
 // Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product of the
@@ -507,7 +522,7 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand, ois);
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
     k_gram_dense_tc<false><<<tiles * n_split, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, n_split, ois);
-    if (n_split > 1) k_gram_reduce<<<tiles * 4, 128, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
+    if (n_split > 1) k_gram_reduce<<<tiles * 16, 256, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
     k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q, ois);
   }
   k_gram_dense_tc<true><<<tiles, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, 1, ois);

@@ -101,9 +101,16 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
 
   // ---- last CTA: every other CTA's histogram is visible now ----
   __threadfence();
-  for (int b = tid; b < kHistBins; b += kThreads) {
-    sh[b] = __ldcg(&p.hist[b]);
-    p.hist[b] = 0;                                   // ready for the next round
+  {
+    // all loads first, then the stores (a store between two loads would order them: one round trip per bin)
+    unsigned int v[kHistBins / kThreads];
+#pragma unroll
+    for (int u = 0; u < kHistBins / kThreads; ++u) v[u] = __ldcg(&p.hist[tid + u * kThreads]);
+#pragma unroll
+    for (int u = 0; u < kHistBins / kThreads; ++u) {
+      sh[tid + u * kThreads] = v[u];
+      p.hist[tid + u * kThreads] = 0;                 // ready for the next round
+    }
   }
   __syncthreads();
   __shared__ int s_bin;
