@@ -453,3 +453,23 @@ def test_window_equals_full_gram(name, n_keep):
     if (name, n_keep) in (("dense_grouped", 120), ("csc_zipf", 300)):
         assert shorts > 0                        # these did exercise the whole-list retry
     assert lazy.status()[0] == 0
+
+
+@pytest.mark.parametrize("name,n_keep,n_cand", [("dense", 24, 1024), ("dense_grouped", 120, 1024), ("dense_grouped", 40, 1024),
+                                                ("csc", 100, 1000), ("csc_zipf", 300, 1500)])
+def test_graph_replay_equals_round_by_round(name, n_keep, n_cand):
+    """strads_run replays a captured graph in which the 3xTF32 fallback and the whole-list retry are IF nodes;
+    the state it leaves must be bit-identical to calling strads_round the same number of times."""
+    cfg = dict(_small_problems()[name], n_keep=n_keep, n_candidates=n_cand)
+    p = wl.make_problem(cfg, seed=14)
+    a, b = _solver(p), _solver(p)
+    n = 70                                            # crosses round 64, where a skipped window is tried again
+    a.run(n)
+    kept_total = 0
+    for _ in range(n):
+        kept_total += int(b.round()[3][2])
+    assert a.get_round() == b.get_round() == n
+    for x, y in ((a.beta, b.beta), (a.resid, b.resid), (a.delta, b.delta)):
+        assert torch.equal(x, y)
+    assert a.totals() == b.totals() and a.totals()["kept"] == kept_total
+    assert a.status()[0] == 0 and b.status()[0] == 0
