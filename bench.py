@@ -30,7 +30,10 @@ from paper_1312_5766_b200 import workloads as wl  # noqa: E402
 
 METRIC = "coordinate updates/sec and % of HBM roofline per STRADS round (1xB200)"
 UNIT = "coordinate updates/s"
-SM_COUNT, FMA_LANES_PER_SM = 148, 128
+# DRAM bytes (read + write) per launch of the window-Gram kernels from ncu (dram__bytes_read.sum +
+# dram__bytes_write.sum; profiles/k_gram_dense_tc_window_c2.md), keyed by (workload, window).  The capture was made
+# with J cut to 20,000; the window kernels read the packed window only, so their traffic does not depend on J.
+GRAM_WINDOW_TRAFFIC = {("c2", 512): 20.6e6}
 
 
 def measured_peaks():
@@ -236,33 +239,53 @@ def main():
     objective = s.objective()
     rc, status_bits = s.status()
 
-    # ---- roofline of the dominant kernel (dense: the candidate Gram, an FP32 contraction) ----------
+    # ---- roofline -----------------------------------------------------------------------------------------
     peaks = measured_peaks()
-    step_ms = {k: prof[k] / max(prof["rounds"], 1) for k in ("sample_ms", "gram_ms", "filter_ms", "update_ms")}
+    step_ms = {k: prof[k] / max(prof["rounds"], 1) for k in ("sample_ms", "pack_ms", "gram_ms", "walk_ms", "update_ms")}
+    kept_per_round = kept_local / args.steps
+    # the Gram is formed on a leading window of the candidates (the library's rule: 1.5 P + 128 rounded up to 128,
+    # used when at most half the list)
+    window = (p.n_keep + p.n_keep // 2 + 128 + 127) // 128 * 128
+    if 2 * window > p.n_candidates:
+        window = p.n_candidates
     if p.layout == wl.DENSE:
-        # algorithmic flops P'(P'-1)N (upper triangle, 2 flop per multiply-add); the kernel issues 3 TF32 MMAs per
-        # product (3xTF32), so the tensor pipe does 3x this -- `achieved` counts the algorithmic flops only
-        flops = float(p.n_candidates) * (p.n_candidates - 1) * p.n_rows
+        # dominant kernel: the tensor-core Gram of the window (k_gram_dense_tc screen + its split-K reduce and the
+        # exact recheck, timed together).  Algorithmic flops W(W-1)N: upper triangle, 2 flop per multiply-add.
+        flops = float(window) * (window - 1) * p.n_rows
         achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
-        peak = peaks["bf16_tflops_sustained"] * 0.5          # TF32 dense = half the BF16 rate (nominal 1.1 vs 2.25 PF)
-        roofline = {"kernel": "k_gram_dense_tc", "bound": "tensor", "achieved": achieved, "peak": peak,
-                    "unit": "TFLOP/s", "frac": achieved / peak, "traffic": None,
-                    "tensor_issue_factor": 3,
-                    "peak_source": f"{peaks['source']} BF16 sustained x 0.5 (nominal TF32:BF16 ratio)"}
+        peak = peaks["bf16_tflops"] * 0.5                    # TF32 dense = half the BF16 rate (nominal 1.1 vs 2.25 PF)
+        roofline = {"kernel": "k_gram_dense_tc<screen> (+ k_gram_reduce, k_gram_recheck)", "bound": "tensor",
+                    "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                    "traffic": GRAM_WINDOW_TRAFFIC.get((args.workload, window)),
+                    "window": window, "launch_ms": step_ms["gram_ms"],
+                    "peak_source": f"{peaks['source']} BF16 burst x 0.5 (nominal TF32:BF16 ratio); the kernel is timed "
+                                   "alone between events"}
     else:
+        # dominant kernel: the pair merges of the window (k_gram_csc); bytes: each window column once
         nnz_col = p.nnz / p.n_cols
-        byts = 8.0 * nnz_col * p.n_candidates
+        byts = 8.0 * nnz_col * window
         achieved = byts / (step_ms["gram_ms"] * 1e-3) / 1e9
         roofline = {"kernel": "k_gram_csc", "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"],
-                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None,
-                    "peak_source": peaks["source"]}
-    # the update kernels against the HBM roofline (bytes: kept columns once + r read and written)
-    kept_per_round = kept_local / args.steps
+                    "unit": "GB/s", "frac": achieved / peaks["hbm_gbs"], "traffic": None, "window": window,
+                    "launch_ms": step_ms["gram_ms"], "peak_source": peaks["source"],
+                    "note": "a few MB of columns against ~1e6 sorted-list merges: bound by ALU/latency, not by HBM"}
+    # streaming kernels against the HBM roofline: pack (window columns read + written) and update (kept columns once
+    # + r read and written)
     if p.layout == wl.DENSE:
         upd_bytes = 4.0 * p.n_rows * kept_per_round + 8.0 * p.n_rows + 16.0 * kept_per_round
+        pack_bytes = 8.0 * p.n_rows * window
     else:
         upd_bytes = 8.0 * (p.nnz / p.n_cols) * kept_per_round + 8.0 * p.n_rows
+        pack_bytes = 0.0
     upd_gbs = upd_bytes / (step_ms["update_ms"] * 1e-3) / 1e9
+    pack_gbs = pack_bytes / (step_ms["pack_ms"] * 1e-3) / 1e9 if pack_bytes else None
+    # the metric's own byte count per round (all P' candidate columns + kept columns + r twice) over the round time:
+    # what a round would have to stream if it formed the whole Gram; the window avoids most of it
+    if p.layout == wl.DENSE:
+        ns_bytes = 4.0 * p.n_rows * (p.n_candidates + kept_per_round) + 8.0 * p.n_rows
+    else:
+        ns_bytes = 8.0 * (p.nnz / p.n_cols) * (p.n_candidates + kept_per_round) + 8.0 * p.n_rows
+    round_gbs = ns_bytes / (ms_local / args.steps * 1e-3) / 1e9
 
     # ---- end to end: state in pinned host memory, copied in and out every step ---------------------
     e2e_steps = min(args.e2e_steps, args.steps)
@@ -319,6 +342,12 @@ def main():
             "roofline": roofline,
             "update_hbm": {"achieved": upd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": upd_gbs / peaks["hbm_gbs"], "bytes_per_round": upd_bytes},
+            "pack_hbm": None if pack_gbs is None else {"achieved": pack_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                                      "frac": pack_gbs / peaks["hbm_gbs"], "bytes_per_round": pack_bytes},
+            "round_hbm": {"achieved": round_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                          "frac": round_gbs / peaks["hbm_gbs"], "bytes_per_round": ns_bytes,
+                          "note": "bytes by the metric's count 4N(P'+P)+8N (CSC: 8 nnz_col (P'+P)+8N) / round time; the "
+                                  "candidate window reads only a fraction of them"},
             "cpu_baseline": cpu_baseline,
             "e2e": {"value": e2e_kept_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},

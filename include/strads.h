@@ -174,14 +174,17 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out);
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);
 
 /* Optional step timing with CUDA events on the handle's stream.  After strads_profile_begin the next
- * max_rounds rounds (strads_round / strads_run / strads_round_host) record an event at every step
- * boundary; strads_profile_end waits for the stream and returns the summed device time in
- * milliseconds of ms[0] sampling, ms[1] Gram (of the candidate window, or of all candidates when no window is
- * used), ms[2] greedy walk (plus the whole-list retry when the window was too short), ms[3] update over
- * *rounds rounds.
+ * max_rounds rounds (strads_round / strads_run / strads_round_host; strads_run then launches kernel by kernel
+ * instead of replaying its graph) record an event at every step boundary; strads_profile_end waits for the
+ * stream and returns the summed device time in milliseconds over *rounds rounds of
+ *   ms[0] candidate sampling,
+ *   ms[1] packing the candidate columns (dense tensor-core path; 0 otherwise),
+ *   ms[2] the Gram kernels (of the candidate window, or of all candidates when no window is used),
+ *   ms[3] the greedy walk, plus the whole-list retry when the window was too short,
+ *   ms[4] the update.
  * Events are host-side driver objects; no device memory is allocated. */
 int strads_profile_begin(strads_handle_t h, int64_t max_rounds);
-int strads_profile_end(strads_handle_t h, double* ms_host_out /* [4] */, int64_t* rounds_host_out);
+int strads_profile_end(strads_handle_t h, double* ms_host_out /* [5] */, int64_t* rounds_host_out);
 
 int strads_destroy(strads_handle_t h);
 

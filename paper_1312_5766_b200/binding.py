@@ -264,10 +264,11 @@ class StradsLasso:
         _check(load().strads_profile_begin(self._h, int(max_rounds)), "strads_profile_begin")
 
     def profile_end(self) -> dict:
-        ms = (C.c_double * 4)()
+        ms = (C.c_double * 5)()
         n = C.c_int64(0)
         _check(load().strads_profile_end(self._h, ms, C.byref(n)), "strads_profile_end")
-        return {"rounds": int(n.value), "sample_ms": ms[0], "gram_ms": ms[1], "filter_ms": ms[2], "update_ms": ms[3]}
+        return {"rounds": int(n.value), "sample_ms": ms[0], "pack_ms": ms[1], "gram_ms": ms[2], "walk_ms": ms[3],
+                "update_ms": ms[4]}
 
     def close(self) -> None:
         if self._h:

@@ -28,6 +28,8 @@ struct strads_lasso_s {
 
 namespace {
 
+constexpr int kProfEvents = 6;   // per round: start, after sample, pack, Gram, walk, update
+
 thread_local char g_cuda_err[256] = "";
 
 int cuda_fail(cudaError_t e, const char* where) {
@@ -107,12 +109,17 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
 cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
-                        bool window = false) {
+                        bool window = false, cudaEvent_t after_pack = nullptr) {
   const Problem& p = h->p;
   cudaStream_t s = h->stream;
+  if (after_pack != nullptr && (p.layout == STRADS_CSC || gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM))) {
+    const cudaError_t e = cudaEventRecord(after_pack, s);          // these paths have no pack kernel
+    if (e != cudaSuccess) return e;
+    after_pack = nullptr;
+  }
   if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, window, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, s);
+  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, after_pack, s);
 }
 
 // The greedy walk stops at P kept, so it normally looks at little more than the first P candidates: form the
@@ -125,15 +132,17 @@ int window_of(const Problem& p, int n_cand) {
   return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
 }
 
-int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, cudaEvent_t after_gram = nullptr) {
+int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, cudaEvent_t after_pack = nullptr,
+                    cudaEvent_t after_gram = nullptr) {
   const Problem& p = h->p;
   if (p.flags & STRADS_FLAG_NO_FILTER) {
+    if (after_pack) CK(cudaEventRecord(after_pack, h->stream));
     if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
     CK(launch_filter(p, cand, n_cand, n_cand, false, p.kept, h->stream));
     return STRADS_OK;
   }
   const int window = gram_dbg != nullptr ? n_cand : window_of(p, n_cand);
-  CK(launch_gram(h, cand, window, gram_dbg, false, window < n_cand));
+  CK(launch_gram(h, cand, window, gram_dbg, false, window < n_cand, after_pack));
   if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
   CK(launch_filter(p, cand, window, n_cand, false, p.kept, h->stream));
   if (window < n_cand) {
@@ -150,20 +159,20 @@ int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_
 
 int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
   const Problem& p = h->p;
-  cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + 5 * h->prof_rounds : nullptr;
+  cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + kProfEvents * h->prof_rounds : nullptr;
   if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
   if (ev) CK(cudaEventRecord(ev[1], h->stream));
   {
-    const int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr);
+    const int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr);
     if (rc) return rc;
   }
-  if (ev) CK(cudaEventRecord(ev[3], h->stream));
+  if (ev) CK(cudaEventRecord(ev[4], h->stream));
   // after a tensor-core Gram the kept columns are read from the packed candidate buffer
   const bool packed = p.layout == STRADS_DENSE_COLMAJOR && !(p.flags & (STRADS_FLAG_NO_FILTER | STRADS_FLAG_SIMT_GRAM)) &&
                       !(out && out->gram);
   CK(launch_update(p, p.kept, 1, packed, h->stream));
-  if (ev) { CK(cudaEventRecord(ev[4], h->stream)); h->prof_rounds += 1; }
+  if (ev) { CK(cudaEventRecord(ev[5], h->stream)); h->prof_rounds += 1; }
   h->round_host += 1;
   if (out != nullptr) {
     if (out->cand) CK(cudaMemcpyAsync(out->cand, p.cand, sizeof(int) * p.n_cand, cudaMemcpyDeviceToDevice, h->stream));
@@ -407,9 +416,9 @@ int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out) {
 int strads_profile_begin(strads_handle_t h, int64_t max_rounds) {
   if (h == nullptr || max_rounds < 1 || max_rounds > (1 << 20)) return STRADS_ERR_INVALID_ARG;
   if (h->prof_events != nullptr) return STRADS_ERR_INVALID_ARG;
-  h->prof_events = new (std::nothrow) cudaEvent_t[5 * max_rounds];
+  h->prof_events = new (std::nothrow) cudaEvent_t[kProfEvents * max_rounds];
   if (h->prof_events == nullptr) return STRADS_ERR_INVALID_ARG;
-  for (long long i = 0; i < 5 * max_rounds; ++i) {
+  for (long long i = 0; i < kProfEvents * max_rounds; ++i) {
     cudaError_t e = cudaEventCreate(&h->prof_events[i]);
     if (e != cudaSuccess) {
       for (long long k = 0; k < i; ++k) cudaEventDestroy(h->prof_events[k]);
@@ -428,17 +437,17 @@ int strads_profile_end(strads_handle_t h, double* ms_host_out, int64_t* rounds_h
   int rc = STRADS_OK;
   cudaError_t e = cudaStreamSynchronize(h->stream);
   if (e != cudaSuccess) rc = cuda_fail(e, "cudaStreamSynchronize");
-  double ms[4] = {0, 0, 0, 0};
+  double ms[kProfEvents - 1] = {0, 0, 0, 0, 0};
   for (long long r = 0; r < h->prof_rounds && rc == STRADS_OK; ++r)
-    for (int k = 0; k < 4; ++k) {
+    for (int k = 0; k < kProfEvents - 1; ++k) {
       float v = 0.f;
-      e = cudaEventElapsedTime(&v, h->prof_events[5 * r + k], h->prof_events[5 * r + k + 1]);
+      e = cudaEventElapsedTime(&v, h->prof_events[kProfEvents * r + k], h->prof_events[kProfEvents * r + k + 1]);
       if (e != cudaSuccess) { rc = cuda_fail(e, "cudaEventElapsedTime"); break; }
       ms[k] += v;
     }
-  if (ms_host_out) for (int k = 0; k < 4; ++k) ms_host_out[k] = ms[k];
+  if (ms_host_out) for (int k = 0; k < kProfEvents - 1; ++k) ms_host_out[k] = ms[k];
   if (rounds_host_out) *rounds_host_out = h->prof_rounds;
-  for (long long i = 0; i < 5 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
+  for (long long i = 0; i < kProfEvents * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
   delete[] h->prof_events;
   h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
   return rc;
@@ -448,7 +457,7 @@ int strads_destroy(strads_handle_t h) {
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
   cudaStreamSynchronize(h->stream);
   if (h->prof_events != nullptr) {
-    for (long long i = 0; i < 5 * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
+    for (long long i = 0; i < kProfEvents * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
     delete[] h->prof_events;
   }
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);

@@ -503,7 +503,7 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
 // pack -> screen [-> split-K reduce] -> exact recheck of the borderline pairs -> (only if their list overflowed)
 // 3xTF32 over everything
 cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
-                                 cudaStream_t s) {
+                                 cudaEvent_t after_pack, cudaStream_t s) {
   const int n_tiles = (n_cand + kTile - 1) / kTile;
   const int tiles = n_tiles * (n_tiles + 1) / 2;
   const int ois = only_if_short ? 1 : 0;
@@ -520,6 +520,10 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   q.cand_cur = cand;
   const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
   k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand, ois);
+  if (after_pack != nullptr) {                         // optional step timing
+    const cudaError_t e = cudaEventRecord(after_pack, s);
+    if (e != cudaSuccess) return e;
+  }
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
     k_gram_dense_tc<false><<<tiles * n_split, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, n_split, ois);
     if (n_split > 1) k_gram_reduce<<<tiles * 16, 256, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
