@@ -119,7 +119,7 @@ cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, fl
   }
   if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, window, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, after_pack, s);
+  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, window, after_pack, s);
 }
 
 // The greedy walk stops at P kept, so it normally looks at little more than the first P candidates: form the

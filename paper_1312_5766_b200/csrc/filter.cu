@@ -22,6 +22,12 @@ constexpr int kBatch = 32;
 __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
                                                       int only_if_short, int* __restrict__ kept_out) {
   if (only_if_short && !p.st->window_short) return;
+  if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
+    // dense window whose TF32 screen left more borderline pairs than the list holds: its bits are incomplete;
+    // the whole-list retry (which has the 3xTF32 fallback) takes over
+    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; }
+    return;
+  }
   if (p.layout == STRADS_CSC && n_cand < n_total && p.st->prefer_walk && (p.st->round & 63ull) != 0) {
     if (threadIdx.x == 0) p.st->window_short = 1;    // window attempt skipped: go straight to the whole-list walk
     return;

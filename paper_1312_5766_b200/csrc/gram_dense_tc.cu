@@ -502,8 +502,10 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
 
 // pack -> screen [-> split-K reduce] -> exact recheck of the borderline pairs -> (only if their list overflowed)
 // 3xTF32 over everything
+// `fallback_elsewhere`: the launch covers a window and a whole-list retry follows; an overflow of the borderline
+// list is then handled by that retry (the window's walk raises window_short), not by a 3xTF32 launch here.
 cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
-                                 cudaEvent_t after_pack, cudaStream_t s) {
+                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s) {
   const int n_tiles = (n_cand + kTile - 1) / kTile;
   const int tiles = n_tiles * (n_tiles + 1) / 2;
   const int ois = only_if_short ? 1 : 0;
@@ -529,7 +531,8 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
     if (n_split > 1) k_gram_reduce<<<tiles * 16, 256, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
     k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q, ois);
   }
-  k_gram_dense_tc<true><<<tiles, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, 1, ois);
+  if (!fallback_elsewhere || (p.flags & STRADS_FLAG_GRAM_3XTF32))
+    k_gram_dense_tc<true><<<tiles, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, 1, ois);
   return cudaGetLastError();
 }
 

@@ -199,7 +199,7 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
 // `only_if_short`: the launch is the whole-list retry of a windowed round and does nothing unless the
 // window's filter set DeviceState::window_short.
 cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
-                                 cudaEvent_t after_pack, cudaStream_t s);
+                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s);
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
                             bool window, cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);

@@ -397,18 +397,20 @@ def test_tensor_core_gram_decisions(cfg):
     assert tc.status() == (0, 0) and tc3.status() == (0, 0)
 
 
-def test_tensor_core_screen_overflow_falls_back_to_3xtf32():
+@pytest.mark.parametrize("J,n_keep", [(1536, 64), (4096, 800)])
+def test_tensor_core_screen_overflow_falls_back_to_3xtf32(J, n_keep):
     # every pair correlates at ~rho: x_j = sqrt(rho) z + sqrt(1 - rho) e_j, so hundreds of thousands of pairs
-    # fall inside the screen's "too close to call" band and its list overflows
+    # fall inside the screen's "too close to call" band and its list overflows -- in the whole-list Gram of the
+    # retry (first case) or already in the candidate window, which then hands over to the retry (second case)
     b = _binding()
-    N, J, rho = 12_000, 1536, 0.25
+    N, rho = 12_000, 0.25
     g = torch.Generator().manual_seed(3)
     z = torch.randn(N, generator=g)
     x = (rho ** 0.5) * z[None, :] + ((1 - rho) ** 0.5) * torch.randn((J, N), generator=g)
     x -= x.mean(dim=1, keepdim=True)
     x /= x.norm(dim=1, keepdim=True)
     y = torch.randn(N, generator=g)
-    mk = lambda flags: b.StradsLasso(wl.DENSE, N, J, x.cuda(), y.cuda(), 0.1, 1e-6, rho, J, 64, seed=0, flags=flags)
+    mk = lambda flags: b.StradsLasso(wl.DENSE, N, J, x.cuda(), y.cuda(), 0.1, 1e-6, rho, J, n_keep, seed=0, flags=flags)
     tc, simt = mk(0), mk(b.FLAG_SIMT_GRAM)
     cand = torch.randperm(J, generator=g).to(torch.int32).cuda()
     kept_tc, counts_tc = tc.filter(cand)
@@ -416,7 +418,7 @@ def test_tensor_core_screen_overflow_falls_back_to_3xtf32():
     X = oracle.Matrix.dense(x.numpy())
     n2 = oracle.colnorm2(X)
     c = counts_tc.cpu().numpy(); nk = int(c[2])
-    _assert_kept_matches(X, n2, cand.cpu().numpy(), 64, float(np.float32(rho)), kept_tc.cpu().numpy()[:nk], int(c[1]))
+    _assert_kept_matches(X, n2, cand.cpu().numpy(), n_keep, float(np.float32(rho)), kept_tc.cpu().numpy()[:nk], int(c[1]))
     # the two FP32-accurate kernels may differ only on pairs within 1e-6 of rho; on this data they agree
     assert torch.equal(kept_tc, kept_s) and torch.equal(counts_tc, counts_s)
     assert tc.status() == (0, 8)                     # informational bit: the fallback did run
