@@ -3,10 +3,10 @@
 //
 // The walk is a serial chain (whether candidate i is kept depends on every earlier decision), and each
 // keep needs the conflict row of the kept candidate: a dependent memory access.  To take that latency
-// off the chain, one CTA works in batches of 32: the next 32 still-unblocked candidates (the only ones
+// off the chain, one CTA works in batches of 64: the next 64 still-unblocked candidates (the only ones
 // that can be kept next) are found with a warp scan, their conflict rows are fetched together into
-// shared memory, each lane extracts its candidate's conflicts with the other 31 into one 32-bit word,
-// and the greedy decision inside the batch is then 32 steps of register arithmetic.  The rows of the
+// shared memory, a thread per candidate extracts its conflicts with the other 63 into one 64-bit word,
+// and the greedy decision inside the batch is then 64 steps of register arithmetic.  The rows of the
 // newly kept candidates are OR-ed into the running `blocked` mask by the whole CTA.
 #include "strads_internal.cuh"
 
@@ -14,7 +14,7 @@ namespace strads {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBatch = 32;
+constexpr int kBatch = 64;          // candidates decided per batch (two per lane of the deciding warp)
 
 // n_cand < n_total: the list is only a leading window of the candidates.  If P are kept inside it the result
 // is final (the walk never looks further); otherwise window_short is raised and the caller's retry over
@@ -40,7 +40,8 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   __shared__ int pos[kBatch];                    // positions (in the candidate list) of the batch
   __shared__ int cval[kBatch];                   // cand[pos[.]]
   __shared__ int s_m, s_cursor, s_kept, s_examined, s_done;
-  __shared__ unsigned int s_keepmask;
+  __shared__ unsigned long long s_keepmask;
+  __shared__ unsigned long long s_conf[kBatch];  // per batch member: conflicts with later members
   const int tid = threadIdx.x, lane = tid & 31;
 
   for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
@@ -96,84 +97,84 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     }
     // 2. fetch their conflict rows (and their coefficient indices) together.  Loads first, stores after:
     //    a store to `rows` between two loads would order them and cost one memory round trip per word.
-    if (tid < m) cval[tid] = cand[pos[tid]];
+    if (tid < m) cval[tid] = cand[pos[tid]];         // (kBatch <= kThreads)
     {
-      const int warp = tid >> 5;                       // warp w fetches rows w, w + 8, w + 16, w + 24
-      const unsigned int* src[4];
+      const int warp = tid >> 5;                       // warp w fetches rows w, w + 8, ..., w + 56
+      const unsigned int* src[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) src[u] = p.conflict + (long long)pos[min(warp + 8 * u, m - 1)] * W;
-      for (int w0 = lane; w0 < W; w0 += 64) {
+      for (int u = 0; u < 8; ++u) src[u] = p.conflict + (long long)pos[min(warp + 8 * u, m - 1)] * W;
+      for (int w0 = lane; w0 < W; w0 += 32) {
         unsigned int v[8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          v[u] = __ldcg(src[u] + w0);
-          v[4 + u] = w0 + 32 < W ? __ldcg(src[u] + w0 + 32) : 0u;
-        }
+        for (int u = 0; u < 8; ++u) v[u] = __ldcg(src[u] + w0);
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < 8; ++u) {
           const int r = warp + 8 * u;
-          if (r < m) {
-            rows[r * Ws + w0] = v[u];
-            if (w0 + 32 < W) rows[r * Ws + w0 + 32] = v[4 + u];
-          }
+          if (r < m) rows[r * Ws + w0] = v[u];
         }
       }
     }
     __syncthreads();
-    // 3. decide the batch in order (warp 0, registers only)
-    if (tid < 32) {
-      // lane q: bit b set <=> candidate q conflicts with the LATER batch member b (row q is valid from its own word on)
-      // (fixed trip counts, so that the 32 reads / shuffles are independent and overlap)
-      const unsigned int valid = m >= 32 ? 0xffffffffu : ((1u << m) - 1u);
-      const int my_row = min(lane, m - 1) * Ws;
-      unsigned int mine = 0u;
-#pragma unroll
+    // 3a. thread q < 64: the conflicts of batch member q with the LATER members, as a 64-bit word
+    //     (a row is valid from its own word on; fixed trip count so that the reads overlap)
+    if (tid < kBatch) {
+      const int my_row = min(tid, m - 1) * Ws;
+      unsigned long long mine = 0ull;
+#pragma unroll 16
       for (int b = 0; b < kBatch; ++b) {
         const int pb = pos[min(b, m - 1)];
-        mine |= ((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << b;
+        mine |= (unsigned long long)((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << b;
       }
-      mine &= valid & ~((2u << lane) - 1u);            // later members only (lane 31: none)
-      if (lane >= m) mine = 0u;
-      unsigned int cq[kBatch];
-#pragma unroll
-      for (int q = 0; q < kBatch; ++q) cq[q] = __shfl_sync(0xffffffffu, mine, q);
-      unsigned int alive = valid;
-      unsigned int keep = 0u;
-#pragma unroll
-      for (int q = 0; q < kBatch; ++q)
-        if ((alive >> q) & 1u) { keep |= 1u << q; alive &= ~cq[q]; }
+      const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
+      const unsigned long long later = tid >= 63 ? 0ull : ~((2ull << tid) - 1ull);
+      s_conf[tid] = tid < m ? (mine & valid & later) : 0ull;
+    }
+    __syncthreads();
+    // 3b. the greedy decision inside the batch: 64 steps of register arithmetic (warp 0; every lane computes the same)
+    if (tid < 32) {
+      const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
+      unsigned long long alive = valid, keep = 0ull;
+#pragma unroll 16
+      for (int q = 0; q < kBatch; ++q) {
+        const unsigned long long cq = s_conf[q];
+        if ((alive >> q) & 1ull) { keep |= 1ull << q; alive &= ~cq; }
+      }
       const int nk = s_kept;
       const int room = p.n_keep - nk;
       bool full = false;
-      if (__popc(keep) >= room) {                      // stop exactly at P: drop the surplus from the back
-        while (__popc(keep) > room) keep &= ~(1u << (31 - __clz(keep)));
+      if (__popcll(keep) >= room) {                    // stop exactly at P: drop the surplus from the back
+        while (__popcll(keep) > room) keep &= ~(1ull << (63 - __clzll(keep)));
         full = true;
       }
-      if ((keep >> lane) & 1u) {
-        const int slot = nk + __popc(keep & ((1u << lane) - 1u));
-        kept_out[slot] = cval[lane];
-        p.kept_pos[slot] = pos[lane];
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {
+        const int q = lane + 32 * half;
+        if ((keep >> q) & 1ull) {
+          const int slot = nk + __popcll(keep & ((1ull << q) - 1ull));
+          kept_out[slot] = cval[q];
+          p.kept_pos[slot] = pos[q];
+        }
       }
       if (lane == 0) {
         s_keepmask = keep;
-        s_kept = nk + __popc(keep);
-        if (full) { s_examined = pos[31 - __clz(keep)] + 1; s_done = 1; }
+        s_kept = nk + __popcll(keep);
+        if (full) { s_examined = pos[63 - __clzll(keep)] + 1; s_done = 1; }
         else s_cursor = pos[m - 1] + 1;
       }
     }
     __syncthreads();
     if (s_done) break;
     // 4. OR the rows of the newly kept candidates into the mask (a row is valid from its own word on)
-    //    Four threads share a word, each takes 8 of the 32 batch members; reads are unconditional so that they overlap.
-    const unsigned int keep = s_keepmask;
+    //    Four threads share a word, each takes 16 of the 64 batch members; reads are unconditional so that they overlap.
+    const unsigned long long keep = s_keepmask;
     for (int u = tid; u < 4 * W; u += kThreads) {
-      const int w = u >> 2, q0 = (u & 3) * 8;
+      const int w = u >> 2, q0 = (u & 3) * 16;
       unsigned int acc = 0u;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
+      for (int i = 0; i < 16; ++i) {
         const int q = q0 + i;
         const unsigned int v = rows[min(q, m - 1) * Ws + w];
-        const bool use = ((keep >> q) & 1u) && w >= (pos[min(q, m - 1)] >> 5);
+        const bool use = ((keep >> q) & 1ull) && w >= (pos[min(q, m - 1)] >> 5);
         acc |= use ? v : 0u;
       }
       if (acc) atomicOr(&blocked[w], acc);
