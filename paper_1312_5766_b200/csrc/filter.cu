@@ -16,6 +16,17 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kBatch = 64;          // candidates decided per batch (two per lane of the deciding warp)
 
+// Position of the n-th (0-based) set bit of x; popc(x) > n.
+__device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
+  int at = 0;
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    const int c = __popc(x & ((1u << s) - 1u));
+    if (n >= c) { n -= c; x >>= s; at += s; }
+  }
+  return at;
+}
+
 // n_cand < n_total: the list is only a leading window of the candidates.  If P are kept inside it the result
 // is final (the walk never looks further); otherwise window_short is raised and the caller's retry over
 // the whole list (launched with only_if_short) replaces the result.
@@ -40,9 +51,11 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   __shared__ int pos[kBatch];                    // positions (in the candidate list) of the batch
   __shared__ int cval[kBatch];                   // cand[pos[.]]
   __shared__ int s_m, s_cursor, s_kept, s_examined, s_done;
-  __shared__ unsigned long long s_keepmask;
   __shared__ unsigned long long s_conf[kBatch];  // per batch member: conflicts with later members
+  __shared__ int s_krow[kBatch], s_kfirst[kBatch], s_nnew;   // newly kept: row offset in `rows`, first valid word
   const int tid = threadIdx.x, lane = tid & 31;
+  int G = 1;                                     // threads per mask word in step 4 (a power of two, G * W <= kThreads)
+  while (G < 32 && 2 * G * W <= kThreads) G <<= 1;
 
   for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
   if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = 0; s_done = 0; }
@@ -77,12 +90,22 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
           if (lane >= o) incl += v;
         }
         const int total = __shfl_sync(0xffffffffu, incl, 31);
-        int slot = m + incl - cnt;                     // where this lane's first free position goes
-        unsigned int fw = freew;
-        while (fw && slot < kBatch) {
-          const int b = __ffs(fw) - 1;
-          fw &= fw - 1;
-          pos[slot++] = (wbase << 5) + b;
+        // slot s of the batch takes the (s - m)-th free position of these 32 words: lane s (and s + 32) finds
+        // the word that holds it from the prefix counts, then the bit inside the word
+        const int excl = incl - cnt;
+#pragma unroll
+        for (int half = 0; half < kBatch / 32; ++half) {
+          const int slot = lane + 32 * half;
+          const int want = slot - m;                   // rank among the free positions found in this sweep
+          int wi = 0;                                  // first lane whose inclusive count exceeds `want`
+#pragma unroll
+          for (int step = 16; step > 0; step >>= 1)
+            if (__shfl_sync(0xffffffffu, incl, wi + step - 1) <= want) wi += step;
+          wi = min(wi, 31);
+          const int ex = __shfl_sync(0xffffffffu, excl, wi);
+          const unsigned int word = __shfl_sync(0xffffffffu, freew, wi);
+          if (want >= 0 && want < total && slot < kBatch)
+            pos[slot] = (((cur >> 5) + wi) << 5) + nth_set_bit(word, want - ex);
         }
         m = min(kBatch, m + total);
         if (m < kBatch) cur = ((cur >> 5) + 32) << 5;  // all 32 words consumed
@@ -115,30 +138,36 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
       }
     }
     __syncthreads();
-    // 3a. thread q < 64: the conflicts of batch member q with the LATER members, as a 64-bit word
-    //     (a row is valid from its own word on; fixed trip count so that the reads overlap)
-    if (tid < kBatch) {
-      const int my_row = min(tid, m - 1) * Ws;
-      unsigned long long mine = 0ull;
-#pragma unroll 16
-      for (int b = 0; b < kBatch; ++b) {
-        const int pb = pos[min(b, m - 1)];
-        mine |= (unsigned long long)((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << b;
+    // 3a. the conflicts of batch member q with the LATER members, as a 64-bit word: four threads per member,
+    //     16 of the 64 bits each (a row is valid from its own word on; fixed trip count so that the reads overlap)
+    {
+      static_assert(kThreads == 4 * kBatch, "four threads per batch member");
+      const int q = tid >> 2, part = tid & 3;
+      const int my_row = min(q, m - 1) * Ws;
+      unsigned int bits = 0u;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const int pb = pos[min(part * 16 + i, m - 1)];
+        bits |= ((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << i;
       }
+      unsigned long long mine = (unsigned long long)bits << (16 * part);
+      mine |= __shfl_xor_sync(0xffffffffu, mine, 1);
+      mine |= __shfl_xor_sync(0xffffffffu, mine, 2);
       const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
-      const unsigned long long later = tid >= 63 ? 0ull : ~((2ull << tid) - 1ull);
-      s_conf[tid] = tid < m ? (mine & valid & later) : 0ull;
+      const unsigned long long later = q >= 63 ? 0ull : ~((2ull << q) - 1ull);
+      if (part == 0) s_conf[q] = q < m ? (mine & valid & later) : 0ull;
     }
     __syncthreads();
     // 3b. the greedy decision inside the batch: 64 steps of register arithmetic (warp 0; every lane computes the same)
     if (tid < 32) {
       const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
       unsigned long long alive = valid, keep = 0ull;
-#pragma unroll 16
-      for (int q = 0; q < kBatch; ++q) {
-        const unsigned long long cq = s_conf[q];
-        if ((alive >> q) & 1ull) { keep |= 1ull << q; alive &= ~cq; }
-      }
+      unsigned long long cq[kBatch];                   // all 64 words into registers first: the loads do not depend
+#pragma unroll                                         // on the chain below and overlap
+      for (int q = 0; q < kBatch; ++q) cq[q] = s_conf[q];
+#pragma unroll
+      for (int q = 0; q < kBatch; ++q)
+        if ((alive >> q) & 1ull) { keep |= 1ull << q; alive &= ~cq[q]; }
       const int nk = s_kept;
       const int room = p.n_keep - nk;
       bool full = false;
@@ -155,8 +184,17 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
           p.kept_pos[slot] = pos[q];
         }
       }
+#pragma unroll
+      for (int half = 0; half < 2; ++half) {           // compact list of the newly kept rows for step 4
+        const int q = lane + 32 * half;
+        if ((keep >> q) & 1ull) {
+          const int r = __popcll(keep & ((1ull << q) - 1ull));
+          s_krow[r] = q * Ws;
+          s_kfirst[r] = pos[q] >> 5;
+        }
+      }
       if (lane == 0) {
-        s_keepmask = keep;
+        s_nnew = __popcll(keep);
         s_kept = nk + __popcll(keep);
         if (full) { s_examined = pos[63 - __clzll(keep)] + 1; s_done = 1; }
         else s_cursor = pos[m - 1] + 1;
@@ -164,20 +202,29 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     }
     __syncthreads();
     if (s_done) break;
-    // 4. OR the rows of the newly kept candidates into the mask (a row is valid from its own word on)
-    //    Four threads share a word, each takes 16 of the 64 batch members; reads are unconditional so that they overlap.
-    const unsigned long long keep = s_keepmask;
-    for (int u = tid; u < 4 * W; u += kThreads) {
-      const int w = u >> 2, q0 = (u & 3) * 16;
+    // 4. OR the rows of the newly kept candidates into the mask (a row is valid from its own word on).
+    //    G threads per mask word share the rows between them (all loads unconditional and independent),
+    //    then combine with shuffles.
+    const int n_new = s_nnew;
+    for (int base = 0; base < W; base += kThreads / G) {
+      const int w = base + tid / G, sub = tid % G;
       unsigned int acc = 0u;
+      if (w < W) {
+        for (int r0 = sub; r0 < n_new; r0 += 8 * G) {
+          int kf[8];
+          unsigned int v[8];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int q = q0 + i;
-        const unsigned int v = rows[min(q, m - 1) * Ws + w];
-        const bool use = ((keep >> q) & 1ull) && w >= (pos[min(q, m - 1)] >> 5);
-        acc |= use ? v : 0u;
+          for (int i = 0; i < 8; ++i) {
+            const int r = min(r0 + i * G, n_new - 1);  // past the end: the last row again (harmless)
+            kf[i] = s_kfirst[r];
+            v[i] = rows[s_krow[r] + w];
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) acc |= w >= kf[i] ? v[i] : 0u;
+        }
       }
-      if (acc) atomicOr(&blocked[w], acc);
+      for (int o = G >> 1; o > 0; o >>= 1) acc |= __shfl_xor_sync(0xffffffffu, acc, o);
+      if (w < W && sub == 0) blocked[w] |= acc;
     }
     __syncthreads();
   }
