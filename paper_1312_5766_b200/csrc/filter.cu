@@ -32,6 +32,7 @@ __device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
 // the whole list (launched with only_if_short) replaces the result.
 __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
                                                       int only_if_short, int* __restrict__ kept_out) {
+  chain_begin();
   if (only_if_short && !p.st->window_short) return;
   if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
     // dense window whose TF32 screen left more borderline pairs than the list holds: its bits are incomplete;
@@ -253,8 +254,7 @@ cudaError_t prepare_filter(const Problem&) {
 
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s) {
-  k_filter<<<1, kThreads, filter_smem_bytes(p), s>>>(p, cand, n_cand, n_total, only_if_short ? 1 : 0, kept_out);
-  return cudaGetLastError();
+  return launch_chained(k_filter, 1, kThreads, filter_smem_bytes(p), s, p, cand, n_cand, n_total, only_if_short ? 1 : 0, kept_out);
 }
 
 }  // namespace strads

@@ -13,6 +13,7 @@ constexpr int kStage = 1024;          // entries of column a staged in shared me
 
 __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __restrict__ cand, int n_cand,
                                                         float* __restrict__ gram_dbg, int only_if_short, int window) {
+  chain_begin();
   if (only_if_short && !p.st->window_short) return;
   if (window && p.st->prefer_walk && (p.st->round & 63ull) != 0) return;   // the window attempt is being skipped
   __shared__ int arow[kStage];
@@ -56,8 +57,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
 
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
                             bool window, cudaStream_t s) {
-  k_gram_csc<<<n_cand, kThreads, 0, s>>>(p, cand, n_cand, gram_dbg, only_if_short ? 1 : 0, window ? 1 : 0);
-  return cudaGetLastError();
+  return launch_chained(k_gram_csc, n_cand, kThreads, 0, s, p, cand, n_cand, gram_dbg, only_if_short ? 1 : 0, window ? 1 : 0);
 }
 
 }  // namespace strads

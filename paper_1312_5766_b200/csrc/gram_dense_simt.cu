@@ -30,6 +30,7 @@ __device__ __forceinline__ float4 load_k4(const float* col, long long k, long lo
 
 __global__ void __launch_bounds__(kThreads) k_gram_dense_simt(Problem p, const int* __restrict__ cand, int n_cand,
                                                                int n_tiles, float* __restrict__ gram_dbg) {
+  chain_begin();
   __shared__ __align__(16) float As[2][BK][BM];
   __shared__ __align__(16) float Bs[2][BK][BM];
   __shared__ double n2a[BM], n2b[BM];
@@ -136,8 +137,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_dense_simt(Problem p, const i
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s) {
   const int n_tiles = (n_cand + BM - 1) / BM;
   const int blocks = n_tiles * (n_tiles + 1) / 2;
-  k_gram_dense_simt<<<blocks, kThreads, 0, s>>>(p, cand, n_cand, n_tiles, gram_dbg);
-  return cudaGetLastError();
+  return launch_chained(k_gram_dense_simt, blocks, kThreads, 0, s, p, cand, n_cand, n_tiles, gram_dbg);
 }
 
 }  // namespace strads

@@ -149,6 +149,7 @@ __device__ __forceinline__ uint32_t decide_word(const Problem& p, const uint32_t
 // One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).
 __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
                                                          int only_if_short) {
+  chain_begin();
   const int a = blockIdx.x;
   if (a >= n_cand || (only_if_short && !p.st->window_short)) return;
   const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)cand[a] * p.ld);
@@ -160,6 +161,7 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
 template <bool k3x>
 __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const __grid_constant__ CUtensorMap tmap,
                                                                 int n_cand, int n_tiles, int n_split, int only_if_short) {
+  chain_begin();
   // A stage holds kSub sub-blocks of 32 floats of K for A, the same for B [3xTF32: plus the two lo tiles].
   constexpr int kSub = k3x ? 1 : 2;
   constexpr int kStageBytes = (k3x ? 4 : 2 * kSub) * kTileBytes;       // 64 KB either way
@@ -386,6 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 // Split-K: sums the partial tiles of one output tile in split order and thresholds (screen rules).
 // One CTA per (tile, 8 rows); a warp owns one row, a lane four of its 128 columns.
 __global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short) {
+  chain_begin();
   if (only_if_short && !p.st->window_short) return;
   const int tile = blockIdx.x >> 4, rgroup = blockIdx.x & 15;
   int ti = 0, rem = tile;
@@ -438,6 +441,7 @@ __global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int 
 // Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product of the
 // packed columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
 __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_short) {
+  chain_begin();
   if (only_if_short && !p.st->window_short) return;
   const unsigned int n = p.st->amb_count;
   if (n > (unsigned)p.cap_amb) return;                 // overflow: the 3xTF32 kernel redoes every bit instead
@@ -521,19 +525,20 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   Problem q = p;
   q.cand_cur = cand;
   const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
-  k_pack_candidates<<<n_cand, 256, 0, s>>>(q, cand, n_cand, ois);
-  if (after_pack != nullptr) {                         // optional step timing
-    const cudaError_t e = cudaEventRecord(after_pack, s);
-    if (e != cudaSuccess) return e;
-  }
+  cudaError_t e;
+  if ((e = launch_chained(k_pack_candidates, n_cand, 256, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
+  if (after_pack != nullptr && (e = cudaEventRecord(after_pack, s)) != cudaSuccess) return e;   // optional step timing
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
-    k_gram_dense_tc<false><<<tiles * n_split, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, n_split, ois);
-    if (n_split > 1) k_gram_reduce<<<tiles * 16, 256, 0, s>>>(q, n_cand, n_tiles, n_split, ois);
-    k_gram_recheck<<<p.sm_count * 2, 256, 0, s>>>(q, ois);
+    if ((e = launch_chained(k_gram_dense_tc<false>, tiles * n_split, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, n_split,
+                            ois)) != cudaSuccess)
+      return e;
+    if (n_split > 1 && (e = launch_chained(k_gram_reduce, tiles * 16, 256, 0, s, q, n_cand, n_tiles, n_split, ois)) != cudaSuccess)
+      return e;
+    if ((e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
   }
   if (!fallback_elsewhere || (p.flags & STRADS_FLAG_GRAM_3XTF32))
-    k_gram_dense_tc<true><<<tiles, kThreads, kDynSmem, s>>>(q, tm, n_cand, n_tiles, 1, ois);
-  return cudaGetLastError();
+    return launch_chained(k_gram_dense_tc<true>, tiles, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, 1, ois);
+  return cudaSuccess;
 }
 
 }  // namespace strads

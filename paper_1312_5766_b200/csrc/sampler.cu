@@ -80,6 +80,7 @@ __device__ void find_bin(const unsigned int* h, int nbins, long long k_rem, int*
 }
 
 __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
+  chain_begin();
   __shared__ unsigned int sh[kHistBins];
   __shared__ int s_last;
   __shared__ SelectState s_sel;
@@ -154,6 +155,7 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
 }
 
 __global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
+  chain_begin();
   const SelectState sel = p.st->sel;
   const unsigned long long t = p.st->round;
   const long long groups = (p.J + 3) >> 2;
@@ -211,6 +213,7 @@ __device__ __forceinline__ ChunkRef chunk_of(const Problem& p, const SelectState
 // (bitonic) and writes it back in place.  One CTA sorting all P' keys would be bound by its own shared-memory
 // bandwidth (~100 us for 16,384 keys); chunks run on as many SMs as there are chunks.
 __global__ void __launch_bounds__(512) k_sample_sort_chunks(Problem p) {
+  chain_begin();
   __shared__ unsigned long long keys[kChunk];
   const SelectState sel = p.st->sel;
   const ChunkRef ch = chunk_of(p, sel, blockIdx.x);
@@ -236,6 +239,7 @@ __device__ __forceinline__ int count_less(const unsigned long long* a, int n, un
 // keys in every other chunk of its buffer (+ n_sure for boundary keys: every sure key is smaller).  The key
 // of rank r < P' is candidate r.  Each other chunk is staged in shared memory and searched there.
 __global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
+  chain_begin();
   __shared__ unsigned long long other[kChunk];
   const SelectState sel = p.st->sel;
   const ChunkRef ch = chunk_of(p, sel, blockIdx.x);
@@ -270,12 +274,12 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   const long long cap = (long long)p.sm_count * 8;
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
-  k_sample_hist<<<(unsigned)blocks, kThreads, 0, s>>>(p);
-  k_sample_collect<<<(unsigned)blocks, kThreads, 0, s>>>(p);
+  cudaError_t e;
+  if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
+  if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
   const int chunks = (p.cap_sure + kChunk - 1) / kChunk + (p.cap_boundary + kChunk - 1) / kChunk;
-  k_sample_sort_chunks<<<chunks, 512, 0, s>>>(p);
-  k_sample_rank<<<chunks, 512, 0, s>>>(p, cand_out);
-  return cudaGetLastError();
+  if ((e = launch_chained(k_sample_sort_chunks, chunks, 512, 0, s, p)) != cudaSuccess) return e;
+  return launch_chained(k_sample_rank, chunks, 512, 0, s, p, cand_out);
 }
 
 }  // namespace strads

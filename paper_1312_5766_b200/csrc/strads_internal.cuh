@@ -186,6 +186,31 @@ __device__ __forceinline__ float sparse_dot(const int* ar, const float* av, int 
 }
 
 // ---------------------------------------------------------------------------------------------
+// Chained launches (programmatic dependent launch).  A round is a chain of short kernels, each needing the
+// one before it, and the gap between two dependent launches is of the order of the kernels themselves.  A
+// kernel launched with launch_chained may be scheduled while the kernel ahead of it in the stream still runs;
+// chain_begin() is where it stops until that kernel has finished and its writes are visible, so it is the
+// first statement of every kernel launched this way (nothing in global memory is touched before it).  It then
+// lets the kernel behind it start in the same manner.  Since every link waits for its predecessor to finish,
+// finishing is transitive along the chain.  Launched the ordinary way, chain_begin() does nothing.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void chain_begin() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// ---------------------------------------------------------------------------------------------
 // Launchers (one per step; all enqueue on `s` and return a cudaError_t).
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_init(const Problem& p, cudaStream_t s);

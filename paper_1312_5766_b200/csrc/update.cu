@@ -57,6 +57,7 @@ struct ColumnSource {
 };
 
 __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __restrict__ kept, ColumnSource src) {
+  chain_begin();
   const int a = blockIdx.y;
   if (a >= p.st->counts[2]) {
     if (blockIdx.x == 0 && threadIdx.x == 0) p.dbeta[a] = 0.f;
@@ -114,6 +115,7 @@ constexpr int kRowsPerCta = 64;
 constexpr int kColSlots = kThreads / 16;   // half-warps per CTA
 
 __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSource src, int advance) {
+  chain_begin();
   __shared__ double part[kColSlots][kRowsPerCta];
   const int n_kept = p.st->counts[2];
   const int slot = threadIdx.x >> 4, l16 = threadIdx.x & 15;
@@ -162,6 +164,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSourc
 // CSC
 // ------------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kThreads) k_dot_csc(Problem p, const int* __restrict__ kept) {
+  chain_begin();
   const int lane = threadIdx.x & 31;
   const int a = (blockIdx.x * kThreads + threadIdx.x) >> 5;
   if (a >= p.n_keep) return;
@@ -181,6 +184,7 @@ constexpr int kMaxRowsCsc = 4096;      // rows owned by one CTA (64-bit accumula
 
 __global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, const int* __restrict__ kept, int rows_per_cta,
                                                          int advance) {
+  chain_begin();
   __shared__ long long acc[kMaxRowsCsc];
   __shared__ double wmax[kThreads / 32];
   __shared__ int s_shift;
@@ -236,10 +240,12 @@ __global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, const int* __
 }
 
 __global__ void k_set_counts(Problem p, int n_cand, int n_examined, int n_kept) {
+  chain_begin();
   p.st->counts[0] = n_cand; p.st->counts[1] = n_examined; p.st->counts[2] = n_kept; p.st->counts[3] = 0;
 }
 
 __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out) {
+  chain_begin();
   const int n_kept = p.st->counts[2];
   for (int a = blockIdx.x * blockDim.x + threadIdx.x; a < p.n_keep; a += gridDim.x * blockDim.x) {
     if (kept_out != nullptr) kept_out[a] = a < n_kept ? kept[a] : -1;
@@ -257,28 +263,27 @@ cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool f
     ColumnSource src;
     if (from_packed) { src.base = p.xc; src.pitch = p.ldc; src.index = p.kept_pos; }
     else { src.base = p.xv; src.pitch = p.ld; src.index = kept; }
-    k_dot_dense<<<dim3(p.dot_parts, p.n_keep), kThreads, 0, s>>>(p, kept, src);
-    k_apply_dense<<<(unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s>>>(p, src, advance);
+    cudaError_t e;
+    if ((e = launch_chained(k_dot_dense, dim3(p.dot_parts, p.n_keep), kThreads, 0, s, p, kept, src)) != cudaSuccess) return e;
+    return launch_chained(k_apply_dense, (unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s, p, src, advance);
   } else {
-    k_dot_csc<<<(p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s>>>(p, kept);
+    cudaError_t e;
+    if ((e = launch_chained(k_dot_csc, (p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, kept)) != cudaSuccess) return e;
     long long grid = (long long)p.sm_count * 2;
     const long long need = (p.N + kMaxRowsCsc - 1) / kMaxRowsCsc;
     if (grid < need) grid = need;
     const int rows_per_cta = (int)((p.N + grid - 1) / grid);
-    k_apply_csc<<<(unsigned)grid, kThreads, 0, s>>>(p, kept, rows_per_cta, advance);
+    return launch_chained(k_apply_csc, (unsigned)grid, kThreads, 0, s, p, kept, rows_per_cta, advance);
   }
-  return cudaGetLastError();
 }
 
 cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s) {
-  k_set_counts<<<1, 1, 0, s>>>(p, n_cand, n_examined, n_kept);
-  return cudaGetLastError();
+  return launch_chained(k_set_counts, 1, 1, 0, s, p, n_cand, n_examined, n_kept);
 }
 
 cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,
                           cudaStream_t s) {
-  k_export<<<(p.n_keep + 255) / 256, 256, 0, s>>>(p, kept, kept_out, dbeta_out, counts_out);
-  return cudaGetLastError();
+  return launch_chained(k_export, (p.n_keep + 255) / 256, 256, 0, s, p, kept, kept_out, dbeta_out, counts_out);
 }
 
 }  // namespace strads
