@@ -140,6 +140,17 @@ def sample(delta, eta, seed, t, n_cand, return_keys=False):
     return (cand, keys) if return_keys else cand
 
 
+def sample_part(delta, eta, seed, t, n_sched, sched, n_cand):
+    """Candidates of scheduler thread `sched` of `n_sched` (it owns j = sched mod n_sched), best first."""
+    delta = _f64(delta)
+    cand = np.empty(n_cand, dtype=np.int32)
+    rc = _load().so_sample_part(C.c_int64(delta.shape[0]), _p(delta), C.c_double(eta), C.c_uint64(seed), C.c_uint64(t),
+                                C.c_int32(n_sched), C.c_int32(sched), C.c_int32(n_cand), _p(cand))
+    if rc:
+        raise ValueError(f"so_sample_part failed: {rc}")
+    return cand
+
+
 def colnorm2(X: Matrix):
     n2 = np.empty(X.n_cols, dtype=np.float64)
     _load().so_colnorm2(X.ref, _p(n2))
@@ -187,8 +198,9 @@ def init(X: Matrix, y, c_init):
     return n2, beta, resid, delta
 
 
-def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, delta):
-    """One round in place. Returns dict(cand, kept, dbeta, counts)."""
+def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, delta, n_sched=1):
+    """One round in place (round t is dispatched by scheduler thread t mod n_sched).
+    Returns dict(cand, kept, dbeta, counts)."""
     for a in (beta, resid, delta):
         assert a.dtype == np.float64 and a.flags.c_contiguous
     n2 = _f64(n2)
@@ -196,9 +208,15 @@ def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, de
     kept = np.full(n_keep, -1, dtype=np.int32)
     dbeta = np.zeros(n_keep, dtype=np.float64)
     counts = np.zeros(4, dtype=np.int32)
-    rc = _load().so_round(X.ref, _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
-                          C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
-                          _p(beta), _p(resid), _p(delta), _p(cand), _p(kept), _p(dbeta), _p(counts))
+    if n_sched == 1:
+        rc = _load().so_round(X.ref, _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
+                              C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
+                              _p(beta), _p(resid), _p(delta), _p(cand), _p(kept), _p(dbeta), _p(counts))
+    else:
+        rc = _load().so_round_part(X.ref, _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
+                                   C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
+                                   C.c_int32(n_sched), _p(beta), _p(resid), _p(delta), _p(cand), _p(kept),
+                                   _p(dbeta), _p(counts))
     if rc:
         raise ValueError(f"so_round failed: {rc}")
     nk = int(counts[2])

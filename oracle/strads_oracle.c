@@ -206,6 +206,33 @@ int so_sample(int64_t J, const double *delta, double eta, uint64_t seed, uint64_
     return 0;
 }
 
+/* STRADS ("Implementation Overview"): S scheduler threads, thread s owning a fixed,
+ * disjoint set of J/S coefficients and sampling only from its own p_s(j).  The
+ * assignment used here: thread s owns { j : j mod S == s } (the paper assigns at
+ * random; the caller may permute the columns).  Ranks the race keys of the
+ * coefficients of thread `s` only and returns the first n_cand, best first.
+ * With S == 1 this is so_sample. */
+int so_sample_part(int64_t J, const double *delta, double eta, uint64_t seed, uint64_t t,
+                   int32_t S, int32_t s, int32_t n_cand, int32_t *cand)
+{
+    if (J <= 0 || S < 1 || s < 0 || s >= S || n_cand < 0) return -1;
+    const int64_t members = (J - s + S - 1) / S;      /* |{ j < J : j mod S == s }| */
+    if (n_cand > members) return -1;
+    so_keyed *own = (so_keyed *)malloc((size_t)(members > 0 ? members : 1) * sizeof(so_keyed));
+    if (!own) return -2;
+    int64_t m = 0;
+    for (int64_t j = s; j < J; j += S) {
+        const float T = so_race_key((float)delta[j], (float)eta, so_draw_word(seed, t, (uint64_t)j));
+        own[m].tbits = f32_bits(T);
+        own[m].j = (int32_t)j;
+        ++m;
+    }
+    qsort(own, (size_t)m, sizeof(so_keyed), keyed_less);
+    for (int32_t a = 0; a < n_cand; ++a) cand[a] = own[a].j;
+    free(own);
+    return 0;
+}
+
 /* ------------------------------------------------------------------------- */
 /* Dependency filter (Algorithm 1, "Choose a set B1 of <= P coefficients from  */
 /* U such that |x_j^T x_k| <= rho"; strict form of SAP step 2).  Walk the      */
@@ -326,6 +353,27 @@ int so_round(const so_matrix *X, const double *n2, double lambda, double eta, do
              int32_t *counts /* [4]: n_cand, n_examined, n_kept, n_nonzero */)
 {
     int rc = so_sample(X->n_cols, delta, eta, seed, t, n_cand, cand, NULL);
+    if (rc) return rc;
+    int32_t nk = 0, ne = 0;
+    so_filter(X, n2, cand, n_cand, n_keep, rho, NULL, 0, 0.0, kept, &nk, &ne, NULL);
+    so_update(X, n2, lambda, kept, nk, beta, resid, delta, dbeta);
+    int32_t nz = 0;
+    for (int32_t a = 0; a < nk; ++a) nz += dbeta[a] != 0.0;
+    counts[0] = n_cand; counts[1] = ne; counts[2] = nk; counts[3] = nz;
+    return 0;
+}
+
+/* One round of STRADS with S scheduler threads taking turns ("thread 1 dispatches
+ * first, then thread 2, ... before returning to thread 1"): round t is dispatched
+ * by thread t mod S, which samples from its own coefficients; the rest of the round
+ * is Algorithm 1's loop body unchanged. */
+int so_round_part(const so_matrix *X, const double *n2, double lambda, double eta, double rho,
+                  int32_t n_cand, int32_t n_keep, uint64_t seed, uint64_t t, int32_t S,
+                  double *beta, double *resid, double *delta,
+                  int32_t *cand, int32_t *kept, double *dbeta, int32_t *counts)
+{
+    if (S < 1) return -1;
+    int rc = so_sample_part(X->n_cols, delta, eta, seed, t, S, (int32_t)(t % (uint64_t)S), n_cand, cand);
     if (rc) return rc;
     int32_t nk = 0, ne = 0;
     so_filter(X, n2, cand, n_cand, n_keep, rho, NULL, 0, 0.0, kept, &nk, &ne, NULL);
