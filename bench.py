@@ -174,6 +174,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=200)
     ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
+    ap.add_argument("--schedulers", type=int, default=4,
+                    help="also time the same workload with this many round-robin scheduler threads (0: skip)")
     ap.add_argument("--n-cols", type=int, default=0,
                     help="profiling aid: same workload with fewer columns J (keeps N, P', P), so that a "
                          "multi-pass ncu capture holds less device memory")
@@ -287,6 +289,28 @@ def main():
         ns_bytes = 8.0 * (p.nnz / p.n_cols) * (p.n_candidates + kept_per_round) + 8.0 * p.n_rows
     round_gbs = ns_bytes / (ms_local / args.steps * 1e-3) / 1e9
 
+    # ---- the same workload with S round-robin scheduler threads (blocks of later rounds prepared during updates) ----
+    round_robin = None
+    if args.schedulers > 1 and p.n_candidates * args.schedulers <= p.n_cols:
+        S = args.schedulers
+        s2 = binding.StradsLasso.from_problem(p, device=device, n_schedulers=S)
+        s2.run(max(args.warmup, 2 * 16 * S))           # includes building the captured sequence
+        kept0 = s2.totals()["kept"]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        s2.run(args.steps)
+        e1.record()
+        barrier()
+        rr_ms_local = e0.elapsed_time(e1)
+        rr_kept_all, rr_ms = aggregate(s2.totals()["kept"] - kept0, rr_ms_local, dist_ok, device)
+        round_robin = {"schedulers": S, "value": rr_kept_all / (rr_ms * 1e-3), "unit": UNIT, "ms_per_step": rr_ms / args.steps,
+                       "steps": args.steps, "objective": s2.objective(), "status_bits": s2.status()[1],
+                       "note": "scheduler s owns the coefficients j mod S == s and dispatches the rounds t mod S == s; "
+                               "results are those of the same rounds run one after another"}
+        del s2
+        torch.cuda.empty_cache()
+
     # ---- end to end: state in pinned host memory, copied in and out every step ---------------------
     e2e_steps = min(args.e2e_steps, args.steps)
     beta_h = s.beta.cpu().pin_memory(); resid_h = s.resid.cpu().pin_memory(); delta_h = s.delta.cpu().pin_memory()
@@ -349,6 +373,7 @@ def main():
                           "note": "bytes by the metric's count 4N(P'+P)+8N (CSC: 8 nnz_col (P'+P)+8N) / round time; the "
                                   "candidate window reads only a fraction of them"},
             "cpu_baseline": cpu_baseline,
+            "round_robin": round_robin,
             "e2e": {"value": e2e_kept_all / (e2e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "steps": e2e_steps},
             "gpu_launches": launches_per_round * args.steps,

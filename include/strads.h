@@ -69,6 +69,7 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
 
 /* limits */
 #define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (one CTA sorts the winners in shared memory) */
+#define STRADS_MAX_SCHEDULERS 8
 
 typedef struct {
   int32_t  layout;                      /* strads_layout_t                                          */
@@ -93,6 +94,8 @@ typedef struct {
   size_t   workspace_bytes;
   void*    stream;                      /* cudaStream_t (NULL = legacy default stream)              */
   uint32_t flags;
+  int32_t  n_schedulers;                /* S: scheduler threads taking turns (Section 3); 0 or 1 = one;
+                                           1 <= S <= STRADS_MAX_SCHEDULERS and P' <= floor(J / S)       */
 } strads_lasso_config_t;
 
 /* Optional per-round outputs; every pointer is a DEVICE address or NULL (= not wanted). */
@@ -126,7 +129,19 @@ int strads_lasso_init(const strads_lasso_config_t* cfg, strads_handle_t* out_han
  * `out` may be NULL.  Asynchronous. */
 int strads_round(strads_handle_t h, const strads_round_out_t* out);
 
-/* n_rounds rounds back to back with no host synchronisation in between. */
+/* n_rounds rounds back to back with no host synchronisation in between.
+ *
+ * Scheduler threads (Section 3, "Implementation Overview" and "Properties"): with n_schedulers = S > 1
+ * the coefficients are split into S fixed disjoint sets, scheduler s owning { j : j mod S == s } (the
+ * paper assigns them at random; permute the columns for that).  Round t is dispatched by scheduler
+ * t mod S, which draws its P' candidates from its own coefficients only (its own p_s(j); the Philox word
+ * of (seed, t, j) as before) and filters them; the update of step 3 is unchanged.  delta_j of scheduler s
+ * changes only in its own rounds, so its block for round t is fully determined once round t - S is over:
+ * strads_run prepares the blocks of up to S - 1 later rounds (steps 1 and 2, on streams of its own) while
+ * the update of the current round runs, which is the paper's "each thread has S-fold more time" and gives
+ * results identical to running the same rounds strictly one after another (strads_round does that).
+ * Each scheduler has its own slice of the workspace.  On return every piece of work has been enqueued and
+ * the configured stream waits for all of it. */
 int strads_run(strads_handle_t h, int64_t n_rounds);
 
 /* The same round as strads_round for callers whose state lives in HOST memory: copies
@@ -146,7 +161,9 @@ int strads_objective(strads_handle_t h, double* host_out);
  *                 kept_dev [P] device, counts_dev [4] device (as strads_round_out_t.counts).
  * strads_update : Eq. 2 + residual + delta refresh for a caller-supplied kept list (device; may be NULL when n_kept is 0;
  *                 distinct indices, n_kept <= P); dbeta_dev [P] device or NULL.
- * None of them advances the round index. */
+ * None of them advances the round index.  With S > 1 schedulers they act for the scheduler whose turn
+ * it is (round index mod S): strads_sample draws from its coefficients, and all three use its slice
+ * of the workspace. */
 int strads_sample(strads_handle_t h, int32_t* cand_dev);
 int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand,
                   int32_t* kept_dev, int32_t* counts_dev, float* gram_dev_or_null);
@@ -173,7 +190,8 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out);
 /* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);
 
-/* Optional step timing with CUDA events on the handle's stream.  After strads_profile_begin the next
+/* Optional step timing with CUDA events on the handle's stream (n_schedulers == 1 only: with more, the
+ * steps of different rounds overlap and have no separate times).  After strads_profile_begin the next
  * max_rounds rounds (strads_round / strads_run / strads_round_host; strads_run then launches kernel by kernel
  * instead of replaying its graph) record an event at every step boundary; strads_profile_end waits for the
  * stream and returns the summed device time in milliseconds over *rounds rounds of

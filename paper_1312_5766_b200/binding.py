@@ -45,6 +45,7 @@ class Config(C.Structure):
         ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
         ("stream", C.c_void_p),
         ("flags", C.c_uint32),
+        ("n_schedulers", C.c_int32),
     ]
 
 
@@ -144,7 +145,7 @@ class StradsLasso:
     """
 
     def __init__(self, layout, n_rows, n_cols, values, y, lam, eta, rho, n_candidates, n_keep, seed=0,
-                 row_idx=None, col_ptr=None, c_init=1e4, flags=0, beta0=None, stream=None):
+                 row_idx=None, col_ptr=None, c_init=1e4, flags=0, beta0=None, stream=None, n_schedulers=1):
         lib = load()
         dev = values.device
         assert dev.type == "cuda", "the design matrix must live on a CUDA device"
@@ -165,6 +166,7 @@ class StradsLasso:
         cfg = Config()
         cfg.layout, cfg.n_rows, cfg.n_cols, cfg.nnz, cfg.ld = self.layout, self.N, self.J, nnz, ld
         cfg.n_candidates, cfg.n_keep = self.n_candidates, self.n_keep
+        self.n_schedulers = cfg.n_schedulers = int(n_schedulers)
         need = C.c_size_t(0)
         _check(lib.strads_workspace_bytes(C.byref(cfg), C.byref(need)), "strads_workspace_bytes")
         self.workspace = torch.empty(int(need.value), dtype=torch.uint8, device=dev)

@@ -10,25 +10,40 @@
 
 using namespace strads;
 
-struct strads_lasso_s {
-  alignas(64) unsigned char gram_tmap[128];   // tensor map over the packed candidate buffer (dense layouts)
+// One scheduler thread of Section 3: its coefficients (Problem::part_index), its slice of the workspace
+// (everything steps 1 and 2 write), and what orders its work against the updates.
+struct Scheduler {
+  alignas(64) unsigned char gram_tmap[128];   // tensor map over its packed candidate buffer (dense layouts)
   Problem p;
+  int walk_grid;             // CTAs of the cooperative on-demand walk (CSC)
+  cudaStream_t stream;       // S > 1: steps 1 and 2 of its rounds are enqueued here
+  cudaEvent_t block_ready;   // its block (the kept list) is complete
+  cudaEvent_t updated;       // the update of its latest round is done: delta of its coefficients is final
+};
+
+struct strads_lasso_s {
+  Scheduler sch[STRADS_MAX_SCHEDULERS];
+  int n_sched;
   cudaStream_t stream;
   int device;
-  long long round_host;     // mirrors DeviceState::round (every round adds exactly one)
-  // optional step timing: 5 events per round (start, after sample, Gram, filter, update)
+  long long round_host;     // the round index t (every round adds exactly one); scheduler t mod S is next
+  // optional step timing: 6 events per round (start, after sample, pack, Gram, walk, update)
   cudaEvent_t* prof_events;
   long long prof_cap, prof_rounds;
-  // strads_run replays one captured round (the launch sequence of a round is fixed for a handle)
-  int walk_grid;            // CTAs of the cooperative on-demand walk (CSC)
+  // strads_run replays a captured launch sequence (fixed for a handle): one round with one scheduler,
+  // kGraphTurns turns of every scheduler, pipelined, with several
   cudaStream_t capture_stream;
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
+  cudaEvent_t fork;          // S > 1: where the schedulers' streams join the caller's stream
 };
 
 namespace {
 
 constexpr int kProfEvents = 6;   // per round: start, after sample, pack, Gram, walk, update
+constexpr int kGraphTurns = 16;  // S > 1: turns of every scheduler in the captured sequence
+
+Scheduler& on_turn(strads_lasso_s* h) { return h->sch[h->round_host % h->n_sched]; }
 
 thread_local char g_cuda_err[256] = "";
 
@@ -52,6 +67,8 @@ struct Layout {
   long long ldc;
 };
 
+int n_sched_of(const strads_lasso_config_t* c) { return c->n_schedulers > 1 ? c->n_schedulers : 1; }
+
 // Checks everything about cfg that does not need its pointers.
 int check_sizes(const strads_lasso_config_t* c) {
   if (c == nullptr) return STRADS_ERR_INVALID_ARG;
@@ -62,10 +79,14 @@ int check_sizes(const strads_lasso_config_t* c) {
   if (c->n_candidates < 1 || c->n_candidates > c->n_cols) return STRADS_ERR_INVALID_ARG;
   if (c->n_candidates > STRADS_MAX_CANDIDATES) return STRADS_ERR_UNSUPPORTED;
   if (c->n_keep < 1 || c->n_keep > c->n_candidates) return STRADS_ERR_INVALID_ARG;
+  if (c->n_schedulers < 0 || c->n_schedulers > STRADS_MAX_SCHEDULERS) return STRADS_ERR_INVALID_ARG;
+  if ((long long)c->n_candidates > c->n_cols / n_sched_of(c)) return STRADS_ERR_INVALID_ARG;   // smallest share: floor(J / S)
   return STRADS_OK;
 }
 
-Layout carve(const strads_lasso_config_t* c) {
+// Slice of the workspace of one scheduler; the first one (`first`) also holds what all share
+// (column norms, the objective's partial sums).
+Layout carve(const strads_lasso_config_t* c, bool first = true) {
   Layout L;
   L.cap_sure = c->n_candidates;
   L.cap_boundary = pow2_ceil(c->n_candidates / 2 > 2048 ? c->n_candidates / 2 : 2048);
@@ -77,7 +98,7 @@ Layout carve(const strads_lasso_config_t* c) {
   size_t o = 0;
   auto take = [&](size_t bytes) { size_t at = o; o = align_up(o + bytes); return at; };
   L.off_state = take(sizeof(DeviceState));
-  L.off_n2 = take(sizeof(double) * (size_t)c->n_cols);
+  L.off_n2 = take(first ? sizeof(double) * (size_t)c->n_cols : 0);
   L.off_hist = take(sizeof(unsigned int) * kHistBins);
   L.off_sure = take(sizeof(unsigned long long) * (size_t)L.cap_sure);
   L.off_boundary = take(sizeof(unsigned long long) * (size_t)L.cap_boundary);
@@ -89,7 +110,7 @@ Layout carve(const strads_lasso_config_t* c) {
   L.off_conflict = take(sizeof(unsigned int) * (size_t)c->n_candidates * L.mask_words);
   L.off_dot_partial = take(sizeof(double) * (size_t)c->n_keep * L.dot_parts);
   L.off_dot_ticket = take(sizeof(unsigned int) * (size_t)c->n_keep);
-  L.off_obj = take(sizeof(double) * 2 * kObjBlocks);
+  L.off_obj = take(first ? sizeof(double) * 2 * kObjBlocks : 0);
   L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // borderline pairs of the TF32 screen (1 MB)
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
   L.ldc = (c->n_rows + 3) / 4 * 4;
@@ -108,10 +129,9 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
-cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
-                        bool window = false, cudaEvent_t after_pack = nullptr) {
-  const Problem& p = h->p;
-  cudaStream_t s = h->stream;
+cudaError_t launch_gram(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, float* gram_dbg,
+                        bool only_if_short, bool window = false, cudaEvent_t after_pack = nullptr) {
+  const Problem& p = sc.p;
   if (after_pack != nullptr && (p.layout == STRADS_CSC || gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM))) {
     const cudaError_t e = cudaEventRecord(after_pack, s);          // these paths have no pack kernel
     if (e != cudaSuccess) return e;
@@ -119,7 +139,7 @@ cudaError_t launch_gram(const strads_lasso_s* h, const int* cand, int n_cand, fl
   }
   if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, window, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, h->gram_tmap, cand, n_cand, only_if_short, window, after_pack, s);
+  return launch_gram_dense_tc(p, sc.gram_tmap, cand, n_cand, only_if_short, window, after_pack, s);
 }
 
 // The greedy walk stops at P kept, so it normally looks at little more than the first P candidates: form the
@@ -132,46 +152,51 @@ int window_of(const Problem& p, int n_cand) {
   return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
 }
 
-int gram_and_filter(strads_lasso_s* h, const int* cand, int n_cand, float* gram_dbg, cudaEvent_t after_pack = nullptr,
-                    cudaEvent_t after_gram = nullptr) {
-  const Problem& p = h->p;
+int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, float* gram_dbg,
+                    cudaEvent_t after_pack = nullptr, cudaEvent_t after_gram = nullptr) {
+  const Problem& p = sc.p;
   if (p.flags & STRADS_FLAG_NO_FILTER) {
-    if (after_pack) CK(cudaEventRecord(after_pack, h->stream));
-    if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
-    CK(launch_filter(p, cand, n_cand, n_cand, false, p.kept, h->stream));
+    if (after_pack) CK(cudaEventRecord(after_pack, s));
+    if (after_gram) CK(cudaEventRecord(after_gram, s));
+    CK(launch_filter(p, cand, n_cand, n_cand, false, p.kept, s));
     return STRADS_OK;
   }
   const int window = gram_dbg != nullptr ? n_cand : window_of(p, n_cand);
-  CK(launch_gram(h, cand, window, gram_dbg, false, window < n_cand, after_pack));
-  if (after_gram) CK(cudaEventRecord(after_gram, h->stream));
-  CK(launch_filter(p, cand, window, n_cand, false, p.kept, h->stream));
+  CK(launch_gram(sc, s, cand, window, gram_dbg, false, window < n_cand, after_pack));
+  if (after_gram) CK(cudaEventRecord(after_gram, s));
+  CK(launch_filter(p, cand, window, n_cand, false, p.kept, s));
   if (window < n_cand) {
     if (p.layout == STRADS_CSC) {
       // whole list, conflict rows formed only for the candidates the walk keeps
-      CK(launch_walk_csc(p, cand, n_cand, h->walk_grid, true, p.kept, h->stream));
+      CK(launch_walk_csc(p, cand, n_cand, sc.walk_grid, true, p.kept, s));
     } else {
-      CK(launch_gram(h, cand, n_cand, nullptr, true));
-      CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, h->stream));
+      CK(launch_gram(sc, s, cand, n_cand, nullptr, true));
+      CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, s));
     }
   }
   return STRADS_OK;
 }
 
+// after a tensor-core Gram the kept columns are read from the packed candidate buffer
+bool update_reads_packed(const Problem& p, bool gram_exported) {
+  return p.layout == STRADS_DENSE_COLMAJOR && !(p.flags & (STRADS_FLAG_NO_FILTER | STRADS_FLAG_SIMT_GRAM)) && !gram_exported;
+}
+
+// One round, every step on the caller's stream, by the scheduler whose turn it is.
 int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
-  const Problem& p = h->p;
+  const Scheduler& sc = on_turn(h);
+  const Problem& p = sc.p;
   cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + kProfEvents * h->prof_rounds : nullptr;
   if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
   if (ev) CK(cudaEventRecord(ev[1], h->stream));
   {
-    const int rc = gram_and_filter(h, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr, ev ? ev[3] : nullptr);
+    const int rc = gram_and_filter(sc, h->stream, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr,
+                                   ev ? ev[3] : nullptr);
     if (rc) return rc;
   }
   if (ev) CK(cudaEventRecord(ev[4], h->stream));
-  // after a tensor-core Gram the kept columns are read from the packed candidate buffer
-  const bool packed = p.layout == STRADS_DENSE_COLMAJOR && !(p.flags & (STRADS_FLAG_NO_FILTER | STRADS_FLAG_SIMT_GRAM)) &&
-                      !(out && out->gram);
-  CK(launch_update(p, p.kept, 1, packed, h->stream));
+  CK(launch_update(p, p.kept, 1, update_reads_packed(p, out && out->gram), h->stream));
   if (ev) { CK(cudaEventRecord(ev[5], h->stream)); h->prof_rounds += 1; }
   h->round_host += 1;
   if (out != nullptr) {
@@ -179,6 +204,86 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
     if (out->kept || out->dbeta || out->counts) CK(launch_export(p, p.kept, out->kept, out->dbeta, out->counts, h->stream));
   }
   return STRADS_OK;
+}
+
+// `count` rounds with S > 1 schedulers, pipelined ("Properties of STRADS": taking turns leaves every
+// scheduler S-fold more time to prepare its block).  Steps 1 and 2 of a round go to its scheduler's own
+// stream and need only that scheduler's previous update; the updates follow one another on `main` in round
+// order, each waiting for its block.  Blocks of up to S - 1 later rounds are therefore prepared while an
+// update runs, with the results of running the rounds one by one.  Everything enqueued here is ordered
+// before whatever is enqueued on `main` afterwards: the last operation of every scheduler stream is a
+// block that an update on `main` waits for.
+int pipelined_rounds(strads_lasso_s* h, long long count, cudaStream_t main) {
+  bool joined[STRADS_MAX_SCHEDULERS] = {};
+  CK(cudaEventRecord(h->fork, main));
+  for (long long i = 0; i < count; ++i) {
+    const int s = (int)(h->round_host % h->n_sched);
+    const Scheduler& sc = h->sch[s];
+    const Problem& p = sc.p;
+    CK(cudaStreamWaitEvent(sc.stream, joined[s] ? sc.updated : h->fork, 0));
+    joined[s] = true;
+    CK(launch_sample(p, p.cand, sc.stream));
+    const int rc = gram_and_filter(sc, sc.stream, p.cand, p.n_cand, nullptr);
+    if (rc) return rc;
+    CK(cudaEventRecord(sc.block_ready, sc.stream));
+    CK(cudaStreamWaitEvent(main, sc.block_ready, 0));
+    CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+    CK(cudaEventRecord(sc.updated, main));
+    h->round_host += 1;
+  }
+  return STRADS_OK;
+}
+
+// Workspace pointers of scheduler `s` of `S` (slice at `ws`, laid out by L); X, y, beta, resid, delta, the
+// column norms and the objective's partial sums are those of the first scheduler.
+void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, char* ws, int s, int S, const Problem* first) {
+  p.layout = c->layout; p.N = c->n_rows; p.J = c->n_cols; p.ld = c->ld;
+  p.xv = c->x_values; p.xrow = c->x_row_idx; p.xptr = reinterpret_cast<const long long*>(c->x_col_ptr);
+  p.y = c->y; p.beta = c->beta; p.resid = c->resid; p.delta = c->delta;
+  p.lambda = c->lambda; p.eta = c->eta; p.rho = c->rho; p.c_init = c->c_init;
+  p.n_cand = c->n_candidates; p.n_keep = c->n_keep; p.seed = c->seed; p.flags = c->flags;
+  p.st = reinterpret_cast<DeviceState*>(ws + L.off_state);
+  p.n2 = first ? first->n2 : reinterpret_cast<double*>(ws + L.off_n2);
+  p.hist = reinterpret_cast<unsigned int*>(ws + L.off_hist);
+  p.sure = reinterpret_cast<unsigned long long*>(ws + L.off_sure);
+  p.boundary = reinterpret_cast<unsigned long long*>(ws + L.off_boundary);
+  p.cap_sure = L.cap_sure; p.cap_boundary = L.cap_boundary;
+  p.cand = reinterpret_cast<int*>(ws + L.off_cand);
+  p.kept = reinterpret_cast<int*>(ws + L.off_kept);
+  p.kept_pos = reinterpret_cast<int*>(ws + L.off_kept_pos);
+  p.dbeta = reinterpret_cast<float*>(ws + L.off_dbeta);
+  p.dbeta64 = reinterpret_cast<double*>(ws + L.off_dbeta64);
+  p.conflict = reinterpret_cast<unsigned int*>(ws + L.off_conflict);
+  p.mask_words = L.mask_words;
+  p.dot_partial = reinterpret_cast<double*>(ws + L.off_dot_partial);
+  p.dot_ticket = reinterpret_cast<unsigned int*>(ws + L.off_dot_ticket);
+  p.dot_parts = L.dot_parts;
+  p.obj_partial = first ? first->obj_partial : reinterpret_cast<double*>(ws + L.off_obj);
+  p.amb_pairs = reinterpret_cast<unsigned int*>(ws + L.off_amb);
+  p.cap_amb = L.cap_amb;
+  p.xc = reinterpret_cast<float*>(ws + L.off_xc);
+  p.ldc = L.ldc;
+  p.cand_cur = nullptr;
+  p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
+  p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
+  p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
+  p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
+  p.partial_tiles = L.partial_tiles;
+  p.part_count = S; p.part_index = s;
+  p.sm_count = first ? first->sm_count : 0;
+}
+
+void release(strads_lasso_s* h) {
+  for (int s = 0; s < STRADS_MAX_SCHEDULERS; ++s) {
+    if (h->sch[s].stream != nullptr) cudaStreamDestroy(h->sch[s].stream);
+    if (h->sch[s].block_ready != nullptr) cudaEventDestroy(h->sch[s].block_ready);
+    if (h->sch[s].updated != nullptr) cudaEventDestroy(h->sch[s].updated);
+  }
+  if (h->fork != nullptr) cudaEventDestroy(h->fork);
+  if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
+  if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
+  if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
+  delete h;
 }
 
 }  // namespace
@@ -189,7 +294,7 @@ int strads_workspace_bytes(const strads_lasso_config_t* cfg, size_t* out_bytes) 
   if (out_bytes == nullptr) return STRADS_ERR_INVALID_ARG;
   const int rc = check_sizes(cfg);
   if (rc) return rc;
-  *out_bytes = carve(cfg).total;
+  *out_bytes = carve(cfg).total + (size_t)(n_sched_of(cfg) - 1) * carve(cfg, false).total;
   return STRADS_OK;
 }
 
@@ -205,68 +310,55 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
     return STRADS_ERR_INVALID_ARG;
   if (!(c->lambda >= 0.f) || !(c->eta > 0.f) || !(c->rho > 0.f) || !(c->c_init > 0.f)) return STRADS_ERR_INVALID_ARG;
   if (!std::isfinite(c->lambda) || !std::isfinite(c->eta) || !std::isfinite(c->c_init)) return STRADS_ERR_INVALID_ARG;
-  const Layout L = carve(c);
-  if (c->workspace_bytes < L.total) return STRADS_ERR_WORKSPACE_TOO_SMALL;
+  const int S = n_sched_of(c);
+  const Layout L = carve(c), Lrest = carve(c, false);
+  if (c->workspace_bytes < L.total + (size_t)(S - 1) * Lrest.total) return STRADS_ERR_WORKSPACE_TOO_SMALL;
 
-  strads_lasso_s* h = new (std::nothrow) strads_lasso_s();
+  strads_lasso_s* h = new (std::nothrow) strads_lasso_s();     // value-initialised: every pointer null
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
-  Problem& p = h->p;
-  p.layout = c->layout; p.N = c->n_rows; p.J = c->n_cols; p.ld = c->ld;
-  p.xv = c->x_values; p.xrow = c->x_row_idx; p.xptr = reinterpret_cast<const long long*>(c->x_col_ptr);
-  p.y = c->y; p.beta = c->beta; p.resid = c->resid; p.delta = c->delta;
-  p.lambda = c->lambda; p.eta = c->eta; p.rho = c->rho; p.c_init = c->c_init;
-  p.n_cand = c->n_candidates; p.n_keep = c->n_keep; p.seed = c->seed; p.flags = c->flags;
-  char* ws = static_cast<char*>(c->workspace);
-  p.st = reinterpret_cast<DeviceState*>(ws + L.off_state);
-  p.n2 = reinterpret_cast<double*>(ws + L.off_n2);
-  p.hist = reinterpret_cast<unsigned int*>(ws + L.off_hist);
-  p.sure = reinterpret_cast<unsigned long long*>(ws + L.off_sure);
-  p.boundary = reinterpret_cast<unsigned long long*>(ws + L.off_boundary);
-  p.cap_sure = L.cap_sure; p.cap_boundary = L.cap_boundary;
-  p.cand = reinterpret_cast<int*>(ws + L.off_cand);
-  p.kept = reinterpret_cast<int*>(ws + L.off_kept);
-  p.kept_pos = reinterpret_cast<int*>(ws + L.off_kept_pos);
-  p.dbeta = reinterpret_cast<float*>(ws + L.off_dbeta);
-  p.dbeta64 = reinterpret_cast<double*>(ws + L.off_dbeta64);
-  p.conflict = reinterpret_cast<unsigned int*>(ws + L.off_conflict);
-  p.mask_words = L.mask_words;
-  p.dot_partial = reinterpret_cast<double*>(ws + L.off_dot_partial);
-  p.dot_ticket = reinterpret_cast<unsigned int*>(ws + L.off_dot_ticket);
-  p.dot_parts = L.dot_parts;
-  p.obj_partial = reinterpret_cast<double*>(ws + L.off_obj);
-  p.amb_pairs = reinterpret_cast<unsigned int*>(ws + L.off_amb);
-  p.cap_amb = L.cap_amb;
-  p.xc = reinterpret_cast<float*>(ws + L.off_xc);
-  p.ldc = L.ldc;
-  p.cand_cur = nullptr;
-  p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
-  p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
-  p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
-  p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
-  p.partial_tiles = L.partial_tiles;
+  h->n_sched = S;
   h->stream = static_cast<cudaStream_t>(c->stream);
   h->round_host = 0;
-  h->prof_events = nullptr; h->prof_cap = 0; h->prof_rounds = 0;
-  h->capture_stream = nullptr; h->round_graph = nullptr; h->round_exec = nullptr;
-
-  auto fail = [&](int code) { delete h; return code; };
+  auto fail = [&](int code) { release(h); return code; };
   cudaError_t e = cudaGetDevice(&h->device);
   if (e != cudaSuccess) return fail(cuda_fail(e, "cudaGetDevice"));
-  e = cudaDeviceGetAttribute(&p.sm_count, cudaDevAttrMultiProcessorCount, h->device);
+  int sm_count = 0;
+  e = cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, h->device);
   if (e != cudaSuccess) return fail(cuda_fail(e, "cudaDeviceGetAttribute"));
-  if ((e = prepare_sample(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_sample"));
-  if ((e = prepare_filter(p)) != cudaSuccess) return fail(cuda_fail(e, "prepare_filter"));
-  if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
-  if (p.layout == STRADS_DENSE_COLMAJOR && (e = encode_gram_tensor_map(p, h->gram_tmap)) != cudaSuccess)
-    return fail(cuda_fail(e, "encode_gram_tensor_map"));
-  h->walk_grid = 0;
-  if (p.layout == STRADS_CSC) {
-    if ((e = prepare_walk_csc(p, &h->walk_grid)) != cudaSuccess) return fail(cuda_fail(e, "prepare_walk_csc"));
-    if ((e = cudaMemsetAsync(p.walk_ctl, 0, sizeof(WalkControl), h->stream)) != cudaSuccess)
-      return fail(cuda_fail(e, "cudaMemsetAsync"));
+
+  char* ws = static_cast<char*>(c->workspace);
+  for (int s = 0; s < S; ++s) {
+    Problem& p = h->sch[s].p;
+    fill_problem(p, c, s == 0 ? L : Lrest, s == 0 ? ws : ws + L.total + (size_t)(s - 1) * Lrest.total, s, S,
+                 s == 0 ? nullptr : &h->sch[0].p);
+    p.sm_count = sm_count;
   }
-  if ((e = launch_init(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
-  if ((e = launch_resid_from_beta(p, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
+  const Problem& p0 = h->sch[0].p;
+  if ((e = prepare_sample(p0)) != cudaSuccess) return fail(cuda_fail(e, "prepare_sample"));
+  if ((e = prepare_filter(p0)) != cudaSuccess) return fail(cuda_fail(e, "prepare_filter"));
+  if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
+  if ((e = launch_init(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
+  if ((e = launch_resid_from_beta(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
+  for (int s = 0; s < S; ++s) {
+    Scheduler& sc = h->sch[s];
+    if (sc.p.layout == STRADS_DENSE_COLMAJOR && (e = encode_gram_tensor_map(sc.p, sc.gram_tmap)) != cudaSuccess)
+      return fail(cuda_fail(e, "encode_gram_tensor_map"));
+    if (sc.p.layout == STRADS_CSC) {
+      if ((e = prepare_walk_csc(sc.p, &sc.walk_grid)) != cudaSuccess) return fail(cuda_fail(e, "prepare_walk_csc"));
+      if ((e = cudaMemsetAsync(sc.p.walk_ctl, 0, sizeof(WalkControl), h->stream)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaMemsetAsync"));
+    }
+    if (s > 0 && (e = launch_init_scheduler(sc.p, p0, h->stream)) != cudaSuccess)
+      return fail(cuda_fail(e, "launch_init_scheduler"));
+    if (S > 1) {
+      if ((e = cudaStreamCreateWithFlags(&sc.stream, cudaStreamNonBlocking)) != cudaSuccess ||
+          (e = cudaEventCreateWithFlags(&sc.block_ready, cudaEventDisableTiming)) != cudaSuccess ||
+          (e = cudaEventCreateWithFlags(&sc.updated, cudaEventDisableTiming)) != cudaSuccess)
+        return fail(cuda_fail(e, "scheduler stream"));
+    }
+  }
+  if (S > 1 && (e = cudaEventCreateWithFlags(&h->fork, cudaEventDisableTiming)) != cudaSuccess)
+    return fail(cuda_fail(e, "cudaEventCreate"));
   *out_handle = h;
   return STRADS_OK;
 }
@@ -276,8 +368,12 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out) {
   return one_round(h, out);
 }
 
-// Captures the kernel sequence of one round into a graph (on a private stream: the caller's may be the legacy
-// default stream, which cannot be captured; nothing executes during capture).
+// Rounds that one launch of the captured sequence runs.
+static long long graph_rounds(const strads_lasso_s* h) { return h->n_sched > 1 ? (long long)kGraphTurns * h->n_sched : 1; }
+
+// Captures the launch sequence of graph_rounds() rounds into a graph (on a private stream: the caller's may be
+// the legacy default stream, which cannot be captured; nothing executes during capture).  With several
+// schedulers the sequence starts with scheduler 0.
 static int build_round_graph(strads_lasso_s* h) {
   CK(cudaStreamCreateWithFlags(&h->capture_stream, cudaStreamNonBlocking));
   cudaStream_t user = h->stream;
@@ -286,7 +382,7 @@ static int build_round_graph(strads_lasso_s* h) {
   cudaError_t e = cudaStreamBeginCapture(h->capture_stream, cudaStreamCaptureModeThreadLocal);
   int rc = STRADS_OK;
   if (e == cudaSuccess) {
-    rc = one_round(h, nullptr);
+    rc = h->n_sched > 1 ? pipelined_rounds(h, graph_rounds(h), h->capture_stream) : one_round(h, nullptr);
     e = cudaStreamEndCapture(h->capture_stream, &h->round_graph);
   }
   h->stream = user;
@@ -299,6 +395,29 @@ static int build_round_graph(strads_lasso_s* h) {
 
 int strads_run(strads_handle_t h, int64_t n_rounds) {
   if (h == nullptr || n_rounds < 0) return STRADS_ERR_INVALID_ARG;
+  if (h->n_sched > 1) {
+    // whole captured sequences where they fit (they start with scheduler 0), the rest enqueued directly
+    const long long R = graph_rounds(h);
+    long long left = n_rounds;
+    while (left > 0) {
+      if (h->round_host % h->n_sched == 0 && left >= R) {
+        if (h->round_exec == nullptr) {
+          const int rc = build_round_graph(h);
+          if (rc) return rc;
+        }
+        CK(cudaGraphLaunch(h->round_exec, h->stream));
+        h->round_host += R;
+        left -= R;
+      } else {
+        const long long to_turn0 = h->n_sched - h->round_host % h->n_sched;
+        const long long count = left < R ? left : to_turn0;
+        const int rc = pipelined_rounds(h, count, h->stream);
+        if (rc) return rc;
+        left -= count;
+      }
+    }
+    return STRADS_OK;
+  }
   const bool use_graph = h->prof_events == nullptr && n_rounds > 1;   // step timing needs events between kernels
   if (use_graph && h->round_exec == nullptr) {
     const int rc = build_round_graph(h);
@@ -319,7 +438,7 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
 int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, float* delta_host,
                       int32_t* kept_host, float* dbeta_host, int32_t* counts_host) {
   if (h == nullptr || !beta_host || !resid_host || !delta_host) return STRADS_ERR_INVALID_ARG;
-  const Problem& p = h->p;
+  const Problem& p = on_turn(h).p;
   CK(cudaMemcpyAsync(p.beta, beta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
   CK(cudaMemcpyAsync(p.resid, resid_host, sizeof(float) * p.N, cudaMemcpyHostToDevice, h->stream));
   CK(cudaMemcpyAsync(p.delta, delta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
@@ -337,33 +456,34 @@ int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, fl
 
 int strads_objective(strads_handle_t h, double* host_out) {
   if (h == nullptr || host_out == nullptr) return STRADS_ERR_INVALID_ARG;
-  CK(launch_objective(h->p, h->stream));
-  CK(cudaMemcpyAsync(host_out, &h->p.st->objective, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
+  CK(launch_objective(h->sch[0].p, h->stream));
+  CK(cudaMemcpyAsync(host_out, &h->sch[0].p.st->objective, sizeof(double), cudaMemcpyDeviceToHost, h->stream));
   CK(cudaStreamSynchronize(h->stream));
   return STRADS_OK;
 }
 
 int strads_sample(strads_handle_t h, int32_t* cand_dev) {
   if (h == nullptr || cand_dev == nullptr) return STRADS_ERR_INVALID_ARG;
-  CK(launch_sample(h->p, cand_dev, h->stream));
+  CK(launch_sample(on_turn(h).p, cand_dev, h->stream));
   return STRADS_OK;
 }
 
 int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand, int32_t* kept_dev, int32_t* counts_dev,
                   float* gram_dev_or_null) {
   if (h == nullptr || cand_dev == nullptr || kept_dev == nullptr) return STRADS_ERR_INVALID_ARG;
-  if (n_cand < 0 || n_cand > h->p.n_cand) return STRADS_ERR_INVALID_ARG;
-  CK(launch_set_counts(h->p, n_cand, 0, 0, h->stream));
-  const int rc = gram_and_filter(h, cand_dev, n_cand, gram_dev_or_null);
+  const Scheduler& sc = on_turn(h);
+  if (n_cand < 0 || n_cand > sc.p.n_cand) return STRADS_ERR_INVALID_ARG;
+  CK(launch_set_counts(sc.p, n_cand, 0, 0, h->stream));
+  const int rc = gram_and_filter(sc, h->stream, cand_dev, n_cand, gram_dev_or_null);
   if (rc) return rc;
-  CK(launch_export(h->p, h->p.kept, kept_dev, nullptr, counts_dev, h->stream));
+  CK(launch_export(sc.p, sc.p.kept, kept_dev, nullptr, counts_dev, h->stream));
   return STRADS_OK;
 }
 
 int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, float* dbeta_dev) {
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
-  if (n_kept < 0 || n_kept > h->p.n_keep || (n_kept > 0 && kept_dev == nullptr)) return STRADS_ERR_INVALID_ARG;
-  const Problem& p = h->p;
+  const Problem& p = on_turn(h).p;
+  if (n_kept < 0 || n_kept > p.n_keep || (n_kept > 0 && kept_dev == nullptr)) return STRADS_ERR_INVALID_ARG;
   CK(launch_set_counts(p, n_kept, n_kept, n_kept, h->stream));
   if (n_kept > 0)
     CK(cudaMemcpyAsync(p.kept, kept_dev, sizeof(int) * n_kept, cudaMemcpyDeviceToDevice, h->stream));
@@ -381,26 +501,35 @@ int strads_get_round(strads_handle_t h, int64_t* t) {
 int strads_set_round(strads_handle_t h, int64_t t) {
   if (h == nullptr || t < 0) return STRADS_ERR_INVALID_ARG;
   h->round_host = t;
-  const unsigned long long v = (unsigned long long)t;
-  CK(cudaMemcpyAsync(&h->p.st->round, &v, sizeof(v), cudaMemcpyHostToDevice, h->stream));
-  CK(cudaStreamSynchronize(h->stream));   // `v` lives on this stack frame
+  unsigned long long next[STRADS_MAX_SCHEDULERS];          // every scheduler's next turn at or after t
+  for (int s = 0; s < h->n_sched; ++s) {
+    next[s] = (unsigned long long)t + (unsigned long long)(((s - t % h->n_sched) + h->n_sched) % h->n_sched);
+    CK(cudaMemcpyAsync(&h->sch[s].p.st->round, &next[s], sizeof(next[s]), cudaMemcpyHostToDevice, h->stream));
+  }
+  CK(cudaStreamSynchronize(h->stream));   // `next` lives on this stack frame
   return STRADS_OK;
 }
 
 int strads_totals(strads_handle_t h, int64_t* totals) {
   if (h == nullptr || totals == nullptr) return STRADS_ERR_INVALID_ARG;
-  unsigned long long t[4];
-  CK(cudaMemcpyAsync(t, h->p.st->totals, sizeof(t), cudaMemcpyDeviceToHost, h->stream));
+  unsigned long long t[STRADS_MAX_SCHEDULERS][4];
+  for (int s = 0; s < h->n_sched; ++s)
+    CK(cudaMemcpyAsync(t[s], h->sch[s].p.st->totals, sizeof(t[s]), cudaMemcpyDeviceToHost, h->stream));
   CK(cudaStreamSynchronize(h->stream));
-  for (int i = 0; i < 4; ++i) totals[i] = (int64_t)t[i];
+  for (int i = 0; i < 4; ++i) {
+    totals[i] = 0;
+    for (int s = 0; s < h->n_sched; ++s) totals[i] += (int64_t)t[s][i];
+  }
   return STRADS_OK;
 }
 
 int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
-  unsigned int bits = 0;
-  CK(cudaMemcpyAsync(&bits, &h->p.st->status, sizeof(bits), cudaMemcpyDeviceToHost, h->stream));
+  unsigned int each[STRADS_MAX_SCHEDULERS] = {}, bits = 0;
+  for (int s = 0; s < h->n_sched; ++s)
+    CK(cudaMemcpyAsync(&each[s], &h->sch[s].p.st->status, sizeof(each[s]), cudaMemcpyDeviceToHost, h->stream));
   CK(cudaStreamSynchronize(h->stream));
+  for (int s = 0; s < h->n_sched; ++s) bits |= each[s];
   if (bits_host_out) *bits_host_out = bits;
   if (bits & STRADS_STATUS_WAIT_EXPIRED) return STRADS_ERR_TIMEOUT;
   if (bits & STRADS_STATUS_NONFINITE) return STRADS_ERR_NUMERIC;
@@ -409,13 +538,13 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
 
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out) {
   if (h == nullptr || dev_ptr_out == nullptr) return STRADS_ERR_INVALID_ARG;
-  *dev_ptr_out = h->p.n2;
+  *dev_ptr_out = h->sch[0].p.n2;
   return STRADS_OK;
 }
 
 int strads_profile_begin(strads_handle_t h, int64_t max_rounds) {
   if (h == nullptr || max_rounds < 1 || max_rounds > (1 << 20)) return STRADS_ERR_INVALID_ARG;
-  if (h->prof_events != nullptr) return STRADS_ERR_INVALID_ARG;
+  if (h->prof_events != nullptr || h->n_sched > 1) return STRADS_ERR_INVALID_ARG;
   h->prof_events = new (std::nothrow) cudaEvent_t[kProfEvents * max_rounds];
   if (h->prof_events == nullptr) return STRADS_ERR_INVALID_ARG;
   for (long long i = 0; i < kProfEvents * max_rounds; ++i) {
@@ -460,10 +589,7 @@ int strads_destroy(strads_handle_t h) {
     for (long long i = 0; i < kProfEvents * h->prof_cap; ++i) cudaEventDestroy(h->prof_events[i]);
     delete[] h->prof_events;
   }
-  if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
-  if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
-  if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
-  delete h;
+  release(h);
   return STRADS_OK;
 }
 

@@ -40,7 +40,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; }
     return;
   }
-  if (p.layout == STRADS_CSC && n_cand < n_total && p.st->prefer_walk && (p.st->round & 63ull) != 0) {
+  if (p.layout == STRADS_CSC && n_cand < n_total && p.st->prefer_walk && ((p.st->round / (unsigned)p.part_count) & 63ull) != 0) {
     if (threadIdx.x == 0) p.st->window_short = 1;    // window attempt skipped: go straight to the whole-list walk
     return;
   }

@@ -15,7 +15,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
                                                         float* __restrict__ gram_dbg, int only_if_short, int window) {
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
-  if (window && p.st->prefer_walk && (p.st->round & 63ull) != 0) return;   // the window attempt is being skipped
+  if (window && p.st->prefer_walk && ((p.st->round / (unsigned)p.part_count) & 63ull) != 0) return;   // the window attempt is being skipped
   __shared__ int arow[kStage];
   __shared__ float aval[kStage];
   const int a = blockIdx.x;

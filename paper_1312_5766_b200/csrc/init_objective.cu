@@ -130,7 +130,28 @@ __global__ void k_objective_final(Problem p) {
   }
 }
 
+// State of a further scheduler: zeroed like the first one's, with what init measured copied over and its
+// first turn (round index = its own index).
+__global__ void k_scheduler_state(Problem p, const DeviceState* first) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x, stride = gridDim.x * blockDim.x;
+  if (i == 0) {
+    DeviceState* st = p.st;
+    st->round = (unsigned long long)p.part_index;
+    st->x_abs_max = first->x_abs_max;
+    st->beta0_nonzero = first->beta0_nonzero;
+  }
+  for (int b = i; b < kHistBins; b += stride) p.hist[b] = 0;
+  for (int a = i; a < p.n_keep; a += stride) p.dot_ticket[a] = 0;
+}
+
 }  // namespace
+
+cudaError_t launch_init_scheduler(const Problem& p, const Problem& first, cudaStream_t s) {
+  const cudaError_t e = cudaMemsetAsync(p.st, 0, sizeof(DeviceState), s);
+  if (e != cudaSuccess) return e;
+  k_scheduler_state<<<16, 256, 0, s>>>(p, first.st);
+  return cudaGetLastError();
+}
 
 cudaError_t launch_init(const Problem& p, cudaStream_t s) {
   cudaError_t e = cudaMemsetAsync(p.st, 0, sizeof(DeviceState), s);

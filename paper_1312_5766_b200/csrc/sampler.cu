@@ -32,6 +32,14 @@ __device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned lon
   philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
   const long long j0 = g * 4;
   const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  if (p.part_count > 1) {                              // only the coefficients this scheduler owns take part
+    const unsigned int S = (unsigned)p.part_count, r0 = (unsigned int)j0 % S;
+#pragma unroll
+    for (unsigned int i = 0; i < 4; ++i)
+      if (j0 + i < p.J && (r0 + i) % S == (unsigned)p.part_index)
+        f(race_key64(__ldg(p.delta + j0 + i), p.eta, w[i], (uint32_t)(j0 + i), uniform));
+    return;
+  }
   if (j0 + 3 < p.J) {
     const float4 d = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
     f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, uniform));

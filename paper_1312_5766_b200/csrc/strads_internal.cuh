@@ -18,7 +18,7 @@ struct SelectState {            // written by the sampler's histogram kernel, re
 };
 
 struct DeviceState {
-  unsigned long long round;     // t, the Philox counter word
+  unsigned long long round;     // t, the Philox counter word (of this scheduler's next round: t mod S == its index)
   unsigned long long totals[4]; // rounds, examined, kept, nonzero
   unsigned int status;          // STRADS_STATUS_* bits
   unsigned int hist_ticket;     // "last block done" tickets
@@ -90,6 +90,8 @@ struct Problem {
   unsigned int* walk_rows;      // [32][mask_words] conflict rows of the batch in flight
   WalkControl* walk_ctl;
   int sm_count;
+  // scheduler threads: this Problem is scheduler part_index of part_count and owns { j : j mod part_count == part_index }
+  int part_count, part_index;
 };
 static constexpr int kObjBlocks = 296;
 
@@ -215,6 +217,7 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
 // ---------------------------------------------------------------------------------------------
 cudaError_t launch_init(const Problem& p, cudaStream_t s);
 cudaError_t launch_resid_from_beta(const Problem& p, cudaStream_t s);
+cudaError_t launch_init_scheduler(const Problem& p, const Problem& first, cudaStream_t s);   // after launch_init of `first`
 cudaError_t launch_objective(const Problem& p, cudaStream_t s);
 cudaError_t prepare_sample(const Problem& p);
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);

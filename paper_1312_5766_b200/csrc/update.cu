@@ -156,7 +156,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSourc
   if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
     DeviceState* st = p.st;
     st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
-    st->round += 1;
+    st->round += (unsigned long long)p.part_count;       // this scheduler's next turn
   }
 }
 
@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, const int* __
   if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
     DeviceState* st = p.st;
     st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
-    st->round += 1;
+    st->round += (unsigned long long)p.part_count;       // this scheduler's next turn
   }
 }
 

@@ -56,6 +56,21 @@ def test_workspace_query_and_size_checks(lib):
     assert lib.strads_workspace_bytes(C.byref(cfg), C.byref(out)) == -7          # beyond STRADS_MAX_CANDIDATES
     assert lib.strads_workspace_bytes(None, C.byref(out)) == -1
     assert lib.strads_workspace_bytes(C.byref(cfg), None) == -1
+    # scheduler threads: every one has its own slice (the column norms are shared), S and P' <= J / S are checked
+    sizes = []
+    for S in (0, 1, 2, 4):
+        cfg = b.Config()
+        cfg.layout, cfg.n_rows, cfg.n_cols, cfg.ld, cfg.n_candidates, cfg.n_keep = 0, 1000, 100_000, 1000, 2048, 256
+        cfg.n_schedulers = S
+        assert lib.strads_workspace_bytes(C.byref(cfg), C.byref(out)) == 0
+        sizes.append(out.value)
+    assert sizes[0] == sizes[1] < sizes[2] < sizes[3]
+    assert sizes[3] - sizes[2] == 2 * (sizes[2] - sizes[1]) and sizes[2] - sizes[1] < sizes[1] - 8 * 100_000 + 4096
+    for S, n_cand in ((-1, 2048), (9, 2048), (4, 16_384 + 0), (8, 12_501)):
+        cfg = b.Config()
+        cfg.layout, cfg.n_rows, cfg.n_cols, cfg.ld, cfg.n_candidates, cfg.n_keep = 0, 1000, 100_000 if S != 4 else 65_000, 1000, n_cand, 256
+        cfg.n_schedulers = S
+        assert lib.strads_workspace_bytes(C.byref(cfg), C.byref(out)) == -1, (S, n_cand)
 
 
 def test_init_rejects_bad_pointers_and_parameters_without_touching_the_gpu(lib):

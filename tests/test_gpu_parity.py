@@ -460,8 +460,9 @@ def test_window_equals_full_gram(name, n_keep):
 @pytest.mark.parametrize("name,n_keep,n_cand", [("dense", 24, 1024), ("dense_grouped", 120, 1024), ("dense_grouped", 40, 1024),
                                                 ("csc", 100, 1000), ("csc_zipf", 300, 1500)])
 def test_graph_replay_equals_round_by_round(name, n_keep, n_cand):
-    """strads_run replays a captured graph in which the 3xTF32 fallback and the whole-list retry are IF nodes;
-    the state it leaves must be bit-identical to calling strads_round the same number of times."""
+    """strads_run replays a captured round in which the whole-list retry and its 3xTF32 fallback are launches
+    that return at once unless the window was too short; the state it leaves must be bit-identical to calling
+    strads_round the same number of times."""
     cfg = dict(_small_problems()[name], n_keep=n_keep, n_candidates=n_cand)
     p = wl.make_problem(cfg, seed=14)
     a, b = _solver(p), _solver(p)
