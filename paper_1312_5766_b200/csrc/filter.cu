@@ -1,37 +1,33 @@
 // SAP step 2 / Algorithm 1 "choose a set B1 of <= P coefficients from U such that |x_j^T x_k| < rho":
 // greedy first-fit over the candidates in sampling order, on the conflict bits of the Gram kernel.
 //
-// The walk is a serial chain (whether candidate i is kept depends on every earlier decision), and each
-// keep needs the conflict row of the kept candidate: a dependent memory access.  To take that latency
-// off the chain, one CTA works in batches of 64: the next 64 still-unblocked candidates (the only ones
-// that can be kept next) are found with a warp scan, their conflict rows are fetched together into
-// shared memory, a thread per candidate extracts its conflicts with the other 63 into one 64-bit word,
-// and the greedy decision inside the batch is then 64 steps of register arithmetic.  The rows of the
-// newly kept candidates are OR-ed into the running `blocked` mask by the whole CTA.
+// The walk is a serial chain (whether candidate i is kept depends on every earlier decision).  One CTA
+// takes the list 64 positions at a time.  For such a range the candidates not blocked so far are two words
+// of the running `blocked` mask, and the conflicts of a member with the other 63 are two words of its
+// conflict row (the range is 64-aligned): nothing is searched or compacted.  One warp settles the range in a
+// few passes of warp-wide ORs (see below) instead of 64 dependent steps, and the rows of the newly kept
+// candidates are then OR-ed into `blocked` for the ranges still to come by the whole CTA.
+// The conflict rows are read from shared memory: all of them are brought in once when they fit (a
+// candidate window does), otherwise the rows of the range's unblocked members are fetched per range.
 #include "strads_internal.cuh"
 
 namespace strads {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kBatch = 64;          // candidates decided per batch (two per lane of the deciding warp)
+constexpr int kRange = 64;                       // positions decided per step of the walk
+constexpr size_t kResidentBytes = 200 * 1024;    // conflict rows of the whole list in shared memory up to this
 
-// Position of the n-th (0-based) set bit of x; popc(x) > n.
-__device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
-  int at = 0;
-#pragma unroll
-  for (int s = 16; s > 0; s >>= 1) {
-    const int c = __popc(x & ((1u << s) - 1u));
-    if (n >= c) { n -= c; x >>= s; at += s; }
-  }
-  return at;
-}
+__host__ __device__ inline int words_of(int n_cand) { return (n_cand + 31) >> 5; }
+__host__ __device__ inline int pitch_of(int n_cand) { return words_of(n_cand) | 1; }      // odd: rows start in different banks
+__host__ __device__ inline int cand_offset(int n_cand) { return (words_of(n_cand) + 2 + 3) & ~3; }   // after blocked[Wn + 2]
+__host__ __device__ inline int rows_offset(int n_cand) { return cand_offset(n_cand) + ((n_cand + 3) & ~3); }   // after s_cand[n_cand]
 
 // n_cand < n_total: the list is only a leading window of the candidates.  If P are kept inside it the result
 // is final (the walk never looks further); otherwise window_short is raised and the caller's retry over
 // the whole list (launched with only_if_short) replaces the result.
 __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
-                                                      int only_if_short, int* __restrict__ kept_out) {
+                                                      int only_if_short, int resident, int* __restrict__ kept_out) {
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
   if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
@@ -45,22 +41,17 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     return;
   }
   extern __shared__ unsigned int sm[];
-  const int W = p.mask_words;
-  const int Ws = W | 1;                          // odd row pitch: column reads of `rows` hit 32 different banks
-  unsigned int* blocked = sm;                    // [W]
-  unsigned int* rows = sm + W;                   // [kBatch][Ws]
-  __shared__ int pos[kBatch];                    // positions (in the candidate list) of the batch
-  __shared__ int cval[kBatch];                   // cand[pos[.]]
-  __shared__ int s_m, s_cursor, s_kept, s_examined, s_done;
-  __shared__ unsigned long long s_conf[kBatch];  // per batch member: conflicts with later members
-  __shared__ int s_krow[kBatch], s_kfirst[kBatch], s_nnew;   // newly kept: row offset in `rows`, first valid word
-  const int tid = threadIdx.x, lane = tid & 31;
-  int G = 1;                                     // threads per mask word in step 4 (a power of two, G * W <= kThreads)
-  while (G < 32 && 2 * G * W <= kThreads) G <<= 1;
+  const int W = p.mask_words;                    // pitch of the conflict rows in global memory
+  const int Wn = words_of(n_cand), Wp = pitch_of(n_cand);
+  unsigned int* blocked = sm;                    // [Wn + 2] (two words of slack: a range always reads a pair)
+  int* s_cand = reinterpret_cast<int*>(sm + cand_offset(n_cand));   // [n_cand] copy of the list
+  unsigned int* rows = sm + rows_offset(n_cand); // resident: [n_cand][Wp]; else the range in flight, [kRange][Wp]
+  __shared__ unsigned long long s_keep;          // members of the range in flight that were kept
+  __shared__ int s_kept, s_examined, s_done;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
-  if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = 0; s_done = 0; }
-  __syncthreads();
+  for (int w = tid; w < Wn + 2; w += kThreads) blocked[w] = 0u;
+  if (tid == 0) { s_kept = 0; s_examined = n_cand; s_done = 0; }
 
   if (p.flags & STRADS_FLAG_NO_FILTER) {
     const int nk = min(n_cand, p.n_keep);
@@ -68,164 +59,158 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; p.st->window_short = 0; }
     return;
   }
+  for (int i = tid; i < n_cand; i += kThreads) s_cand[i] = cand[i];
+  if (resident) {
+    // all rows at once: independent loads, eight in flight per thread, before any store
+    const int total = n_cand * Wn;
+    for (int i0 = tid; i0 < total; i0 += 8 * kThreads) {
+      unsigned int v[8];
+      int at[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        const int i = min(i0 + u * kThreads, total - 1);
+        const int r = i / Wn, w = i - r * Wn;
+        at[u] = r * Wp + w;
+        v[u] = __ldcg(p.conflict + (long long)r * W + w);
+      }
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (i0 + u * kThreads < total) rows[at[u]] = v[u];
+    }
+  }
+  __syncthreads();
 
-  while (true) {
-    // 1. the next <= kBatch candidates at or after the cursor that are not blocked yet (warp 0)
+  for (int cur = 0; cur < n_cand; cur += kRange) {
+    const int m = min(kRange, n_cand - cur);
+    const int w0 = cur >> 5;                           // even: the range is words w0, w0 + 1 of every mask
+    const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
+    const unsigned long long alive0 = ~(((unsigned long long)blocked[w0 + 1] << 32) | blocked[w0]) & valid;
+    if (alive0 == 0ull) continue;                      // (uniform) everything here is blocked already
+    if (!resident) {
+      // rows of the unblocked members, words w0 .. Wn - 1 (earlier words are never looked at again).  One CTA
+      // has few loads in flight, so they are 128-bit where the row pitch allows: a task is four consecutive
+      // words of one member's row, sixteen tasks in flight per thread, loads before stores.
+      if ((W & 3) == 0) {
+        // thread -> member tid / 4 and every fourth 128-bit group of its row from tid % 4 on (four lanes read 64
+        // consecutive bytes)
+        const int q = tid >> 2, v0 = w0 >> 2, vend = (Wn + 3) >> 2;                  // (W % 4 == 0: 4 * vend <= W)
+        const bool on = (alive0 >> q) & 1ull;
+        const uint4* src = reinterpret_cast<const uint4*>(p.conflict + (long long)(cur + q) * W);
+        unsigned int* dst = rows + q * Wp;
+        for (int c0 = v0 + (tid & 3); c0 < vend; c0 += 4 * 16) {
+          uint4 v[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const int c = c0 + 4 * u;
+            v[u] = make_uint4(0u, 0u, 0u, 0u);
+            if (on && c < vend) v[u] = __ldcg(src + c);
+          }
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const int c = c0 + 4 * u;
+            if (c < vend) {
+              dst[4 * c] = v[u].x;
+              if (4 * c + 1 < Wn) dst[4 * c + 1] = v[u].y;
+              if (4 * c + 2 < Wn) dst[4 * c + 2] = v[u].z;
+              if (4 * c + 3 < Wn) dst[4 * c + 3] = v[u].w;
+            }
+          }
+        }
+      } else {
+        const int chunks = (Wn - w0 + 31) >> 5, tasks = kRange * chunks;
+        for (int t0 = warp; t0 < tasks; t0 += 16 * (kThreads / 32)) {
+          unsigned int v[16];
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const int task = t0 + u * (kThreads / 32);
+            const int q = task & (kRange - 1), wd = w0 + ((task >> 6) << 5) + lane;
+            v[u] = (task < tasks && wd < Wn && ((alive0 >> q) & 1ull)) ? __ldcg(p.conflict + (long long)(cur + q) * W + wd) : 0u;
+          }
+#pragma unroll
+          for (int u = 0; u < 16; ++u) {
+            const int task = t0 + u * (kThreads / 32);
+            const int q = task & (kRange - 1), wd = w0 + ((task >> 6) << 5) + lane;
+            if (task < tasks && wd < Wn) rows[q * Wp + wd] = v[u];
+          }
+        }
+      }
+      __syncthreads();
+    }
+    // The greedy decision inside the range, by warp 0; lane l holds members l and l + 32 with their conflicts
+    // with LATER members (all the Gram kernels guarantee).  Instead of 64 dependent steps it settles the range in
+    // passes: members hit by a member kept in the last pass are out; a member that no earlier undecided member
+    // conflicts with is kept (all its earlier neighbours are out).  The first undecided member is always kept, so
+    // the passes end; with few conflicts two or three do.  Same set as the one-by-one walk.
     if (tid < 32) {
-      int m = 0;
-      int cur = s_cursor;
-      while (cur < n_cand && m < kBatch) {
-        const int wbase = (cur >> 5) + lane;           // 32 mask words at a time, one per lane
-        unsigned int freew = 0u;
-        if (wbase < W) {
-          freew = ~blocked[wbase];
-          const int first = wbase << 5;
-          if (first < cur) freew &= 0xffffffffu << (cur - first);                         // only lane 0 can be cut
-          if (first + 32 > n_cand) freew &= first >= n_cand ? 0u : (0xffffffffu >> (first + 32 - n_cand));
+      const unsigned int full = 0xffffffffu;
+      const int base = resident ? cur * Wp + w0 : w0;
+      const int cva = lane < m ? s_cand[cur + lane] : -1;
+      const int cvb = lane + 32 < m ? s_cand[cur + lane + 32] : -1;
+      const int ata = base + min(lane, m - 1) * Wp, atb = base + min(lane + 32, m - 1) * Wp;
+      const unsigned int later = lane == 31 ? 0u : (full << (lane + 1));
+      const unsigned int a_lo = rows[ata] & later, a_hi = rows[ata + 1], b_hi = rows[atb + 1] & later;
+      unsigned int und_lo = (unsigned int)alive0, und_hi = (unsigned int)(alive0 >> 32);
+      unsigned int keep_lo = 0u, keep_hi = 0u, new_lo = 0u, new_hi = 0u;
+      for (int pass = 0; pass < kRange && (und_lo | und_hi) != 0u; ++pass) {
+        if (pass > 0) {
+          const bool ka = (new_lo >> lane) & 1u, kb = (new_hi >> lane) & 1u;
+          und_lo &= ~__reduce_or_sync(full, ka ? a_lo : 0u);
+          und_hi &= ~__reduce_or_sync(full, (ka ? a_hi : 0u) | (kb ? b_hi : 0u));
         }
-        const int cnt = __popc(freew);
-        int incl = cnt;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += v;
-        }
-        const int total = __shfl_sync(0xffffffffu, incl, 31);
-        // slot s of the batch takes the (s - m)-th free position of these 32 words: lane s (and s + 32) finds
-        // the word that holds it from the prefix counts, then the bit inside the word
-        const int excl = incl - cnt;
-#pragma unroll
-        for (int half = 0; half < kBatch / 32; ++half) {
-          const int slot = lane + 32 * half;
-          const int want = slot - m;                   // rank among the free positions found in this sweep
-          int wi = 0;                                  // first lane whose inclusive count exceeds `want`
-#pragma unroll
-          for (int step = 16; step > 0; step >>= 1)
-            if (__shfl_sync(0xffffffffu, incl, wi + step - 1) <= want) wi += step;
-          wi = min(wi, 31);
-          const int ex = __shfl_sync(0xffffffffu, excl, wi);
-          const unsigned int word = __shfl_sync(0xffffffffu, freew, wi);
-          if (want >= 0 && want < total && slot < kBatch)
-            pos[slot] = (((cur >> 5) + wi) << 5) + nth_set_bit(word, want - ex);
-        }
-        m = min(kBatch, m + total);
-        if (m < kBatch) cur = ((cur >> 5) + 32) << 5;  // all 32 words consumed
+        const bool ua = (und_lo >> lane) & 1u, ub = (und_hi >> lane) & 1u;
+        const unsigned int thr_lo = __reduce_or_sync(full, ua ? a_lo : 0u);
+        const unsigned int thr_hi = __reduce_or_sync(full, (ua ? a_hi : 0u) | (ub ? b_hi : 0u));
+        new_lo = und_lo & ~thr_lo; new_hi = und_hi & ~thr_hi;
+        keep_lo |= new_lo; keep_hi |= new_hi;
+        und_lo &= ~new_lo; und_hi &= ~new_hi;
       }
-      if (lane == 0) s_m = m;
-    }
-    __syncthreads();
-    const int m = s_m;
-    if (m == 0) {                                      // list exhausted
-      if (tid == 0) s_examined = n_cand;
-      break;
-    }
-    // 2. fetch their conflict rows (and their coefficient indices) together.  Loads first, stores after:
-    //    a store to `rows` between two loads would order them and cost one memory round trip per word.
-    if (tid < m) cval[tid] = cand[pos[tid]];         // (kBatch <= kThreads)
-    {
-      const int warp = tid >> 5;                       // warp w fetches rows w, w + 8, ..., w + 56
-      const unsigned int* src[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) src[u] = p.conflict + (long long)pos[min(warp + 8 * u, m - 1)] * W;
-      for (int w0 = lane; w0 < W; w0 += 32) {
-        unsigned int v[8];
-#pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = __ldcg(src[u] + w0);
-#pragma unroll
-        for (int u = 0; u < 8; ++u) {
-          const int r = warp + 8 * u;
-          if (r < m) rows[r * Ws + w0] = v[u];
-        }
-      }
-    }
-    __syncthreads();
-    // 3a. the conflicts of batch member q with the LATER members, as a 64-bit word: four threads per member,
-    //     16 of the 64 bits each (a row is valid from its own word on; fixed trip count so that the reads overlap)
-    {
-      static_assert(kThreads == 4 * kBatch, "four threads per batch member");
-      const int q = tid >> 2, part = tid & 3;
-      const int my_row = min(q, m - 1) * Ws;
-      unsigned int bits = 0u;
-#pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const int pb = pos[min(part * 16 + i, m - 1)];
-        bits |= ((rows[my_row + (pb >> 5)] >> (pb & 31)) & 1u) << i;
-      }
-      unsigned long long mine = (unsigned long long)bits << (16 * part);
-      mine |= __shfl_xor_sync(0xffffffffu, mine, 1);
-      mine |= __shfl_xor_sync(0xffffffffu, mine, 2);
-      const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
-      const unsigned long long later = q >= 63 ? 0ull : ~((2ull << q) - 1ull);
-      if (part == 0) s_conf[q] = q < m ? (mine & valid & later) : 0ull;
-    }
-    __syncthreads();
-    // 3b. the greedy decision inside the batch: 64 steps of register arithmetic (warp 0; every lane computes the same)
-    if (tid < 32) {
-      const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
-      unsigned long long alive = valid, keep = 0ull;
-      unsigned long long cq[kBatch];                   // all 64 words into registers first: the loads do not depend
-#pragma unroll                                         // on the chain below and overlap
-      for (int q = 0; q < kBatch; ++q) cq[q] = s_conf[q];
-#pragma unroll
-      for (int q = 0; q < kBatch; ++q)
-        if ((alive >> q) & 1ull) { keep |= 1ull << q; alive &= ~cq[q]; }
+      unsigned long long keep = ((unsigned long long)keep_hi << 32) | keep_lo;
       const int nk = s_kept;
       const int room = p.n_keep - nk;
-      bool full = false;
+      bool full_now = false;
       if (__popcll(keep) >= room) {                    // stop exactly at P: drop the surplus from the back
         while (__popcll(keep) > room) keep &= ~(1ull << (63 - __clzll(keep)));
-        full = true;
+        full_now = true;
       }
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         const int q = lane + 32 * half;
         if ((keep >> q) & 1ull) {
-          const int slot = nk + __popcll(keep & ((1ull << q) - 1ull));
-          kept_out[slot] = cval[q];
-          p.kept_pos[slot] = pos[q];
-        }
-      }
-#pragma unroll
-      for (int half = 0; half < 2; ++half) {           // compact list of the newly kept rows for step 4
-        const int q = lane + 32 * half;
-        if ((keep >> q) & 1ull) {
           const int r = __popcll(keep & ((1ull << q) - 1ull));
-          s_krow[r] = q * Ws;
-          s_kfirst[r] = pos[q] >> 5;
+          kept_out[nk + r] = half ? cvb : cva;
+          p.kept_pos[nk + r] = cur + q;
         }
       }
       if (lane == 0) {
-        s_nnew = __popcll(keep);
+        s_keep = keep;
         s_kept = nk + __popcll(keep);
-        if (full) { s_examined = pos[63 - __clzll(keep)] + 1; s_done = 1; }
-        else s_cursor = pos[m - 1] + 1;
+        if (full_now) { s_examined = cur + (63 - __clzll(keep)) + 1; s_done = 1; }
       }
     }
     __syncthreads();
     if (s_done) break;
-    // 4. OR the rows of the newly kept candidates into the mask (a row is valid from its own word on).
-    //    G threads per mask word share the rows between them (all loads unconditional and independent),
-    //    then combine with shuffles.
-    const int n_new = s_nnew;
-    for (int base = 0; base < W; base += kThreads / G) {
-      const int w = base + tid / G, sub = tid % G;
-      unsigned int acc = 0u;
-      if (w < W) {
-        for (int r0 = sub; r0 < n_new; r0 += 8 * G) {
-          int kf[8];
-          unsigned int v[8];
+    // OR the rows of the newly kept candidates into the mask of the ranges still to come.  A lane per mask
+    // word (32 consecutive words per trip), warp k takes the members k, k + 8, ... of the range: no reduction
+    // across lanes, eight independent reads per trip, and one shared-memory atomic OR per word and warp.
+    {
+      const unsigned long long keep = s_keep;
+      int kr[kRange / 8];
+      bool any = false;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = min(r0 + i * G, n_new - 1);  // past the end: the last row again (harmless)
-            kf[i] = s_kfirst[r];
-            v[i] = rows[s_krow[r] + w];
-          }
+      for (int u = 0; u < kRange / 8; ++u) {
+        const int q = warp + 8 * u;
+        const bool k = (keep >> q) & 1ull;
+        kr[u] = k ? (resident ? cur + q : q) * Wp : -1;
+        any |= k;
+      }
+      if (any) {
+        for (int w = w0 + 2 + lane; w < Wn; w += 32) {
+          unsigned int acc = 0u;
 #pragma unroll
-          for (int i = 0; i < 8; ++i) acc |= w >= kf[i] ? v[i] : 0u;
+          for (int u = 0; u < kRange / 8; ++u) acc |= kr[u] >= 0 ? rows[kr[u] + w] : 0u;
+          if (acc != 0u) atomicOr(&blocked[w], acc);
         }
       }
-      for (int o = G >> 1; o > 0; o >>= 1) acc |= __shfl_xor_sync(0xffffffffu, acc, o);
-      if (w < W && sub == 0) blocked[w] |= acc;
     }
     __syncthreads();
   }
@@ -241,20 +226,27 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
 
 }  // namespace
 
-size_t filter_smem_bytes(const Problem& p) {
-  return ((size_t)p.mask_words + (size_t)kBatch * (p.mask_words | 1)) * sizeof(unsigned int);
+static size_t filter_smem_bytes(int n_cand, bool* resident) {
+  // + 4 words: the pair of words a range reads from the last row may reach one word past it (odd word count)
+  const size_t all = ((size_t)rows_offset(n_cand) + (size_t)n_cand * pitch_of(n_cand) + 4) * sizeof(unsigned int);
+  *resident = all <= kResidentBytes;
+  return *resident ? all : ((size_t)rows_offset(n_cand) + (size_t)kRange * pitch_of(n_cand) + 4) * sizeof(unsigned int);
 }
 
 // Kernel-wide attribute: the largest size any handle can need (see prepare_sample).
 cudaError_t prepare_filter(const Problem&) {
-  constexpr int kMaxWords = STRADS_MAX_CANDIDATES / 32;
-  return cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                              (int)((kMaxWords + kBatch * (kMaxWords | 1)) * sizeof(unsigned int)));
+  bool r;
+  size_t most = filter_smem_bytes(STRADS_MAX_CANDIDATES, &r);
+  if (most < kResidentBytes) most = kResidentBytes;
+  return cudaFuncSetAttribute(k_filter, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)most);
 }
 
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s) {
-  return launch_chained(k_filter, 1, kThreads, filter_smem_bytes(p), s, p, cand, n_cand, n_total, only_if_short ? 1 : 0, kept_out);
+  bool resident;
+  const size_t smem = filter_smem_bytes(n_cand, &resident);
+  return launch_chained(k_filter, 1, kThreads, smem, s, p, cand, n_cand, n_total, only_if_short ? 1 : 0, resident ? 1 : 0,
+                        kept_out);
 }
 
 }  // namespace strads
