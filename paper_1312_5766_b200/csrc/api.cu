@@ -91,6 +91,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.cap_sure = c->n_candidates;
   L.cap_boundary = pow2_ceil(c->n_candidates / 2 > 2048 ? c->n_candidates / 2 : 2048);
   L.mask_words = (c->n_candidates + 31) / 32;
+  // CTAs per kept column in the dot kernel: about 1024 CTAs in all, so that every one of them is resident at
+  // once (the kernel is a chain of dependent loads per CTA; residency, not depth per thread, hides it)
   long long parts = (1024 + c->n_keep - 1) / c->n_keep;
   const long long max_parts = c->n_rows / 2048 > 1 ? c->n_rows / 2048 : 1;
   if (parts > max_parts) parts = max_parts;

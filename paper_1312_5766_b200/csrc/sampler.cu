@@ -12,7 +12,8 @@
 //                    expectation whatever the weights are; if it ever exceeds the boundary buffer,
 //                    that CTA alone refines the boundary over further 12-bit digits (rare, exact).
 //   k_sample_collect pass 2: appends "sure" and "boundary" keys to two small buffers.
-//   k_sample_sort_chunks / k_sample_rank   order the winners: 1024-key chunks sorted in shared memory by
+//   k_sample_rank_direct (P' <= 2048)  orders the winners by counting, for every key, the smaller ones.
+//   k_sample_sort_chunks / k_sample_rank (larger P')  1024-key chunks sorted in shared memory by
 //                    one CTA each, then every key's rank by binary search in the other chunks.
 #include <cstddef>
 #include <mutex>
@@ -272,6 +273,39 @@ __global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
   if (i1 < ch.n && r1 < p.n_cand) cand_out[r1] = (int)(k1 & 0xffffffffull);
 }
 
+// Small P': the order of the winners straight from the definition, with no sort.  The rank of a key is the
+// number of smaller keys in its buffer (+ n_sure for boundary keys: every sure key is smaller); the key of
+// rank r < P' is candidate r.  A CTA takes 32 keys of one buffer, stages the whole buffer (<= 2048 keys) in
+// shared memory and counts with eight threads per key, each over an eighth of the buffer.
+constexpr int kDirectMax = 2048;         // P' and the boundary buffer up to this many keys (beyond, sorting wins)
+constexpr int kDirectKeys = 32;          // keys per CTA
+__global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand_out) {
+  chain_begin();
+  __shared__ unsigned long long all[kDirectMax];
+  const SelectState sel = p.st->sel;
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
+  const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
+  const int sure_ctas = (p.cap_sure + kDirectKeys - 1) / kDirectKeys;
+  const bool is_sure = (int)blockIdx.x < sure_ctas;
+  const int first = (is_sure ? blockIdx.x : blockIdx.x - sure_ctas) * kDirectKeys;
+  const int total = is_sure ? n_sure : n_bnd;
+  if (first >= total) return;
+  const unsigned long long* buf = is_sure ? p.sure : p.boundary;
+  for (int i = threadIdx.x; i < total; i += 256) all[i] = __ldcg(buf + i);
+  __syncthreads();
+  const int k = first + (threadIdx.x >> 3), slice = threadIdx.x & 7;
+  const unsigned long long key = k < total ? all[k] : 0ull;
+  const int per = (total + 7) >> 3, i0 = slice * per, i1 = min(total, i0 + per);
+  int below = 0;
+#pragma unroll 8
+  for (int i = i0; i < i1; ++i) below += all[i] < key;
+  below += __shfl_xor_sync(0xffffffffu, below, 1);
+  below += __shfl_xor_sync(0xffffffffu, below, 2);
+  below += __shfl_xor_sync(0xffffffffu, below, 4);
+  const int rank = below + (is_sure ? 0 : n_sure);
+  if (slice == 0 && k < total && rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
+}
+
 }  // namespace
 
 cudaError_t prepare_sample(const Problem&) { return cudaSuccess; }
@@ -285,6 +319,10 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   cudaError_t e;
   if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
+  if (p.cap_sure <= kDirectMax && p.cap_boundary <= kDirectMax) {
+    const int ctas = (p.cap_sure + kDirectKeys - 1) / kDirectKeys + (p.cap_boundary + kDirectKeys - 1) / kDirectKeys;
+    return launch_chained(k_sample_rank_direct, ctas, 256, 0, s, p, cand_out);
+  }
   const int chunks = (p.cap_sure + kChunk - 1) / kChunk + (p.cap_boundary + kChunk - 1) / kChunk;
   if ((e = launch_chained(k_sample_sort_chunks, chunks, 512, 0, s, p)) != cudaSuccess) return e;
   return launch_chained(k_sample_rank, chunks, 512, 0, s, p, cand_out);
