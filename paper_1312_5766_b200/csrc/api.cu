@@ -62,8 +62,9 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl, total;
-  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles;
+      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
+      off_bucket_count, off_bucket_items, off_pairs, total;
+  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap;
   long long ldc;
 };
 
@@ -123,6 +124,12 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
   L.off_walk_rows = take(csc ? sizeof(unsigned int) * 32 * (size_t)L.mask_words : 0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
+  // CSC Gram by row buckets: provided for while the buckets stay below 64 MB (N <= 2^20)
+  const bool buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);
+  L.pair_cap = buckets ? (1 << 20) : 0;
+  L.off_bucket_count = take(buckets ? sizeof(unsigned int) * (size_t)c->n_rows : 0);
+  L.off_bucket_items = take(buckets ? sizeof(int) * (size_t)c->n_rows * kBucketSlots : 0);
+  L.off_pairs = take(sizeof(unsigned int) * (size_t)L.pair_cap);
   L.total = o;
   return L;
 }
@@ -269,6 +276,10 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
   p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
   p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
+  p.pair_cap = L.pair_cap;
+  p.bucket_count = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
+  p.bucket_items = L.pair_cap ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;
+  p.pair_list = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_pairs) : nullptr;
   p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
   p.partial_tiles = L.partial_tiles;
   p.part_count = S; p.part_index = s;
@@ -348,6 +359,9 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
     if (sc.p.layout == STRADS_CSC) {
       if ((e = prepare_walk_csc(sc.p, &sc.walk_grid)) != cudaSuccess) return fail(cuda_fail(e, "prepare_walk_csc"));
       if ((e = cudaMemsetAsync(sc.p.walk_ctl, 0, sizeof(WalkControl), h->stream)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaMemsetAsync"));
+      if (sc.p.bucket_count != nullptr &&
+          (e = cudaMemsetAsync(sc.p.bucket_count, 0, sizeof(unsigned int) * (size_t)sc.p.N, h->stream)) != cudaSuccess)
         return fail(cuda_fail(e, "cudaMemsetAsync"));
     }
     if (s > 0 && (e = launch_init_scheduler(sc.p, p0, h->stream)) != cudaSuccess)

@@ -32,6 +32,10 @@ struct DeviceState {
   unsigned int amb_count;       // pairs the TF32 screen of the dense Gram left to the exact recheck
   int window_short;             // the filter ran out of its candidate window before P were kept: redo on all P'
   int prefer_walk;              // CSC: the last round needed the whole list, so skip the window attempt for a while
+  unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
+  int bucket_failed;            // ... a bucket or the pair list overflowed this round: the all-pairs kernel redoes the bits
+  int bucket_avoid;             // ... it overflowed lately: go straight to the all-pairs kernel for a while
+  int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int pad;
 };
 
@@ -43,6 +47,7 @@ struct WalkControl {            // shared by the CTAs of the cooperative on-dema
   int cval[32];                 // their coefficient indices
 };
 
+static constexpr int kBucketSlots = 16;   // candidates per row bucket (more: the round falls back to all pairs)
 static constexpr int kHistBits = 12;
 static constexpr int kHistBins = 1 << kHistBits;
 
@@ -89,6 +94,11 @@ struct Problem {
   unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words]
   unsigned int* walk_rows;      // [32][mask_words] conflict rows of the batch in flight
   WalkControl* walk_ctl;
+  // CSC Gram by row buckets (null / 0 when not provided for)
+  unsigned int* bucket_count;   // [N] candidates of this round's list with an entry in row i (zero between rounds)
+  int* bucket_items;            // [N][kBucketSlots] their positions in the list
+  unsigned int* pair_list;      // [pair_cap] (a << 16 | b), a < b: positions of two candidates that share a row
+  int pair_cap;
   int sm_count;
   // scheduler threads: this Problem is scheduler part_index of part_count and owns { j : j mod part_count == part_index }
   int part_count, part_index;
