@@ -122,7 +122,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
-  L.off_walk_rows = take(csc ? sizeof(unsigned int) * 32 * (size_t)L.mask_words : 0);
+  L.off_walk_rows = take(0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
   // CSC Gram by row buckets: provided for while the buckets stay below 64 MB (N <= 2^20)
   const bool buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);

@@ -41,10 +41,8 @@ struct DeviceState {
 
 struct WalkControl {            // shared by the CTAs of the cooperative on-demand walk (CSC)
   unsigned int bar_count, bar_gen;   // grid barrier
-  int m;                        // batch size (0: list exhausted)
-  int cursor, n_kept, examined, done, failed;
-  int pos[32];                  // positions of the batch in the candidate list
-  int cval[32];                 // their coefficient indices
+  int failed;
+  int pad;
 };
 
 static constexpr int kBucketSlots = 16;   // candidates per row bucket (more: the round falls back to all pairs)
@@ -91,8 +89,8 @@ struct Problem {
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
   float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
   int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles
-  unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words]
-  unsigned int* walk_rows;      // [32][mask_words] conflict rows of the batch in flight
+  unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words], OR-ed into by the whole grid
+  unsigned int* walk_rows;      // (unused)
   WalkControl* walk_ctl;
   // CSC Gram by row buckets (null / 0 when not provided for)
   unsigned int* bucket_count;   // [N] candidates of this round's list with an entry in row i (zero between rounds)
@@ -191,6 +189,73 @@ __device__ __forceinline__ float sparse_dot(const int* ar, const float* av, int 
       } else {
         if (++q >= qe) break;
         rb = __ldg(p.xrow + q);
+      }
+    }
+  }
+  return dot;
+}
+
+// The same sum with both columns given as arrays (shared or global memory).
+__device__ __forceinline__ float sparse_dot_arrays(const int* ar, const float* av, int na, const int* br, const float* bv,
+                                                   int nb) {
+  float dot = 0.f;
+  int i = 0, k = 0;
+  if (na > 0 && nb > 0) {
+    int ra = ar[0], rb = br[0];
+    while (true) {
+      if (ra == rb) {
+        dot = fmaf(av[i], bv[k], dot);
+        if (++i >= na || ++k >= nb) break;
+        ra = ar[i]; rb = br[k];
+      } else if (ra < rb) {
+        if (++i >= na) break;
+        ra = ar[i];
+      } else {
+        if (++k >= nb) break;
+        rb = br[k];
+      }
+    }
+  }
+  return dot;
+}
+
+// The same sum again, for a lane that merges alone: the first kPre row indices of column b are fetched together
+// (one memory round trip instead of one per step); values are read only where the rows match.
+template <int kPre>
+__device__ __forceinline__ float sparse_dot_prefetched(const int* ar, const float* av, int na, const Problem& p, int jb) {
+  const long long q0 = p.xptr[jb];
+  const int nb = (int)(p.xptr[jb + 1] - q0);
+  int rb[kPre];
+#pragma unroll
+  for (int k = 0; k < kPre; ++k) rb[k] = k < nb ? __ldg(p.xrow + q0 + k) : 0x7fffffff;
+  float dot = 0.f;
+  int i = 0;
+  int ra = na > 0 ? ar[0] : 0x7fffffff;
+#pragma unroll
+  for (int k = 0; k < kPre; ++k) {
+    if (k < nb && i < na) {
+      while (ra < rb[k]) {
+        if (++i >= na) { ra = 0x7fffffff; break; }
+        ra = ar[i];
+      }
+      if (i < na && ra == rb[k]) dot = fmaf(av[i], __ldg(p.xv + q0 + k), dot);
+    }
+  }
+  if (nb > kPre && i < na) {                            // the rest of a long column, step by step
+    long long q = q0 + kPre;
+    const long long qe = q0 + nb;
+    int r2 = __ldg(p.xrow + q);
+    while (true) {
+      if (ra == r2) {
+        dot = fmaf(av[i], __ldg(p.xv + q), dot);
+        if (++i >= na || ++q >= qe) break;
+        ra = ar[i]; r2 = __ldg(p.xrow + q);
+      } else if (ra < r2) {
+        if (++i >= na) break;
+        ra = ar[i];
+      } else {
+        if (++q >= qe) break;
+        r2 = __ldg(p.xrow + q);
       }
     }
   }

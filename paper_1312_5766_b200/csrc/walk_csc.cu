@@ -1,19 +1,24 @@
 // SAP step 2, CSC X, when the walk needs the whole candidate list: greedy first-fit that forms conflict
-// rows ON DEMAND.  Only the row of a candidate that is about to be kept is ever needed (it tells which
-// later candidates it blocks), so with heavy rejection -- skewed rows make most pairs of columns overlap,
-// a few dozen candidates are kept out of 16,384 -- forming all P'(P'-1)/2 correlations first would do
-// 100x more merges than the walk consults.
+// rows ON DEMAND.  Only the row of a candidate that is kept is ever needed (it tells which later candidates
+// it blocks), so with heavy rejection -- skewed rows make most pairs of columns overlap, a few dozen
+// candidates are kept out of 16,384 -- forming all P'(P'-1)/2 correlations first would do 100x more merges
+// than the walk consults.
 //
-// One cooperative kernel, a few CTAs per SM, in batches of 32 like k_filter:
-//   A  CTA 0 picks the next 32 candidates that are not blocked yet;
-//   B  all CTAs compute those 32 conflict rows (a row: the candidate's column, staged in shared memory,
-//      merged against every later candidate's column; one lane per pair, one ballot per mask word);
-//   C  CTA 0 decides the batch in order with register arithmetic and ORs the rows of the newly kept
-//      candidates into the running mask;
-// with a grid-wide barrier between the phases.  The barrier is a counter + generation word in global
-// memory; every spin has an iteration limit, after which the CTA raises STRADS_STATUS_WAIT_EXPIRED
+// One cooperative kernel, two CTAs per SM, in batches of 32 candidates.  Every CTA holds the running
+// `blocked` mask in shared memory and does the cheap, serial part of a batch itself, identically to all the
+// others, so that nothing has to be broadcast:
+//   A  pick the next 32 candidates that are not blocked yet;
+//   B  stage their columns in shared memory and merge the <= 496 pairs among them;
+//   C  decide the batch (who is kept) from those in-batch conflicts;
+// then the expensive part is shared out over the grid:
+//   D  for every candidate just kept, merge its column against all later unblocked candidates (a warp per
+//      32 of them, a lane per pair) and OR the resulting conflict words into the mask in global memory
+//      (integer OR: any order gives the same mask);
+// one grid-wide barrier, and every CTA reloads the mask.  The barrier is a counter + generation word in
+// global memory; every spin has an iteration limit, after which the CTA raises STRADS_STATUS_WAIT_EXPIRED
 // and leaves (the launch is cooperative, so all CTAs are resident and the limit is never met in practice).
-// The kept list equals that of the full-Gram walk: same correlations (sparse_dot), same order.
+// The kept list equals that of the full-Gram walk: same correlations (same order of the same products),
+// same order of decisions.
 #include "strads_internal.cuh"
 
 namespace strads {
@@ -21,8 +26,20 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kBatch = 32;
-constexpr int kStage = 1024;          // entries of a column staged in shared memory (longer columns: global)
+constexpr int kColCap = 64;           // entries of a batch member's column staged in shared memory (longer: global)
+constexpr int kMaxWords = STRADS_MAX_CANDIDATES / 32;
 constexpr unsigned int kSpinLimit = 1u << 26;
+
+// Position of the n-th (0-based) set bit of x; popc(x) > n.
+__device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
+  int at = 0;
+#pragma unroll
+  for (int s = 16; s > 0; s >>= 1) {
+    const int c = __popc(x & ((1u << s) - 1u));
+    if (n >= c) { n -= c; x >>= s; at += s; }
+  }
+  return at;
+}
 
 // Grid-wide barrier.  Returns false when the wait gave up (or an earlier one did).
 __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* status) {
@@ -53,162 +70,172 @@ __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* 
 __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __restrict__ cand, int n_cand,
                                                         int only_if_short, int* __restrict__ kept_out) {
   if (only_if_short && !p.st->window_short) return;      // uniform over the grid: nobody reaches a barrier
-  __shared__ int arow[kStage];
-  __shared__ float aval[kStage];
-  __shared__ int s_pos[kBatch];
+  __shared__ unsigned int blocked[kMaxWords];
+  __shared__ int brow[kBatch][kColCap];
+  __shared__ float bval[kBatch][kColCap];
+  __shared__ int s_pos[kBatch], s_col[kBatch], s_len[kBatch];
+  __shared__ long long s_ptr[kBatch];
+  __shared__ double s_n2[kBatch];
+  __shared__ unsigned int s_conf[kBatch];
   __shared__ unsigned int s_keep;
+  __shared__ int s_m, s_cursor, s_kept, s_examined, s_done;
   WalkControl* c = p.walk_ctl;
-  const int W = p.mask_words;
+  const int W = (n_cand + 31) >> 5;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const unsigned int n_ctas = gridDim.x;
-  unsigned int* blocked = p.walk_blocked;
-  unsigned int* rows = p.walk_rows;
+  const unsigned int full = 0xffffffffu;
+  unsigned int* blocked_g = p.walk_blocked;
   const double rho = (double)p.rho;
 
-  if (blockIdx.x == 0) {
-    for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
-    if (tid == 0) { c->m = 0; c->cursor = 0; c->n_kept = 0; c->examined = 0; c->done = 0; }
-  }
-  bool ok = grid_barrier(c, n_ctas, &p.st->status);
+  for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
+  if (blockIdx.x == 0)
+    for (int w = tid; w < W; w += kThreads) blocked_g[w] = 0u;
+  if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = n_cand; s_done = 0; }
+  bool ok = grid_barrier(c, n_ctas, &p.st->status);       // nobody ORs into the global mask before it is cleared
 
   while (ok) {
-    // ---- A: CTA 0, warp 0: the next <= 32 candidates at or after the cursor that are not blocked ----
-    if (blockIdx.x == 0 && tid < 32) {
+    // ---- A: the next <= 32 candidates at or after the cursor that are not blocked (warp 0) ----
+    if (tid < 32) {
       int m = 0;
-      int cur = c->cursor;
+      int cur = s_cursor;
       while (cur < n_cand && m < kBatch) {
-        const int wbase = (cur >> 5) + lane;
+        const int wbase = (cur >> 5) + lane;           // 32 mask words at a time, one per lane
         unsigned int freew = 0u;
         if (wbase < W) {
-          freew = ~__ldcg(&blocked[wbase]);
+          freew = ~blocked[wbase];
           const int first = wbase << 5;
-          if (first < cur) freew &= 0xffffffffu << (cur - first);
-          if (first + 32 > n_cand) freew &= first >= n_cand ? 0u : (0xffffffffu >> (first + 32 - n_cand));
+          if (first < cur) freew &= full << (cur - first);                                  // only lane 0 can be cut
+          if (first + 32 > n_cand) freew &= first >= n_cand ? 0u : (full >> (first + 32 - n_cand));
         }
         const int cnt = __popc(freew);
         int incl = cnt;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          const int v = __shfl_up_sync(full, incl, o);
           if (lane >= o) incl += v;
         }
-        const int total = __shfl_sync(0xffffffffu, incl, 31);
-        int slot = m + incl - cnt;
-        unsigned int fw = freew;
-        while (fw && slot < kBatch) {
-          const int b = __ffs(fw) - 1;
-          fw &= fw - 1;
-          const int ps = (wbase << 5) + b;
-          c->pos[slot] = ps;
-          c->cval[slot] = cand[ps];
-          ++slot;
-        }
+        const int total = __shfl_sync(full, incl, 31);
+        // slot `lane` of the batch takes the (lane - m)-th free position of these 32 words
+        const int want = lane - m;
+        int wi = 0;                                    // first lane whose inclusive count exceeds `want`
+#pragma unroll
+        for (int step = 16; step > 0; step >>= 1)
+          if (__shfl_sync(full, incl, wi + step - 1) <= want) wi += step;
+        wi = min(wi, 31);
+        const int ex = __shfl_sync(full, incl - cnt, wi);
+        const unsigned int word = __shfl_sync(full, freew, wi);
+        if (want >= 0 && want < total) s_pos[lane] = (((cur >> 5) + wi) << 5) + nth_set_bit(word, want - ex);
         m = min(kBatch, m + total);
-        if (m < kBatch) cur = ((cur >> 5) + 32) << 5;
+        if (m < kBatch) cur = ((cur >> 5) + 32) << 5;  // all 32 words consumed
       }
-      if (lane == 0) c->m = m;
+      if (lane == 0) s_m = m;
+      s_conf[lane] = 0u;
     }
-    ok = grid_barrier(c, n_ctas, &p.st->status);
-    if (!ok) break;
-    const int m = *reinterpret_cast<volatile int*>(&c->m);
-    if (m == 0) {                                          // list exhausted
-      if (blockIdx.x == 0 && tid == 0) c->examined = n_cand;
-      break;
+    __syncthreads();
+    const int m = s_m;
+    if (m == 0) break;                                 // list exhausted (the same in every CTA)
+
+    // ---- B: stage the members' columns (warp w: members w, w + 8, ...), then the pairs among them ----
+    for (int q = warp; q < m; q += kThreads / 32) {
+      const int j = cand[s_pos[q]];
+      const long long a0 = p.xptr[j];
+      const int na = (int)(p.xptr[j + 1] - a0);
+      if (lane == 0) { s_col[q] = j; s_ptr[q] = a0; s_len[q] = na; s_n2[q] = p.n2[j]; }
+      if (na <= kColCap)
+        for (int e = lane; e < na; e += 32) { brow[q][e] = __ldg(p.xrow + a0 + e); bval[q][e] = __ldg(p.xv + a0 + e); }
     }
-    if (tid < kBatch) s_pos[tid] = __ldcg(&c->pos[min(tid, m - 1)]);
+    __syncthreads();
+    {
+      const int qa = tid >> 3;                         // eight threads per member qa: partners qb = tid % 8 + 8 k
+      if (qa < m) {
+        const int na = s_len[qa];
+        const int* ar = na <= kColCap ? brow[qa] : p.xrow + s_ptr[qa];
+        const float* av = na <= kColCap ? bval[qa] : p.xv + s_ptr[qa];
+        unsigned int hits = 0u;
+        for (int qb = (tid & 7); qb < m; qb += 8) {
+          if (qb <= qa) continue;
+          const int nb = s_len[qb];
+          const int* br = nb <= kColCap ? brow[qb] : p.xrow + s_ptr[qb];
+          const float* bv = nb <= kColCap ? bval[qb] : p.xv + s_ptr[qb];
+          const float dot = sparse_dot_arrays(ar, av, na, br, bv, nb);
+          const double den = sqrt(s_n2[qa] * s_n2[qb]);
+          if (den > 0.0 && fabs((double)dot) >= rho * den) hits |= 1u << qb;
+        }
+        if (hits) atomicOr(&s_conf[qa], hits);
+      }
+    }
     __syncthreads();
 
-    // ---- B: all CTAs: conflict rows of the batch.  CTA k works on batch member k mod m. ----
+    // ---- C: decide the batch (warp 0, lane = member; the same in every CTA).  Passes of warp-wide ORs: members hit
+    //      by one kept in the last pass are out; a member no earlier undecided member conflicts with is kept. ----
+    if (tid < 32) {
+      const unsigned int valid = m >= 32 ? full : ((1u << m) - 1u);
+      const unsigned int mine = s_conf[lane];          // conflicts with LATER members only
+      unsigned int und = valid, keep = 0u, fresh = 0u;
+      for (int pass = 0; pass < kBatch && und != 0u; ++pass) {
+        if (pass > 0) und &= ~__reduce_or_sync(full, ((fresh >> lane) & 1u) ? mine : 0u);
+        const unsigned int thr = __reduce_or_sync(full, ((und >> lane) & 1u) ? mine : 0u);
+        fresh = und & ~thr;
+        keep |= fresh;
+        und &= ~fresh;
+      }
+      const int nk = s_kept;
+      const int room = p.n_keep - nk;
+      bool done = false;
+      if (__popc(keep) >= room) {                      // stop exactly at P: drop the surplus from the back
+        while (__popc(keep) > room) keep &= ~(1u << (31 - __clz(keep)));
+        done = true;
+      }
+      if (blockIdx.x == 0 && ((keep >> lane) & 1u)) kept_out[nk + __popc(keep & ((1u << lane) - 1u))] = s_col[lane];
+      if (lane == 0) {
+        s_keep = keep;
+        s_kept = nk + __popc(keep);
+        if (done) { s_examined = s_pos[31 - __clz(keep)] + 1; s_done = 1; }
+        else s_cursor = s_pos[m - 1] + 1;
+      }
+    }
+    __syncthreads();
+    if (s_done) break;                                 // P kept: what they block no longer matters
+
+    // ---- D: the kept members' conflicts with the later unblocked candidates, shared out over the grid:
+    //      task (kept member k, mask word w) -> one warp, a lane per candidate of the word ----
     {
-      const int q = blockIdx.x % m;
-      const int share = (int)((n_ctas - q + m - 1) / m);   // CTAs working on member q
-      const int mine = blockIdx.x / m;                      // this CTA's rank among them
-      const int a = s_pos[q];
-      const int ja = cand[a];
-      const long long a0 = p.xptr[ja];
-      const int na = (int)(p.xptr[ja + 1] - a0);
-      const bool staged = na <= kStage;
-      if (staged)
-        for (int e = tid; e < na; e += kThreads) { arow[e] = p.xrow[a0 + e]; aval[e] = p.xv[a0 + e]; }
-      __syncthreads();
-      const int* ar = staged ? arow : p.xrow + a0;
-      const float* av = staged ? aval : p.xv + a0;
-      const double n2a = p.n2[ja];
-      for (int w = (a >> 5) + mine * (kThreads / 32) + warp; w < W; w += share * (kThreads / 32)) {
+      const unsigned int keep = s_keep;
+      const int n_new = __popc(keep);
+      const long long tasks = (long long)n_new * W;
+      const long long n_warps = (long long)n_ctas * (kThreads / 32);
+      for (long long t = (long long)blockIdx.x * (kThreads / 32) + warp; t < tasks; t += n_warps) {
+        const int k = (int)(t / W), w = (int)(t - (long long)k * W);
+        const int q = nth_set_bit(keep, k);
+        const int a = s_pos[q];
+        if (w < (a >> 5)) continue;
         const int b = w * 32 + lane;
         bool hit = false;
-        if (b < n_cand && b != a) {
+        if (b < n_cand && b > a && !((blocked[w] >> lane) & 1u)) {
+          const int na = s_len[q];
+          const int* ar = na <= kColCap ? brow[q] : p.xrow + s_ptr[q];
+          const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
           const int jb = cand[b];
-          const float dot = sparse_dot(ar, av, na, p, jb);
-          const double den = sqrt(n2a * p.n2[jb]);
+          const float dot = sparse_dot_prefetched<32>(ar, av, na, p, jb);
+          const double den = sqrt(s_n2[q] * p.n2[jb]);
           hit = den > 0.0 && fabs((double)dot) >= rho * den;
         }
-        const unsigned int word = __ballot_sync(0xffffffffu, hit);
-        if (lane == 0) rows[(long long)q * W + w] = word;
+        const unsigned int word = __ballot_sync(full, hit);
+        if (lane == 0 && word != 0u) atomicOr(&blocked_g[w], word);
       }
     }
     ok = grid_barrier(c, n_ctas, &p.st->status);
     if (!ok) break;
-
-    // ---- C: CTA 0 decides the batch in order and extends the mask ----
-    if (blockIdx.x == 0) {
-      if (tid < 32) {
-        const unsigned int valid = m >= 32 ? 0xffffffffu : ((1u << m) - 1u);
-        const long long my_row = (long long)min(lane, m - 1) * W;
-        unsigned int confl = 0u;
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-          const int pb = s_pos[b];                       // (entries past m repeat the last member; masked below)
-          confl |= ((__ldcg(&rows[my_row + (pb >> 5)]) >> (pb & 31)) & 1u) << b;
-        }
-        confl &= valid & ~((2u << lane) - 1u);           // later members only; a row is valid from its own word on
-        if (lane >= m) confl = 0u;
-        unsigned int cq[kBatch];
-#pragma unroll
-        for (int q = 0; q < kBatch; ++q) cq[q] = __shfl_sync(0xffffffffu, confl, q);
-        unsigned int alive = valid, keep = 0u;
-#pragma unroll
-        for (int q = 0; q < kBatch; ++q)
-          if ((alive >> q) & 1u) { keep |= 1u << q; alive &= ~cq[q]; }
-        const int nk = c->n_kept;
-        const int room = p.n_keep - nk;
-        bool full = false;
-        if (__popc(keep) >= room) {
-          while (__popc(keep) > room) keep &= ~(1u << (31 - __clz(keep)));
-          full = true;
-        }
-        if ((keep >> lane) & 1u) kept_out[nk + __popc(keep & ((1u << lane) - 1u))] = __ldcg(&c->cval[lane]);
-        if (lane == 0) {
-          s_keep = keep;
-          c->n_kept = nk + __popc(keep);
-          if (full) { c->examined = s_pos[31 - __clz(keep)] + 1; c->done = 1; }
-          else c->cursor = s_pos[m - 1] + 1;
-        }
-      }
-      __syncthreads();
-      const unsigned int keep = s_keep;
-      for (int w = tid; w < W; w += kThreads) {
-        unsigned int acc = 0u;
-        unsigned int k = keep;
-        while (k) {
-          const int q = __ffs(k) - 1;
-          k &= k - 1;
-          if (w >= (s_pos[q] >> 5)) acc |= __ldcg(&rows[(long long)q * W + w]);
-        }
-        if (acc) blocked[w] |= acc;
-      }
-    }
-    ok = grid_barrier(c, n_ctas, &p.st->status);
-    if (!ok) break;
-    if (*reinterpret_cast<volatile int*>(&c->done)) break;
+    for (int w = tid; w < W; w += kThreads) blocked[w] = __ldcg(&blocked_g[w]);
+    __syncthreads();
   }
 
   if (blockIdx.x == 0) {
     __syncthreads();
-    const int nk = *reinterpret_cast<volatile int*>(&c->n_kept);
+    const int nk = s_kept;
     for (int i = nk + tid; i < p.n_keep; i += kThreads) kept_out[i] = -1;
     if (tid == 0) {
-      p.st->counts[1] = c->examined; p.st->counts[2] = nk; p.st->counts[3] = 0;
+      p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0;
       p.st->amb_count = 0; p.st->window_short = 0; p.st->prefer_walk = 1;
       c->failed = 0;
     }
