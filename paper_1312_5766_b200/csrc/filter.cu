@@ -36,7 +36,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; }
     return;
   }
-  if (p.layout == STRADS_CSC && n_cand < n_total && p.st->prefer_walk && ((p.st->round / (unsigned)p.part_count) & 63ull) != 0) {
+  if (p.layout == STRADS_CSC && n_cand < n_total && window_skipped(p)) {
     if (threadIdx.x == 0) p.st->window_short = 1;    // window attempt skipped: go straight to the whole-list walk
     return;
   }
@@ -220,7 +220,10 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (tid == 0) {
     p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0;
     p.st->window_short = (!only_if_short && nk < p.n_keep && n_cand < n_total) ? 1 : 0;
-    if (!only_if_short && n_cand < n_total && !p.st->window_short) p.st->prefer_walk = 0;
+    if (!only_if_short && n_cand < n_total) {          // a window attempt: remember how it went
+      if (p.st->window_short) p.st->walk_streak = min(p.st->walk_streak + 1, 16);
+      else { p.st->prefer_walk = 0; p.st->walk_streak = 0; }
+    }
   }
 }
 

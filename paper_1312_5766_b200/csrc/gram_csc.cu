@@ -22,7 +22,7 @@ constexpr int kStage = 1024;          // entries of column a staged in shared me
 // Whether this launch has anything to do (same test in every kernel of the step).
 __device__ __forceinline__ bool gram_wanted(const Problem& p, int only_if_short, int window) {
   if (only_if_short && !p.st->window_short) return false;
-  if (window && p.st->prefer_walk && ((p.st->round / (unsigned)p.part_count) & 63ull) != 0) return false;   // the window attempt is being skipped
+  if (window && window_skipped(p)) return false;
   return true;
 }
 

@@ -35,6 +35,7 @@ struct DeviceState {
   unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
   int bucket_failed;            // ... a bucket or the pair list overflowed this round: the all-pairs kernel redoes the bits
   int bucket_avoid;             // ... it overflowed lately: go straight to the all-pairs kernel for a while
+  int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int pad;
 };
@@ -102,6 +103,17 @@ struct Problem {
   int part_count, part_index;
 };
 static constexpr int kObjBlocks = 296;
+
+// CSC: whether this round leaves the candidate window out and goes straight to the on-demand walk: after a
+// window that was too short, the next attempt comes 64 rounds (of this scheduler) later, and twice as late
+// after every further failure (up to 65,536).
+__device__ __forceinline__ bool window_skipped(const Problem& p) {
+  const DeviceState* st = p.st;
+  if (!st->prefer_walk) return false;
+  const unsigned long long period = 64ull << min(max(st->walk_streak - 1, 0), 10);
+  return ((st->round / (unsigned)p.part_count) & (period - 1ull)) != 0ull;
+}
+
 
 // ---------------------------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11) and the FP32 race key.
