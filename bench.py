@@ -344,10 +344,22 @@ def main():
                         "sample": f"{rounds} full oracle rounds of {args.workload} from the state after the timed "
                                   f"region ({sec:.1f} s, single thread; host has {os.cpu_count()} cores)"}
 
-    # kernels per round: sampler 4, window Gram (dense: pack, screen, split-K reduce, recheck, 3xTF32 gate = 5;
-    # CSC: 1), walk 1, whole-list retry (dense 4 + 1, CSC: the on-demand walk, 1; they return at once when not
-    # needed), update 2
-    launches_per_round = 4 + (5 + 1 + 5 if p.layout == wl.DENSE else 1 + 1 + 1) + 2
+    # kernels launched per round (the library's fixed sequence; launches of the whole-list retry return at once when
+    # the window sufficed): sampler hist + collect + ordering (1 kernel for P' <= 2048, else chunk sort + rank);
+    # dense Gram of n candidates: pack, screen, split-K reduce (few tiles only), recheck, and a 3xTF32 launch unless a
+    # retry follows; CSC Gram: bucket fill, bucket pairs, pair bits, all-pairs fallback; walk 1; update 2
+    def gram_launches(n, retry_follows):
+        if p.layout != wl.DENSE:
+            return 4
+        nt = (n + 127) // 128
+        tiles = nt * (nt + 1) // 2
+        return 3 + (1 if tiles * 2 <= 148 else 0) + (0 if retry_follows else 1)
+    launches_per_round = 2 + (1 if p.n_candidates <= 2048 else 2) + 2
+    if window < p.n_candidates:
+        launches_per_round += gram_launches(window, True) + 1
+        launches_per_round += (gram_launches(p.n_candidates, False) + 1) if p.layout == wl.DENSE else 1
+    else:
+        launches_per_round += gram_launches(p.n_candidates, False) + 1
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
