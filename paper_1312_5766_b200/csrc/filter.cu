@@ -60,7 +60,33 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     return;
   }
   for (int i = tid; i < n_cand; i += kThreads) s_cand[i] = cand[i];
-  if (resident) {
+  if (resident && (W & 3) == 0 && Wn <= 64) {
+    // all rows at once, 128-bit loads: 8 or 16 lanes per row (one per group of four words), sixteen rows in
+    // flight per thread, loads before stores
+    const int quads = (Wn + 3) >> 2;                   // (W % 4 == 0: 4 * quads <= W)
+    const int lpr_log = quads <= 8 ? 3 : 4, lpr = 1 << lpr_log;
+    const int c = tid & (lpr - 1), rstep = kThreads >> lpr_log;
+    for (int r0 = tid >> lpr_log; r0 < n_cand; r0 += 16 * rstep) {
+      uint4 v[16];
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        const int r = r0 + u * rstep;
+        v[u] = make_uint4(0u, 0u, 0u, 0u);
+        if (r < n_cand && c < quads) v[u] = __ldcg(reinterpret_cast<const uint4*>(p.conflict + (long long)r * W) + c);
+      }
+#pragma unroll
+      for (int u = 0; u < 16; ++u) {
+        const int r = r0 + u * rstep;
+        if (r < n_cand && c < quads) {
+          unsigned int* dst = rows + r * Wp + 4 * c;
+          dst[0] = v[u].x;
+          if (4 * c + 1 < Wn) dst[1] = v[u].y;
+          if (4 * c + 2 < Wn) dst[2] = v[u].z;
+          if (4 * c + 3 < Wn) dst[3] = v[u].w;
+        }
+      }
+    }
+  } else if (resident) {
     // all rows at once: independent loads, eight in flight per thread, before any store
     const int total = n_cand * Wn;
     for (int i0 = tid; i0 < total; i0 += 8 * kThreads) {
