@@ -277,7 +277,7 @@ __global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
 // number of smaller keys in its buffer (+ n_sure for boundary keys: every sure key is smaller); the key of
 // rank r < P' is candidate r.  A CTA takes 32 keys of one buffer, stages the whole buffer (<= 2048 keys) in
 // shared memory and counts with eight threads per key, each over an eighth of the buffer.
-constexpr int kDirectMax = 2048;         // P' and the boundary buffer up to this many keys (beyond, sorting wins)
+constexpr int kDirectMax = 2048;         // P' and the boundary buffer up to this many keys (beyond, sorting is as fast)
 constexpr int kDirectKeys = 32;          // keys per CTA
 __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand_out) {
   chain_begin();
@@ -295,10 +295,9 @@ __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand
   __syncthreads();
   const int k = first + (threadIdx.x >> 3), slice = threadIdx.x & 7;
   const unsigned long long key = k < total ? all[k] : 0ull;
-  const int per = (total + 7) >> 3, i0 = slice * per, i1 = min(total, i0 + per);
-  int below = 0;
-#pragma unroll 8
-  for (int i = i0; i < i1; ++i) below += all[i] < key;
+  int below = 0;                                        // thread `slice` looks at keys slice, slice + 8, ...: the eight
+#pragma unroll 8                                        // threads of a key read eight consecutive words (no bank conflict)
+  for (int i = slice; i < total; i += 8) below += all[i] < key;
   below += __shfl_xor_sync(0xffffffffu, below, 1);
   below += __shfl_xor_sync(0xffffffffu, below, 2);
   below += __shfl_xor_sync(0xffffffffu, below, 4);
