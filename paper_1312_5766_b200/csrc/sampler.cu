@@ -26,19 +26,41 @@ namespace {
 
 constexpr int kThreads = 256;
 
-// Calls f(key) for each of the (up to) four coefficients of Philox block g.
+// Whether the race key of a coefficient (last change d, Philox word x) is certainly above `cut` (> 0), from
+// a few operations instead of the whole key: T = E / w and the computed E is never below
+// v = (x + 1/2) / 2^32 (-ln(1 - v) >= v; checked against the key's arithmetic over its whole range of x), so
+// v > 1.01 cut w  implies  T > cut.  Nearly all coefficients are far above the boundary of the P' smallest.
+__device__ __forceinline__ bool key_surely_above(float cut, float d, float eta, uint32_t x, bool uniform) {
+  const float w = uniform ? 1.0f : __fmaf_rn(d, d, eta);
+  const float v = __fmaf_rn(__uint2float_rn(x), __uint_as_float(0x2f800000u), __uint_as_float(0x2f000000u));
+  return v > __fmul_rn(__fmul_rn(cut, w), 1.01f);
+}
+
+// Calls f(key) for each of the (up to) four coefficients of Philox block g, leaving out those whose key is
+// certainly above `cut` (cut <= 0: none is left out).
 template <typename F>
-__device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned long long t, long long g, F&& f) {
+__device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned long long t, long long g, float cut, F&& f) {
   uint32_t w[4];
   philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
   const long long j0 = g * 4;
   const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  if (cut > 0.f && p.part_count <= 1 && j0 + 3 < p.J) {
+    const float4 d = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
+    if (!key_surely_above(cut, d.x, p.eta, w[0], uniform)) f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, uniform));
+    if (!key_surely_above(cut, d.y, p.eta, w[1], uniform)) f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, uniform));
+    if (!key_surely_above(cut, d.z, p.eta, w[2], uniform)) f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, uniform));
+    if (!key_surely_above(cut, d.w, p.eta, w[3], uniform)) f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, uniform));
+    return;
+  }
   if (p.part_count > 1) {                              // only the coefficients this scheduler owns take part
     const unsigned int S = (unsigned)p.part_count, r0 = (unsigned int)j0 % S;
 #pragma unroll
     for (unsigned int i = 0; i < 4; ++i)
-      if (j0 + i < p.J && (r0 + i) % S == (unsigned)p.part_index)
-        f(race_key64(__ldg(p.delta + j0 + i), p.eta, w[i], (uint32_t)(j0 + i), uniform));
+      if (j0 + i < p.J && (r0 + i) % S == (unsigned)p.part_index) {
+        const float d = __ldg(p.delta + j0 + i);
+        if (cut > 0.f && key_surely_above(cut, d, p.eta, w[i], uniform)) continue;
+        f(race_key64(d, p.eta, w[i], (uint32_t)(j0 + i), uniform));
+      }
     return;
   }
   if (j0 + 3 < p.J) {
@@ -52,6 +74,56 @@ __device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned lon
     for (int i = 0; i < 4; ++i)
       if (j0 + i < p.J) f(race_key64(p.delta[j0 + i], p.eta, w[i], (uint32_t)(j0 + i), uniform));
   }
+}
+
+// The same with a cutoff, for a whole warp: lane l looks at Philox block g0 + l.  Few coefficients survive the
+// cheap test, so computing their keys on the spot would leave most lanes idle while one works; the survivors
+// (index, Philox word) go to a queue of the warp in shared memory instead and the keys of a full queue are
+// computed by all lanes together.  drain_keys() must follow the last call.
+constexpr int kQueue = 256;              // entries per warp; a call appends at most 128
+struct KeyQueue { uint2* slots; int n; };
+
+template <typename F>
+__device__ __forceinline__ void drain_keys(const Problem& p, KeyQueue& q, F&& f) {
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  __syncwarp();
+  for (int i = (int)(threadIdx.x & 31); i < q.n; i += 32) {
+    const uint2 e = q.slots[i];
+    f(race_key64(__ldg(p.delta + e.x), p.eta, e.y, e.x, uniform));
+  }
+  __syncwarp();
+  q.n = 0;
+}
+
+template <typename F>
+__device__ __forceinline__ void queue_keys_of_groups(const Problem& p, unsigned long long t, long long g0, long long groups,
+                                                     float cut, KeyQueue& q, F&& f) {
+  const int lane = threadIdx.x & 31;
+  const long long g = g0 + lane;
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  float d[4] = {0.f, 0.f, 0.f, 0.f};
+  const long long j0 = g * 4;
+  if (g < groups) {
+    philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
+    if (j0 + 3 < p.J) {
+      const float4 v = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
+      d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) if (j0 + i < p.J) d[i] = p.delta[j0 + i];
+    }
+  }
+  const unsigned int S = (unsigned)max(p.part_count, 1), r0 = (unsigned int)j0 % S;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const bool in = g < groups && j0 + i < p.J && (S == 1u || (r0 + i) % S == (unsigned)p.part_index) &&
+                    !key_surely_above(cut, d[i], p.eta, w[i], uniform);
+    const unsigned int mask = __ballot_sync(0xffffffffu, in);
+    if (in) q.slots[q.n + __popc(mask & ((1u << lane) - 1u))] = make_uint2((uint32_t)(j0 + i), w[i]);
+    q.n += __popc(mask);
+  }
+  if (q.n > kQueue - 128) drain_keys(p, q, f);
 }
 
 // Whole CTA (kThreads threads): the bin b with before(b) < k_rem <= before(b) + h[b], where before(b)
@@ -88,8 +160,12 @@ __device__ void find_bin(const unsigned int* h, int nbins, long long k_rem, int*
   __syncthreads();
 }
 
-__global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
+// mode 0: plain.  mode 1: bins only the keys below a cutoff carried over from the previous round (four times that
+// round's boundary; the keys certainly above it are not even computed); if fewer than P' keys turn out to lie
+// below it, nothing is published and the launch behind (mode 2: plain, and only then) does the pass again.
+__global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
   chain_begin();
+  if (mode == 2 && !p.st->sample_redo) return;
   __shared__ unsigned int sh[kHistBins];
   __shared__ int s_last;
   __shared__ SelectState s_sel;
@@ -98,8 +174,22 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
   __syncthreads();
   const unsigned long long t = p.st->round;
   const long long groups = (p.J + 3) >> 2;
-  for (long long g = (long long)blockIdx.x * kThreads + tid; g < groups; g += (long long)gridDim.x * kThreads)
-    for_keys_of_group(p, t, g, [&](unsigned long long key) { atomicAdd(&sh[key >> (64 - kHistBits)], 1u); });
+  const float cut = mode == 1 ? p.st->t_cut : 0.f;
+  const unsigned int cut_bin = cut > 0.f ? (__float_as_uint(cut) >> (32 - kHistBits)) : (unsigned)kHistBins;   // bins below it are complete
+  auto count = [&](unsigned long long key) {
+    const unsigned int bin = (unsigned int)(key >> (64 - kHistBits));
+    if (bin < cut_bin) atomicAdd(&sh[bin], 1u);
+  };
+  if (cut > 0.f) {
+    __shared__ uint2 s_queue[kThreads / 32][kQueue];
+    KeyQueue q = {s_queue[tid >> 5], 0};
+    for (long long g0 = (long long)blockIdx.x * kThreads + (tid & ~31); g0 < groups; g0 += (long long)gridDim.x * kThreads)
+      queue_keys_of_groups(p, t, g0, groups, cut, q, count);
+    drain_keys(p, q, count);
+  } else {
+    for (long long g = (long long)blockIdx.x * kThreads + tid; g < groups; g += (long long)gridDim.x * kThreads)
+      for_keys_of_group(p, t, g, 0.f, count);
+  }
   __syncthreads();
   for (int b = tid; b < kHistBins; b += kThreads)
     if (sh[b]) atomicAdd(&p.hist[b], sh[b]);
@@ -125,8 +215,25 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
   __syncthreads();
   __shared__ int s_bin;
   __shared__ long long s_before;
+  if (cut > 0.f) {                                     // enough keys below the cutoff?
+    __shared__ unsigned int s_total;
+    if (tid == 0) s_total = 0u;
+    __syncthreads();
+    unsigned int mine = 0u;
+    for (int b = tid; b < kHistBins; b += kThreads) mine += sh[b];
+    atomicAdd(&s_total, mine);
+    __syncthreads();
+    if (s_total < (unsigned)p.n_cand) {
+      if (tid == 0) { p.st->hist_ticket = 0; p.st->sample_redo = 1; p.st->t_cut = 0.f; }
+      return;
+    }
+  }
   find_bin(sh, kHistBins, p.n_cand, &s_bin, &s_before);
   if (tid == 0) {
+    p.st->sample_redo = 0;
+    // next round's cutoff: four times the upper edge of this boundary bin (none if that is not a finite number)
+    const unsigned int edge = ((unsigned int)s_bin + 1u) << (32 - kHistBits);
+    p.st->t_cut = edge < 0x7f800000u ? __fmul_rn(4.0f, __uint_as_float(edge)) : 0.f;
     p.st->hist_ticket = 0;
     p.st->sure_count = 0;                             // append cursors of the collect pass that follows
     p.st->boundary_count = 0;
@@ -145,7 +252,7 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p) {
     for (int b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
     __syncthreads();
     for (long long g = tid; g < groups; g += kThreads)
-      for_keys_of_group(p, t, g, [&](unsigned long long key) {
+      for_keys_of_group(p, t, g, 0.f, [&](unsigned long long key) {
         if ((key >> (64 - bits)) == prefix)
           atomicAdd(&sh[(key >> (64 - bits - width)) & ((1u << width) - 1u)], 1u);
       });
@@ -169,18 +276,30 @@ __global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
   const unsigned long long t = p.st->round;
   const long long groups = (p.J + 3) >> 2;
   const int shift = 64 - sel.bits;
-  for (long long g = (long long)blockIdx.x * kThreads + threadIdx.x; g < groups;
-       g += (long long)gridDim.x * kThreads)
-    for_keys_of_group(p, t, g, [&](unsigned long long key) {
-      const unsigned long long pfx = key >> shift;
-      if (pfx < sel.prefix) {
-        const unsigned int i = atomicAdd(&p.st->sure_count, 1u);
-        if (i < (unsigned)p.cap_sure) p.sure[i] = key;
-      } else if (pfx == sel.prefix) {
-        const unsigned int i = atomicAdd(&p.st->boundary_count, 1u);
-        if (i < (unsigned)p.cap_boundary) p.boundary[i] = key;
-      }
-    });
+  // keys certainly above the boundary's upper edge are not computed
+  unsigned long long edge = sel.bits <= 32 ? ((sel.prefix + 1ull) << (32 - sel.bits)) : (sel.prefix >> (sel.bits - 32));
+  const float cut = edge < 0x7f800000ull && edge > 0ull ? __uint_as_float((unsigned int)edge) : 0.f;
+  auto take = [&](unsigned long long key) {
+    const unsigned long long pfx = key >> shift;
+    if (pfx < sel.prefix) {
+      const unsigned int i = atomicAdd(&p.st->sure_count, 1u);
+      if (i < (unsigned)p.cap_sure) p.sure[i] = key;
+    } else if (pfx == sel.prefix) {
+      const unsigned int i = atomicAdd(&p.st->boundary_count, 1u);
+      if (i < (unsigned)p.cap_boundary) p.boundary[i] = key;
+    }
+  };
+  const int tid = threadIdx.x;
+  if (cut > 0.f) {
+    __shared__ uint2 s_queue[kThreads / 32][kQueue];
+    KeyQueue q = {s_queue[tid >> 5], 0};
+    for (long long g0 = (long long)blockIdx.x * kThreads + (tid & ~31); g0 < groups; g0 += (long long)gridDim.x * kThreads)
+      queue_keys_of_groups(p, t, g0, groups, cut, q, take);
+    drain_keys(p, q, take);
+  } else {
+    for (long long g = (long long)blockIdx.x * kThreads + tid; g < groups; g += (long long)gridDim.x * kThreads)
+      for_keys_of_group(p, t, g, 0.f, take);
+  }
 }
 
 // Ascending bitonic sort of n (a power of two) keys in shared memory by the whole CTA.
@@ -316,7 +435,11 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   cudaError_t e;
-  if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
+  // many coefficients: the first pass leaves out the keys far above the last boundary (and a second launch
+  // repeats it in full in the rare round where that boundary was a bad guide)
+  const bool guided = p.J >= (1 << 22);     // (below that the passes are bound by latency, not by arithmetic)
+  if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, guided ? 1 : 0)) != cudaSuccess) return e;
+  if (guided && (e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, 2)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
   if (p.cap_sure <= kDirectMax && p.cap_boundary <= kDirectMax) {
     const int ctas = (p.cap_sure + kDirectKeys - 1) / kDirectKeys + (p.cap_boundary + kDirectKeys - 1) / kDirectKeys;

@@ -35,6 +35,8 @@ struct DeviceState {
   unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
   int bucket_failed;            // ... a bucket or the pair list overflowed this round: the all-pairs kernel redoes the bits
   int bucket_avoid;             // ... it overflowed lately: go straight to the all-pairs kernel for a while
+  float t_cut;                  // sampler: cutoff for the next round's first pass (0: none), see k_sample_hist
+  int sample_redo;              // sampler: the guided first pass found too few keys; the plain pass behind it runs
   int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int pad;

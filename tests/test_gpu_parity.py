@@ -90,6 +90,30 @@ def test_sampler_refinement_path_is_exact():
     assert np.array_equal(s.sample().cpu().numpy(), oracle.sample(d2.astype(np.float64), p.eta, 0, 0, n_cand))
 
 
+def test_guided_first_pass_is_exact_when_the_guide_is_good_bad_or_absent():
+    """For J >= 2^22 the sampler's first pass leaves out the keys certainly above four times the previous
+    round's boundary and repeats itself in full when too few keys lie below it.  Same candidates as ranking
+    all J keys, whatever the previous round was like."""
+    J, n_cand = 4_400_000, 1500
+    cfg = dict(kind="csc_uniform", n_rows=2000, n_cols=J, n_true=50, lam_frac=0.01, nnz_col=4,
+               n_candidates=n_cand, n_keep=64, rho=0.1)
+    p = wl.make_problem(cfg, seed=2)
+    s = _solver(p)
+    rng = np.random.default_rng(4)
+    base = np.abs(rng.normal(size=J)).astype(np.float32)
+    steps = [("initial C everywhere", None), ("same again: guided", None), ("weights / 1e6: guide far too low", base * 1e-3),
+             ("weights x 1e6: guide far too high", base), ("mostly zero changes", np.where(rng.random(J) < 0.99, 0, base).astype(np.float32)),
+             ("same again: guided", None)]
+    for t, (what, delta) in enumerate(steps):
+        if delta is not None:
+            s.delta.copy_(torch.from_numpy(delta))
+        s.set_round(t)
+        got = s.sample().cpu().numpy()
+        want = oracle.sample(s.delta.cpu().numpy(), float(np.float32(p.eta)), p.seed, t, n_cand)
+        assert np.array_equal(got, want), what
+    assert s.status()[0] == 0
+
+
 def test_uniform_draw_flag_ignores_delta():
     b = _binding()
     J, n_cand = 50_000, 500
