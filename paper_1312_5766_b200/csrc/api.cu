@@ -63,7 +63,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, total;
+      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap;
   long long ldc;
 };
@@ -130,6 +130,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_bucket_count = take(buckets ? sizeof(unsigned int) * (size_t)c->n_rows : 0);
   L.off_bucket_items = take(buckets ? sizeof(int) * (size_t)c->n_rows * kBucketSlots : 0);
   L.off_pairs = take(sizeof(unsigned int) * (size_t)L.pair_cap);
+  L.off_resid_acc = take(csc ? sizeof(long long) * (size_t)c->n_rows : 0);
   L.total = o;
   return L;
 }
@@ -276,6 +277,7 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
   p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
   p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
+  p.resid_acc = reinterpret_cast<long long*>(ws + L.off_resid_acc);
   p.pair_cap = L.pair_cap;
   p.bucket_count = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
   p.bucket_items = L.pair_cap ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;
@@ -359,6 +361,8 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
     if (sc.p.layout == STRADS_CSC) {
       if ((e = prepare_walk_csc(sc.p, &sc.walk_grid)) != cudaSuccess) return fail(cuda_fail(e, "prepare_walk_csc"));
       if ((e = cudaMemsetAsync(sc.p.walk_ctl, 0, sizeof(WalkControl), h->stream)) != cudaSuccess)
+        return fail(cuda_fail(e, "cudaMemsetAsync"));
+      if ((e = cudaMemsetAsync(sc.p.resid_acc, 0, sizeof(long long) * (size_t)sc.p.N, h->stream)) != cudaSuccess)
         return fail(cuda_fail(e, "cudaMemsetAsync"));
       if (sc.p.bucket_count != nullptr &&
           (e = cudaMemsetAsync(sc.p.bucket_count, 0, sizeof(unsigned int) * (size_t)sc.p.N, h->stream)) != cudaSuccess)

@@ -35,6 +35,8 @@ struct DeviceState {
   unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
   int bucket_failed;            // ... a bucket or the pair list overflowed this round: the all-pairs kernel redoes the bits
   int bucket_avoid;             // ... it overflowed lately: go straight to the all-pairs kernel for a while
+  unsigned long long dmax_bits; // CSC update: bits of max |change| of this round (non-negative doubles order like integers)
+  int resid_shift;              // CSC update: this round's fixed-point scale is 2^resid_shift (INT_MIN: nothing moved)
   float t_cut;                  // sampler: cutoff for the next round's first pass (0: none), see k_sample_hist
   int sample_redo;              // sampler: the guided first pass found too few keys; the plain pass behind it runs
   int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
@@ -95,6 +97,7 @@ struct Problem {
   unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words], OR-ed into by the whole grid
   unsigned int* walk_rows;      // (unused)
   WalkControl* walk_ctl;
+  long long* resid_acc;         // CSC: [N] fixed-point accumulators of the residual update (zero between rounds)
   // CSC Gram by row buckets (null / 0 when not provided for)
   unsigned int* bucket_count;   // [N] candidates of this round's list with an entry in row i (zero between rounds)
   int* bucket_items;            // [N][kBucketSlots] their positions in the list

@@ -5,12 +5,12 @@
 //     g_j = x_j^T r,   beta_j' = S(beta_j + g_j / n_j, lambda / n_j),   S(a, k) = sign(a) max(|a| - k, 0)
 // then beta_j <- beta_j', delta_j <- |beta_j' - beta_j|, r <- r - sum_j x_j (beta_j' - beta_j).
 //
-// Two kernels per layout.  "dot" streams the kept columns once against r (FP64 accumulation in a fixed
-// order; the last CTA of a column sums the partials in index order and applies the soft threshold).
-// "apply" updates r with every row owned by exactly one CTA: dense rows are summed over the kept
-// columns in list order; CSC contributions are added as 64-bit fixed-point integers in shared memory
-// (integer addition is associative, so hot rows shared by thousands of columns still give the same
-// bits whatever the order) -- no floating-point atomics anywhere.
+// "dot" streams the kept columns once against r (FP64 accumulation in a fixed order; the last CTA of a
+// column sums the partials in index order and applies the soft threshold).  The residual update has every
+// dense row owned by exactly one CTA and summed over the kept columns in list order; CSC contributions are
+// added as 64-bit fixed-point integers with integer atomics (integer addition is associative, so hot rows
+// shared by thousands of columns still give the same bits whatever the order) -- no floating-point atomics
+// anywhere.
 #include <climits>
 
 #include "strads_internal.cuh"
@@ -177,65 +177,64 @@ __global__ void __launch_bounds__(kThreads) k_dot_csc(Problem p, const int* __re
   for (long long q = p.xptr[j] + lane; q < p.xptr[j + 1]; q += 32)
     acc += (double)__ldg(p.xv + q) * (double)p.resid[__ldg(p.xrow + q)];
   acc = warp_sum(acc);
-  if (lane == 0) finish_coefficient(p, a, j, acc);
+  if (lane == 0) {
+    finish_coefficient(p, a, j, acc);
+    atomicMax(&p.st->dmax_bits, (unsigned long long)__double_as_longlong(fabs(p.dbeta64[a])));
+  }
 }
 
-constexpr int kMaxRowsCsc = 4096;      // rows owned by one CTA (64-bit accumulators in shared memory)
+// r <- r - sum_a x_a dbeta_a for sparse columns, in two kernels.  Contributions are added as 64-bit fixed-point
+// integers with atomics into one accumulator per row (integer addition is associative: a row shared by
+// thousands of columns gets the same bits in any order); then every row with a non-zero accumulator is
+// updated once and its accumulator cleared.  Scale: every row sum is below n_kept * max|x| * max|dbeta| < 2^e;
+// the unit is 2^-(61 - e).
+__device__ __forceinline__ int csc_resid_shift(const Problem& p, int n_kept) {
+  const double m = __longlong_as_double((long long)p.st->dmax_bits);
+  if (!(m > 0.0) || !isfinite(m)) return INT_MIN;
+  int e = 0;
+  frexp(m * (double)p.st->x_abs_max * (double)max(n_kept, 1), &e);
+  return 61 - e;
+}
 
-__global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, const int* __restrict__ kept, int rows_per_cta,
-                                                         int advance) {
+__global__ void __launch_bounds__(kThreads) k_scatter_csc(Problem p, const int* __restrict__ kept) {
   chain_begin();
-  __shared__ long long acc[kMaxRowsCsc];
-  __shared__ double wmax[kThreads / 32];
-  __shared__ int s_shift;
   const int n_kept = p.st->counts[2];
-  const long long r0 = (long long)blockIdx.x * rows_per_cta;
-  const long long r1 = min(p.N, r0 + rows_per_cta);
-  // scale: every row sum is below n_kept * max|x| * max|dbeta| < 2^e, stored in units of 2^-(61 - e)
-  double dmax = 0.0;
-  for (int a = threadIdx.x; a < n_kept; a += kThreads) dmax = fmax(dmax, fabs(p.dbeta64[a]));
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) dmax = fmax(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
-  if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = dmax;
-  for (int r = threadIdx.x; r < rows_per_cta; r += kThreads) acc[r] = 0;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    double m = 0.0;
-    for (int w = 0; w < kThreads / 32; ++w) m = fmax(m, wmax[w]);
-    int e = 0;
-    if (m > 0.0 && isfinite(m)) frexp(m * (double)p.st->x_abs_max * (double)max(n_kept, 1), &e);
-    s_shift = (m > 0.0 && isfinite(m)) ? 61 - e : INT_MIN;
+  const int shift = csc_resid_shift(p, n_kept);
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->resid_shift = shift;     // for the apply kernel (nobody here reads it)
+  if (shift == INT_MIN) return;
+  const int lane = threadIdx.x & 31;
+  const int a = (blockIdx.x * kThreads + threadIdx.x) >> 5;             // a warp per kept column
+  if (a >= n_kept) return;
+  const double d = p.dbeta64[a];
+  if (d == 0.0) return;
+  const int j = kept[a];
+  const long long q1 = p.xptr[j + 1];
+  for (long long q = p.xptr[j] + lane; q < q1; q += 32) {
+    const long long fx = __double2ll_rn(ldexp((double)__ldg(p.xv + q) * d, shift));
+    atomicAdd(reinterpret_cast<unsigned long long*>(p.resid_acc + __ldg(p.xrow + q)), (unsigned long long)fx);
   }
-  __syncthreads();
-  const int shift = s_shift;
-  if (shift != INT_MIN && r0 < p.N) {
-    for (int a = threadIdx.x; a < n_kept; a += kThreads) {
-      const double d = p.dbeta64[a];
-      if (d == 0.0) continue;
-      const int j = kept[a];
-      long long lo = p.xptr[j], hi = p.xptr[j + 1];
-      const long long end = hi;
-      while (lo < hi) {                                    // first entry with row >= r0
-        const long long mid = (lo + hi) >> 1;
-        if (__ldg(p.xrow + mid) < r0) lo = mid + 1; else hi = mid;
-      }
-      for (long long q = lo; q < end; ++q) {
-        const long long r = __ldg(p.xrow + q);
-        if (r >= r1) break;
-        const long long fx = __double2ll_rn(ldexp((double)__ldg(p.xv + q) * d, shift));
-        atomicAdd(reinterpret_cast<unsigned long long*>(&acc[r - r0]), (unsigned long long)fx);
+}
+
+__global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, int advance) {
+  chain_begin();
+  const int shift = p.st->resid_shift;
+  if (shift != INT_MIN) {
+    const long long stride = (long long)gridDim.x * kThreads;
+    for (long long r = (long long)blockIdx.x * kThreads + threadIdx.x; r < p.N; r += stride) {
+      const long long v = p.resid_acc[r];
+      if (v != 0) {
+        p.resid[r] = (float)((double)p.resid[r] - ldexp((double)v, -shift));
+        p.resid_acc[r] = 0;
       }
     }
-    __syncthreads();
-    for (long long r = r0 + threadIdx.x; r < r1; r += kThreads) {
-      const long long v = acc[r - r0];
-      if (v != 0) p.resid[r] = (float)((double)p.resid[r] - ldexp((double)v, -shift));
-    }
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
     DeviceState* st = p.st;
-    st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
-    st->round += (unsigned long long)p.part_count;       // this scheduler's next turn
+    st->dmax_bits = 0ull;                                // (read by the scatter kernel only)
+    if (advance) {
+      st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
+      st->round += (unsigned long long)p.part_count;     // this scheduler's next turn
+    }
   }
 }
 
@@ -269,11 +268,10 @@ cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool f
   } else {
     cudaError_t e;
     if ((e = launch_chained(k_dot_csc, (p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, kept)) != cudaSuccess) return e;
-    long long grid = (long long)p.sm_count * 2;
-    const long long need = (p.N + kMaxRowsCsc - 1) / kMaxRowsCsc;
-    if (grid < need) grid = need;
-    const int rows_per_cta = (int)((p.N + grid - 1) / grid);
-    return launch_chained(k_apply_csc, (unsigned)grid, kThreads, 0, s, p, kept, rows_per_cta, advance);
+    if ((e = launch_chained(k_scatter_csc, (p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, kept)) != cudaSuccess) return e;
+    long long grid = (p.N + kThreads - 1) / kThreads;
+    if (grid > (long long)p.sm_count * 8) grid = (long long)p.sm_count * 8;
+    return launch_chained(k_apply_csc, (unsigned)grid, kThreads, 0, s, p, advance);
   }
 }
 
