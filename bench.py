@@ -347,14 +347,15 @@ def main():
     # kernels launched per round (the library's fixed sequence; launches of the whole-list retry return at once when
     # the window sufficed): sampler hist (+ its full repeat for J >= 2^22, returns at once) + collect + ordering (1 kernel for P' <= 2048, else chunk sort + rank);
     # dense Gram of n candidates: pack, screen, split-K reduce (few tiles only), recheck, and a 3xTF32 launch unless a
-    # retry follows; CSC Gram: bucket fill, bucket pairs, pair bits, all-pairs fallback; walk 1; update 2 (CSC: 3)
+    # retry follows; CSC Gram: bucket fill, bucket pairs, pair bits, all-pairs fallback; walk 1; update: dense 1 (the
+    # pack kernel has formed the changes), CSC 3
     def gram_launches(n, retry_follows):
         if p.layout != wl.DENSE:
             return 4
         nt = (n + 127) // 128
         tiles = nt * (nt + 1) // 2
         return 3 + (1 if tiles * 2 <= 148 else 0) + (0 if retry_follows else 1)
-    launches_per_round = 2 + (1 if p.n_cols >= (1 << 22) else 0) + (1 if p.n_candidates <= 2048 else 2) + (2 if p.layout == wl.DENSE else 3)
+    launches_per_round = 2 + (1 if p.n_cols >= (1 << 22) else 0) + (1 if p.n_candidates <= 2048 else 2) + (1 if p.layout == wl.DENSE else 3)
     if window < p.n_candidates:
         launches_per_round += gram_launches(window, True) + 1
         launches_per_round += (gram_launches(p.n_candidates, False) + 1) if p.layout == wl.DENSE else 1

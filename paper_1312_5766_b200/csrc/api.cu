@@ -62,7 +62,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
       off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap;
   long long ldc;
@@ -111,6 +111,9 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_dbeta = take(sizeof(float) * (size_t)c->n_keep);
   L.off_dbeta64 = take(sizeof(double) * (size_t)c->n_keep);
   L.off_conflict = take(sizeof(unsigned int) * (size_t)c->n_candidates * L.mask_words);
+  const bool dense = c->layout == STRADS_DENSE_COLMAJOR;
+  L.off_cand_dbeta64 = take(dense ? sizeof(double) * (size_t)c->n_candidates : 0);
+  L.off_cand_bnew = take(dense ? sizeof(float) * (size_t)c->n_candidates : 0);
   L.off_dot_partial = take(sizeof(double) * (size_t)c->n_keep * L.dot_parts);
   L.off_dot_ticket = take(sizeof(unsigned int) * (size_t)c->n_keep);
   L.off_obj = take(first ? sizeof(double) * 2 * kObjBlocks : 0);
@@ -273,6 +276,11 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.cap_amb = L.cap_amb;
   p.xc = reinterpret_cast<float*>(ws + L.off_xc);
   p.ldc = L.ldc;
+  p.cand_dbeta64 = reinterpret_cast<double*>(ws + L.off_cand_dbeta64);
+  p.cand_bnew = reinterpret_cast<float*>(ws + L.off_cand_bnew);
+  // with one scheduler a round's steps follow one another on one stream, so r at pack time is r at update time;
+  // with several, blocks are prepared while earlier updates still change r
+  p.proposals = (c->layout == STRADS_DENSE_COLMAJOR && S == 1) ? 1 : 0;
   p.cand_cur = nullptr;
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
   p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);

@@ -146,16 +146,99 @@ __device__ __forceinline__ uint32_t decide_word(const Problem& p, const uint32_t
   return word;
 }
 
-// One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).
+// acc += x * r with acc = hi + lo a pair of floats: the product's rounding error (one fma) and the sum's (two-sum)
+// are both exact and collected in lo, so the pair carries about 2^-46 of the summed magnitudes -- FP64-grade
+// accumulation on the FP32 pipe, where conversions to double would cost more than the copy they ride on.
+// Explicitly rounded operations only: the sequence is the same bits everywhere.
+__device__ __forceinline__ void dot_step(float x, float r, float& hi, float& lo) {
+  const float pr = __fmul_rn(x, r);
+  const float pe = __fmaf_rn(x, r, -pr);
+  const float s = __fadd_rn(hi, pr);
+  const float bb = __fsub_rn(s, hi);
+  const float se = __fadd_rn(__fsub_rn(hi, __fsub_rn(s, bb)), __fsub_rn(pr, bb));
+  hi = s;
+  lo = __fadd_rn(lo, __fadd_rn(se, pe));
+}
+
+// One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).  With p.proposals the column is
+// also multiplied into the residual as it streams by (fixed order: per-thread strided sums, lanes by shuffle
+// tree, warps in index order) and the candidate's would-be update follows from it at once (Eq. 2): the update
+// step then only has to apply the proposals of the kept candidates.
 __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
                                                          int only_if_short) {
   chain_begin();
   const int a = blockIdx.x;
   if (a >= n_cand || (only_if_short && !p.st->window_short)) return;
-  const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)cand[a] * p.ld);
+  const int j = cand[a];
+  const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)j * p.ld);
   float4* dst = reinterpret_cast<float4*>(p.xc + (long long)a * p.ldc);
   const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
-  for (long long g = threadIdx.x; g < n4; g += blockDim.x) dst[g] = __ldg(src + g);
+  if (!p.proposals) {
+    for (long long g = threadIdx.x; g < n4; g += blockDim.x) dst[g] = __ldg(src + g);
+    return;
+  }
+  const float4* r4 = reinterpret_cast<const float4*>(p.resid);
+  const long long n4_full = p.N >> 2;                   // float4 groups that lie wholly inside the N rows
+  double n = 0.0;
+  float b_old = 0.f;
+  if (threadIdx.x == 0) { n = p.n2[j]; b_old = p.beta[j]; }   // two far gathers, under way while the column streams
+  float h0 = 0.f, l0 = 0.f, h1 = 0.f, l1 = 0.f;
+  constexpr int kU = 4;                                 // column loads in flight per thread
+  for (long long g0 = threadIdx.x; g0 < n4; g0 += (long long)kU * blockDim.x) {
+    float4 xv[kU], rv[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const long long g = g0 + (long long)u * blockDim.x;
+      xv[u] = g < n4 ? __ldg(src + g) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const long long g = g0 + (long long)u * blockDim.x;
+      if (g < n4_full) {
+        rv[u] = r4[g];
+      } else if (g < n4) {                              // the last, partial group: rows past N do not exist
+        const long long i = g << 2;
+        rv[u].x = p.resid[i];
+        rv[u].y = i + 1 < p.N ? p.resid[i + 1] : 0.f;
+        rv[u].z = i + 2 < p.N ? p.resid[i + 2] : 0.f;
+        rv[u].w = 0.f;
+      } else {
+        rv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const long long g = g0 + (long long)u * blockDim.x;
+      if (g < n4) dst[g] = xv[u];
+      if (g >= n4_full) {                               // padding of the column (and groups past the end) stay out of the sum
+        const long long i = g << 2;
+        if (i >= p.N) xv[u].x = 0.f;
+        if (i + 1 >= p.N) xv[u].y = 0.f;
+        if (i + 2 >= p.N) xv[u].z = 0.f;
+        xv[u].w = 0.f;
+      }
+      dot_step(xv[u].x, rv[u].x, h0, l0); dot_step(xv[u].y, rv[u].y, h1, l1);
+      dot_step(xv[u].z, rv[u].z, h0, l0); dot_step(xv[u].w, rv[u].w, h1, l1);
+    }
+  }
+  __shared__ double wsum[8];
+  double v = ((double)h0 + (double)l0) + ((double)h1 + (double)l1);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = v;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    double g = 0.0;
+    for (int w = 0; w < 8; ++w) g += wsum[w];
+    float b_new = b_old;
+    if (n > 0.0) {
+      const double z = (double)b_old + g / n;
+      const double m = fabs(z) - (double)p.lambda / n;
+      b_new = (float)(m <= 0.0 ? 0.0 : (z > 0.0 ? m : -m));
+    }
+    p.cand_bnew[a] = b_new;
+    p.cand_dbeta64[a] = isfinite(g) ? (double)b_new - (double)b_old : g - g;   // a non-finite product shows as NaN
+  }
 }
 
 template <bool k3x>
@@ -193,11 +276,6 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   unsigned char* tiles_ptr = dyn_smem + (tiles0 - smem_u32(dyn_smem));
   const uint32_t full0 = smem_u32(&bars[0]), empty0 = smem_u32(&bars[kStages]), done_bar = smem_u32(&bars[2 * kStages]);
 
-  if (tid < kTile) {
-    const int ga = ti * kTile + tid, gb = tj * kTile + tid;
-    normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
-    normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
-  }
   if (tid == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(full0 + 8 * s, kFullCount); mbar_init(empty0 + 8 * s, 1); }
     mbar_init(done_bar, 1);
@@ -346,6 +424,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 
   // ------------------------------ epilogue (warps 0..3: TMEM lanes 32 w .. 32 w + 31) ------------------------------
   if (warp < kProducerWarps) {
+    if (n_split == 1) {                                // (screen: while the main loop runs) the norms of the tile
+      const int ga = ti * kTile + tid, gb = tj * kTile + tid;
+      normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
+      normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps see all of them
+    }
     bool ok = !s_abort && mbar_wait(done_bar, 0u);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }

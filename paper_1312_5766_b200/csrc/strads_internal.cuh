@@ -91,6 +91,11 @@ struct Problem {
   int cap_amb;
   float* xc;                    // dense: packed copy of the candidate columns, [n_cand][ldc]
   long long ldc;                // N rounded up to a multiple of 4
+  // dense, one scheduler: the pack kernel also forms x_c^T r and with it the change every candidate would
+  // make if kept (valid while r is untouched between the pack and the update: same stream, same round)
+  int proposals;                // 1: the pack kernel fills the two arrays below and the update applies them
+  double* cand_dbeta64;         // [n_cand] proposed change of candidate position a
+  float* cand_bnew;             // [n_cand] proposed new beta
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
   float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
   int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles

@@ -107,42 +107,59 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
   }
 }
 
-// r <- r - sum_a x_a dbeta_a with every row owned by one CTA: 64 rows per CTA, a half-warp per column
-// (16 lanes x float4), so a warp reads two columns per instruction and the 16 half-warps of the CTA take the
-// kept columns round-robin, four loads in flight each.  The per-row sums of the half-warps are added in a
-// fixed order.
-constexpr int kRowsPerCta = 64;
-constexpr int kColSlots = kThreads / 16;   // half-warps per CTA
+// r <- r - sum_a x_a dbeta_a with every row owned by one CTA: 32 rows per CTA, a quarter-warp per column
+// (8 lanes x float4 = one 128-byte line), so a warp reads four columns per instruction and the 32 quarter-warps
+// of the CTA take the kept columns round-robin, eight loads in flight each.  The kept columns' addresses and
+// changes are staged in shared memory first, so the column loads depend on nothing.  The per-row sums of the
+// quarter-warps are added in a fixed order.
+// proposals = 1: the changes were formed by the pack kernel for every candidate (cand_dbeta64 / cand_bnew by
+// position in the list, src.index = positions of the kept ones); this kernel then also does the bookkeeping of
+// the kept coefficients (beta, delta, dbeta), spread over its CTAs.  Nothing here reads beta or delta.
+constexpr int kRowsPerCta = 32;
+constexpr int kColSlots = kThreads / 8;    // quarter-warps per CTA
+constexpr int kStageCols = 2048;           // kept columns staged per pass (24 KB of shared memory)
 
-__global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSource src, int advance) {
+__global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* __restrict__ kept, ColumnSource src,
+                                                          int advance, int proposals) {
   chain_begin();
   __shared__ double part[kColSlots][kRowsPerCta];
+  __shared__ double s_d[kStageCols];
+  __shared__ long long s_off[kStageCols];
   const int n_kept = p.st->counts[2];
-  const int slot = threadIdx.x >> 4, l16 = threadIdx.x & 15;
-  const long long i = (long long)blockIdx.x * kRowsPerCta + l16 * 4;
+  const int slot = threadIdx.x >> 3, l8 = threadIdx.x & 7;
+  const long long i = (long long)blockIdx.x * kRowsPerCta + l8 * 4;
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-  if (i < p.N) {
-    for (int a0 = slot; a0 < n_kept; a0 += kColSlots * 4) {
-      float4 xv[4];
-      double d[4];
+  for (int base = 0; base < n_kept; base += kStageCols) {
+    const int n_here = min(kStageCols, n_kept - base);
+    if (base > 0) __syncthreads();
+    for (int a = threadIdx.x; a < n_here; a += kThreads) {
+      const int idx = src.index[base + a];
+      s_off[a] = (long long)idx * src.pitch;
+      s_d[a] = proposals ? p.cand_dbeta64[idx] : p.dbeta64[base + a];
+    }
+    __syncthreads();
+    if (i < p.N) {
+      for (int a0 = slot; a0 < n_here; a0 += kColSlots * 8) {
+        float4 xv[8];
+        double d[8];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int a = a0 + u * kColSlots;
-        d[u] = a < n_kept ? p.dbeta64[a] : 0.0;
-        const int ai = a < n_kept ? a : a0;
-        xv[u] = __ldg(reinterpret_cast<const float4*>(src.base + (long long)src.index[ai] * src.pitch + i));
-      }
+        for (int u = 0; u < 8; ++u) {
+          const int a = a0 + u * kColSlots;
+          d[u] = a < n_here ? s_d[a] : 0.0;
+          xv[u] = __ldg(reinterpret_cast<const float4*>(src.base + s_off[a < n_here ? a : a0] + i));
+        }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        if (d[u] != 0.0) {
-          s0 += (double)xv[u].x * d[u]; s1 += (double)xv[u].y * d[u];
-          s2 += (double)xv[u].z * d[u]; s3 += (double)xv[u].w * d[u];
+        for (int u = 0; u < 8; ++u) {
+          if (d[u] != 0.0) {
+            s0 += (double)xv[u].x * d[u]; s1 += (double)xv[u].y * d[u];
+            s2 += (double)xv[u].z * d[u]; s3 += (double)xv[u].w * d[u];
+          }
         }
       }
     }
   }
-  part[slot][l16 * 4 + 0] = s0; part[slot][l16 * 4 + 1] = s1;
-  part[slot][l16 * 4 + 2] = s2; part[slot][l16 * 4 + 3] = s3;
+  part[slot][l8 * 4 + 0] = s0; part[slot][l8 * 4 + 1] = s1;
+  part[slot][l8 * 4 + 2] = s2; part[slot][l8 * 4 + 3] = s3;
   __syncthreads();
   if (threadIdx.x < kRowsPerCta) {
     const long long r = (long long)blockIdx.x * kRowsPerCta + threadIdx.x;
@@ -153,9 +170,26 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, ColumnSourc
       if (s != 0.0) p.resid[r] = (float)((double)p.resid[r] - s);
     }
   }
+  DeviceState* st = p.st;
+  if (proposals) {
+    for (int a = blockIdx.x * kThreads + threadIdx.x; a < p.n_keep; a += gridDim.x * kThreads) {
+      if (a >= n_kept) { p.dbeta[a] = 0.f; continue; }
+      const int pos = src.index[a], j = kept[a];
+      const double d = p.cand_dbeta64[pos];
+      p.beta[j] = p.cand_bnew[pos];
+      p.delta[j] = (float)fabs(d);
+      p.dbeta[a] = (float)d;
+      p.dbeta64[a] = d;
+      if (d != 0.0) {                                    // counted here and in the running total: CTA 0 may be done already
+        atomicAdd(&st->counts[3], 1);
+        if (advance) atomicAdd(&st->totals[3], 1ull);
+      }
+      if (!isfinite(d)) atomicOr(&st->status, STRADS_STATUS_NONFINITE);
+    }
+  }
   if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
-    DeviceState* st = p.st;
-    st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2]; st->totals[3] += st->counts[3];
+    st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2];
+    if (!proposals) st->totals[3] += st->counts[3];
     st->round += (unsigned long long)p.part_count;       // this scheduler's next turn
   }
 }
@@ -263,8 +297,11 @@ cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool f
     if (from_packed) { src.base = p.xc; src.pitch = p.ldc; src.index = p.kept_pos; }
     else { src.base = p.xv; src.pitch = p.ld; src.index = kept; }
     cudaError_t e;
-    if ((e = launch_chained(k_dot_dense, dim3(p.dot_parts, p.n_keep), kThreads, 0, s, p, kept, src)) != cudaSuccess) return e;
-    return launch_chained(k_apply_dense, (unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s, p, src, advance);
+    const int proposals = from_packed && p.proposals ? 1 : 0;     // the pack kernel of this round left the changes
+    if (!proposals && (e = launch_chained(k_dot_dense, dim3(p.dot_parts, p.n_keep), kThreads, 0, s, p, kept, src)) != cudaSuccess)
+      return e;
+    return launch_chained(k_apply_dense, (unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s, p, kept, src,
+                          advance, proposals);
   } else {
     cudaError_t e;
     if ((e = launch_chained(k_dot_csc, (p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, kept)) != cudaSuccess) return e;
