@@ -356,6 +356,9 @@ def main():
         tiles = nt * (nt + 1) // 2
         return 3 + (1 if tiles * 2 <= 148 else 0) + (0 if retry_follows else 1)
     launches_per_round = 2 + (1 if p.n_cols >= (1 << 22) else 0) + (1 if p.n_candidates <= 2048 else 2) + (1 if p.layout == wl.DENSE else 3)
+    sampling_ahead = p.layout == wl.DENSE and p.n_keep <= 4096
+    if sampling_ahead:
+        launches_per_round += 1        # the early list's correction; the early draw itself launches what a plain draw does
     if window < p.n_candidates:
         launches_per_round += gram_launches(window, True) + 1
         launches_per_round += (gram_launches(p.n_candidates, False) + 1) if p.layout == wl.DENSE else 1
@@ -375,7 +378,10 @@ def main():
             "objective": objective, "status_bits": status_bits,
             "step_ms": step_ms, "step_ms_rounds": prof["rounds"],
             "step_ms_note": "device time per step over the rounds right after the timed region, launched kernel by "
-                            "kernel with CUDA events between steps (the timed region itself replays a CUDA graph)",
+                            "kernel with CUDA events between steps (the timed region itself replays a CUDA graph"
+                            + (", in which the draw of the next round runs beside the Gram and walk on a second "
+                               "stream, so sample_ms is not on its critical path)" if sampling_ahead else ")"),
+            "sampling_ahead": sampling_ahead,
             "roofline": roofline,
             "update_hbm": {"achieved": upd_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                            "frac": upd_gbs / peaks["hbm_gbs"], "bytes_per_round": upd_bytes},

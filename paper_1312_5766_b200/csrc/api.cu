@@ -36,12 +36,21 @@ struct strads_lasso_s {
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
   cudaEvent_t fork;          // S > 1: where the schedulers' streams join the caller's stream
+  // Sampling ahead (one scheduler; strads_run only): the draw of round t + 1 runs on its own stream beside the Gram
+  // and walk of round t, and the round then starts from that list corrected for round t's update.
+  bool ahead_ok;             // the configuration allows it
+  Problem ahead;             // the early draw's view of the problem: own sampler state and buffers, P' + P winners
+  cudaStream_t ahead_stream;
+  cudaEvent_t ahead_fork, ahead_done;
+  long long ahead_round;     // the round whose early list is in place (-1: none)
 };
 
 namespace {
 
 constexpr int kProfEvents = 6;   // per round: start, after sample, pack, Gram, walk, update
 constexpr int kGraphTurns = 16;  // S > 1: turns of every scheduler in the captured sequence
+constexpr int kGraphRoundsAhead = 8;  // one scheduler, sampling ahead: rounds in the captured sequence
+constexpr int kAheadMaxKeep = 4096;   // sampling ahead: the patch kernel holds 2 P keys in shared memory
 
 Scheduler& on_turn(strads_lasso_s* h) { return h->sch[h->round_host % h->n_sched]; }
 
@@ -63,8 +72,9 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, total;
-  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap;
+      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev,
+      off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
+  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary;
   long long ldc;
 };
 
@@ -134,6 +144,20 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_bucket_items = take(buckets ? sizeof(int) * (size_t)c->n_rows * kBucketSlots : 0);
   L.off_pairs = take(sizeof(unsigned int) * (size_t)L.pair_cap);
   L.off_resid_acc = take(csc ? sizeof(long long) * (size_t)c->n_rows : 0);
+  L.off_delta_prev = take(sizeof(float) * (size_t)c->n_keep);
+  // sampling ahead (one scheduler, P <= kAheadMaxKeep): a second set of sampler buffers for P' + P winners.
+  // Dense layouts only: measured on CSC workloads, whose rounds contain a cooperative kernel, a draw running
+  // beside the round made it slower (c4: 140 -> 203 us), not faster.
+  const bool ahead = first && n_sched_of(c) == 1 && c->n_keep <= kAheadMaxKeep && c->layout == STRADS_DENSE_COLMAJOR;
+  const long long n_ahead = (long long)c->n_candidates + c->n_keep < c->n_cols ? (long long)c->n_candidates + c->n_keep : c->n_cols;
+  L.n_ahead = ahead ? (int)n_ahead : 0;
+  L.cap_ahead_boundary = ahead ? pow2_ceil(L.n_ahead / 2 > 2048 ? L.n_ahead / 2 : 2048) : 0;
+  L.off_ahead_state = take(ahead ? sizeof(DeviceState) : 0);
+  L.off_ahead_hist = take(ahead ? sizeof(unsigned int) * kHistBins : 0);
+  L.off_ahead_sure = take(sizeof(unsigned long long) * (size_t)L.n_ahead);
+  L.off_ahead_boundary = take(sizeof(unsigned long long) * (size_t)L.cap_ahead_boundary);
+  L.off_ahead_keys = take(sizeof(unsigned long long) * (size_t)L.n_ahead);
+  L.off_ahead_idx = take(sizeof(int) * (size_t)L.n_ahead);
   L.total = o;
   return L;
 }
@@ -197,6 +221,7 @@ bool update_reads_packed(const Problem& p, bool gram_exported) {
 
 // One round, every step on the caller's stream, by the scheduler whose turn it is.
 int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
+  h->ahead_round = -1;                                 // delta changes without a new early list
   const Scheduler& sc = on_turn(h);
   const Problem& p = sc.p;
   cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + kProfEvents * h->prof_rounds : nullptr;
@@ -216,6 +241,27 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
     if (out->cand) CK(cudaMemcpyAsync(out->cand, p.cand, sizeof(int) * p.n_cand, cudaMemcpyDeviceToDevice, h->stream));
     if (out->kept || out->dbeta || out->counts) CK(launch_export(p, p.kept, out->kept, out->dbeta, out->counts, h->stream));
   }
+  return STRADS_OK;
+}
+
+// One round of strads_run with one scheduler, sampling ahead.  `main`: candidates (from the early list if there
+// is one for this round, else a draw made now), Gram, walk, update; `ahead_stream`: the early draw of the next
+// round, which reads delta and so lies between this round's candidates and its update.
+int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
+  const Scheduler& sc = h->sch[0];
+  const Problem& p = sc.p;
+  if (have_list) CK(launch_sample_patch(p, h->ahead, p.cand, main));
+  else CK(launch_sample(p, p.cand, main));
+  CK(cudaEventRecord(h->ahead_fork, main));
+  CK(cudaStreamWaitEvent(h->ahead_stream, h->ahead_fork, 0));
+  CK(launch_sample(h->ahead, h->ahead.cand, h->ahead_stream));
+  CK(cudaEventRecord(h->ahead_done, h->ahead_stream));
+  const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr);
+  if (rc) return rc;
+  CK(cudaStreamWaitEvent(main, h->ahead_done, 0));
+  CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+  h->round_host += 1;
+  h->ahead_round = h->round_host;
   return STRADS_OK;
 }
 
@@ -294,6 +340,24 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.partial_tiles = L.partial_tiles;
   p.part_count = S; p.part_index = s;
   p.sm_count = first ? first->sm_count : 0;
+  p.round_ptr = &p.st->round; p.round_ahead = 0;
+  p.keys_out = nullptr;
+  p.delta_prev = reinterpret_cast<float*>(ws + L.off_delta_prev);
+}
+
+// The early draw's view: everything of scheduler 0, except its own sampler state and buffers, P' + P winners with
+// their keys, and the round index one ahead of the round in progress.
+void fill_ahead(Problem& a, const Problem& p0, const Layout& L, char* ws) {
+  a = p0;
+  a.st = reinterpret_cast<DeviceState*>(ws + L.off_ahead_state);
+  a.hist = reinterpret_cast<unsigned int*>(ws + L.off_ahead_hist);
+  a.sure = reinterpret_cast<unsigned long long*>(ws + L.off_ahead_sure);
+  a.boundary = reinterpret_cast<unsigned long long*>(ws + L.off_ahead_boundary);
+  a.cap_sure = L.n_ahead; a.cap_boundary = L.cap_ahead_boundary;
+  a.n_cand = L.n_ahead;
+  a.cand = reinterpret_cast<int*>(ws + L.off_ahead_idx);
+  a.keys_out = reinterpret_cast<unsigned long long*>(ws + L.off_ahead_keys);
+  a.round_ptr = &p0.st->round; a.round_ahead = 1;
 }
 
 void release(strads_lasso_s* h) {
@@ -303,6 +367,9 @@ void release(strads_lasso_s* h) {
     if (h->sch[s].updated != nullptr) cudaEventDestroy(h->sch[s].updated);
   }
   if (h->fork != nullptr) cudaEventDestroy(h->fork);
+  if (h->ahead_stream != nullptr) cudaStreamDestroy(h->ahead_stream);
+  if (h->ahead_fork != nullptr) cudaEventDestroy(h->ahead_fork);
+  if (h->ahead_done != nullptr) cudaEventDestroy(h->ahead_done);
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
   if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
   if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
@@ -362,6 +429,18 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
   if ((e = launch_init(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
   if ((e = launch_resid_from_beta(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
+  h->ahead_round = -1;
+  h->ahead_ok = L.n_ahead > 0;
+  if (h->ahead_ok) {
+    fill_ahead(h->ahead, p0, L, ws);
+    if ((e = launch_init_scheduler(h->ahead, p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init_scheduler"));
+    int prio_least = 0, prio_greatest = 0;             // the early draw yields to the round's own kernels
+    if ((e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest)) != cudaSuccess) return fail(cuda_fail(e, "priority range"));
+    if ((e = cudaStreamCreateWithPriority(&h->ahead_stream, cudaStreamNonBlocking, prio_least)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->ahead_fork, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->ahead_done, cudaEventDisableTiming)) != cudaSuccess)
+      return fail(cuda_fail(e, "sampling-ahead stream"));
+  }
   for (int s = 0; s < S; ++s) {
     Scheduler& sc = h->sch[s];
     if (sc.p.layout == STRADS_DENSE_COLMAJOR && (e = encode_gram_tensor_map(sc.p, sc.gram_tmap)) != cudaSuccess)
@@ -397,21 +476,35 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out) {
 }
 
 // Rounds that one launch of the captured sequence runs.
-static long long graph_rounds(const strads_lasso_s* h) { return h->n_sched > 1 ? (long long)kGraphTurns * h->n_sched : 1; }
+static long long graph_rounds(const strads_lasso_s* h) {
+  return h->n_sched > 1 ? (long long)kGraphTurns * h->n_sched : (h->ahead_ok ? kGraphRoundsAhead : 1);
+}
 
 // Captures the launch sequence of graph_rounds() rounds into a graph (on a private stream: the caller's may be
 // the legacy default stream, which cannot be captured; nothing executes during capture).  With several
 // schedulers the sequence starts with scheduler 0.
 static int build_round_graph(strads_lasso_s* h) {
-  CK(cudaStreamCreateWithFlags(&h->capture_stream, cudaStreamNonBlocking));
+  {
+    int prio_least = 0, prio_greatest = 0;
+    CK(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
+    CK(cudaStreamCreateWithPriority(&h->capture_stream, cudaStreamNonBlocking, prio_greatest));
+  }
   cudaStream_t user = h->stream;
   const long long round_before = h->round_host;
   h->stream = h->capture_stream;
   cudaError_t e = cudaStreamBeginCapture(h->capture_stream, cudaStreamCaptureModeThreadLocal);
   int rc = STRADS_OK;
   if (e == cudaSuccess) {
-    rc = h->n_sched > 1 ? pipelined_rounds(h, graph_rounds(h), h->capture_stream) : one_round(h, nullptr);
+    const long long ahead_before = h->ahead_round;
+    if (h->n_sched > 1) {
+      rc = pipelined_rounds(h, graph_rounds(h), h->capture_stream);
+    } else if (h->ahead_ok) {
+      for (long long i = 0; i < graph_rounds(h) && rc == STRADS_OK; ++i) rc = round_sampling_ahead(h, true, h->capture_stream);
+    } else {
+      rc = one_round(h, nullptr);
+    }
     e = cudaStreamEndCapture(h->capture_stream, &h->round_graph);
+    h->ahead_round = ahead_before;
   }
   h->stream = user;
   h->round_host = round_before;
@@ -451,8 +544,20 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
     const int rc = build_round_graph(h);
     if (rc) return rc;
   }
+  const long long R = graph_rounds(h);
   for (int64_t i = 0; i < n_rounds; ++i) {
-    if (use_graph) {
+    if (use_graph && h->ahead_ok) {
+      const bool have_list = h->ahead_round == h->round_host;
+      if (have_list && n_rounds - i >= R) {            // the early list of this round is in place: captured rounds
+        CK(cudaGraphLaunch(h->round_exec, h->stream));
+        h->round_host += R;
+        h->ahead_round = h->round_host;
+        i += R - 1;
+      } else {                                         // first round of a run (draw now, start drawing ahead), last few
+        const int rc = round_sampling_ahead(h, have_list, h->stream);
+        if (rc) return rc;
+      }
+    } else if (use_graph) {
       CK(cudaGraphLaunch(h->round_exec, h->stream));
       h->round_host += 1;
     } else {
@@ -501,6 +606,7 @@ int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand, in
   if (h == nullptr || cand_dev == nullptr || kept_dev == nullptr) return STRADS_ERR_INVALID_ARG;
   const Scheduler& sc = on_turn(h);
   if (n_cand < 0 || n_cand > sc.p.n_cand) return STRADS_ERR_INVALID_ARG;
+  h->ahead_round = -1;                                 // (the early list is corrected from the last round's kept list)
   CK(launch_set_counts(sc.p, n_cand, 0, 0, h->stream));
   const int rc = gram_and_filter(sc, h->stream, cand_dev, n_cand, gram_dev_or_null);
   if (rc) return rc;
@@ -512,6 +618,7 @@ int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, fl
   if (h == nullptr) return STRADS_ERR_INVALID_ARG;
   const Problem& p = on_turn(h).p;
   if (n_kept < 0 || n_kept > p.n_keep || (n_kept > 0 && kept_dev == nullptr)) return STRADS_ERR_INVALID_ARG;
+  h->ahead_round = -1;
   CK(launch_set_counts(p, n_kept, n_kept, n_kept, h->stream));
   if (n_kept > 0)
     CK(cudaMemcpyAsync(p.kept, kept_dev, sizeof(int) * n_kept, cudaMemcpyDeviceToDevice, h->stream));
@@ -529,6 +636,7 @@ int strads_get_round(strads_handle_t h, int64_t* t) {
 int strads_set_round(strads_handle_t h, int64_t t) {
   if (h == nullptr || t < 0) return STRADS_ERR_INVALID_ARG;
   h->round_host = t;
+  h->ahead_round = -1;
   unsigned long long next[STRADS_MAX_SCHEDULERS];          // every scheduler's next turn at or after t
   for (int s = 0; s < h->n_sched; ++s) {
     next[s] = (unsigned long long)t + (unsigned long long)(((s - t % h->n_sched) + h->n_sched) % h->n_sched);

@@ -172,7 +172,7 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
   const int tid = threadIdx.x;
   for (int b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
   __syncthreads();
-  const unsigned long long t = p.st->round;
+  const unsigned long long t = *p.round_ptr + (unsigned long long)p.round_ahead;
   const long long groups = (p.J + 3) >> 2;
   const float cut = mode == 1 ? p.st->t_cut : 0.f;
   const unsigned int cut_bin = cut > 0.f ? (__float_as_uint(cut) >> (32 - kHistBits)) : (unsigned)kHistBins;   // bins below it are complete
@@ -273,7 +273,7 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
 __global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
   chain_begin();
   const SelectState sel = p.st->sel;
-  const unsigned long long t = p.st->round;
+  const unsigned long long t = *p.round_ptr + (unsigned long long)p.round_ahead;
   const long long groups = (p.J + 3) >> 2;
   const int shift = 64 - sel.bits;
   // keys certainly above the boundary's upper edge are not computed
@@ -388,8 +388,8 @@ __global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
     r0 += count_less(other, n, k0);
     r1 += count_less(other, n, k1);
   }
-  if (i0 < ch.n && r0 < p.n_cand) cand_out[r0] = (int)(k0 & 0xffffffffull);
-  if (i1 < ch.n && r1 < p.n_cand) cand_out[r1] = (int)(k1 & 0xffffffffull);
+  if (i0 < ch.n && r0 < p.n_cand) { cand_out[r0] = (int)(k0 & 0xffffffffull); if (p.keys_out) p.keys_out[r0] = k0; }
+  if (i1 < ch.n && r1 < p.n_cand) { cand_out[r1] = (int)(k1 & 0xffffffffull); if (p.keys_out) p.keys_out[r1] = k1; }
 }
 
 // Small P': the order of the winners straight from the definition, with no sort.  The rank of a key is the
@@ -421,17 +421,90 @@ __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand
   below += __shfl_xor_sync(0xffffffffu, below, 2);
   below += __shfl_xor_sync(0xffffffffu, below, 4);
   const int rank = below + (is_sure ? 0 : n_sure);
-  if (slice == 0 && k < total && rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
+  if (slice == 0 && k < total && rank < p.n_cand) {
+    cand_out[rank] = (int)(key & 0xffffffffull);
+    if (p.keys_out) p.keys_out[rank] = key;
+  }
+}
+
+// Sampling ahead.  The draw of round t is made during round t - 1 (beside its Gram and walk) from the delta of
+// that round's start, for P' + P winners instead of P'; the update of round t - 1 then changes delta for at most P
+// coefficients.  Every other coefficient keeps its key, and one of them that belongs to the true P' smallest has
+// fewer than P' + P keys below it in the early ranking, so it is on the early list L.  The candidates are
+// therefore the P' smallest of (L without the updated coefficients) + (the updated coefficients with their new
+// keys): exactly the list a draw made now would give.  Rank of an element of L at index i:
+// i - #(old keys of updated coefficients below it) + #(new keys below it); of a new key: its insertion point in L
+// instead of i.  (An old key below an element of L is itself on L, L being a prefix of the full ranking; a new key
+// beyond the end of a list shorter than J ranks >= P' and is left out.)  A thread per element; the <= P old and
+// new keys are recomputed by every CTA into shared memory and counted against by brute force.
+__global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned long long* __restrict__ list, int n_list,
+                                                      int* __restrict__ cand_out) {
+  chain_begin();
+  extern __shared__ unsigned long long s_keys[];       // [n_keep] old keys, then [n_keep] new keys
+  const int nk = p.st->counts[2];                      // coefficients the last update touched
+  unsigned long long* old_k = s_keys;
+  unsigned long long* new_k = s_keys + p.n_keep;
+  const unsigned long long t = *p.round_ptr + (unsigned long long)p.round_ahead;
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  for (int a = threadIdx.x; a < nk; a += 256) {
+    const uint32_t j = (uint32_t)p.kept[a];
+    uint32_t w[4];
+    philox4x32_10(j >> 2, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
+    const uint32_t word = w[j & 3u];
+    old_k[a] = race_key64(p.delta_prev[a], p.eta, word, j, uniform);
+    new_k[a] = race_key64(p.delta[j], p.eta, word, j, uniform);
+  }
+  __syncthreads();
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
+  const int item = blockIdx.x * 256 + threadIdx.x;
+  unsigned long long key;
+  int at;                                              // elements of L below the key
+  if (item < n_list) {
+    key = list[item];
+    at = item;
+  } else if (item - n_list < nk) {
+    key = new_k[item - n_list];
+    int lo = 0, hi = n_list;
+    while (lo < hi) {
+      const int mid = (lo + hi) >> 1;
+      if (list[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    if (lo == n_list && (long long)n_list < p.J) return;
+    at = lo;
+  } else {
+    return;
+  }
+  int below_old = 0, below_new = 0;
+  bool is_old = false;
+  for (int a = 0; a < nk; ++a) {
+    const unsigned long long o = old_k[a];
+    below_old += o < key;
+    is_old |= o == key;
+    below_new += new_k[a] < key;
+  }
+  if (item < n_list && is_old) return;                 // an updated coefficient: its new key stands in for it
+  const int rank = at - below_old + below_new;
+  if (rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
 }
 
 }  // namespace
 
-cudaError_t prepare_sample(const Problem&) { return cudaSuccess; }
+// Kernel-wide attribute: the patch kernel's key arrays (sampling ahead is used up to P = 4096: 64 KB).
+cudaError_t prepare_sample(const Problem&) {
+  return cudaFuncSetAttribute(k_sample_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 8 * 4096);
+}
+
+cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s) {
+  const int items = ahead.n_cand + p.n_keep;
+  return launch_chained(k_sample_patch, (items + 255) / 256, 256, 2 * sizeof(unsigned long long) * (size_t)p.n_keep, s, p,
+                        (const unsigned long long*)ahead.keys_out, ahead.n_cand, cand_out);
+}
 
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   const long long groups = (p.J + 3) >> 2;
   long long blocks = (groups + kThreads - 1) / kThreads;
-  const long long cap = (long long)p.sm_count * 8;
+  // (an early draw runs beside the round's Gram and walk and leaves them most of every SM)
+  const long long cap = (long long)p.sm_count * (p.round_ahead ? 2 : 8);
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   cudaError_t e;
@@ -530,5 +603,6 @@ extern "C" int strads_sample_static(const float* delta_dev, int64_t n_cols, floa
   p.cap_sure = n_candidates;
   p.cap_boundary = STRADS_STATIC_MAX_CANDIDATES / 2;
   p.sm_count = sms;
+  p.round_ptr = &sc->st.round;
   return launch_sample(p, cand_dev, s) == cudaSuccess ? STRADS_OK : STRADS_ERR_CUDA;
 }

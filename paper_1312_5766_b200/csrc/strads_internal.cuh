@@ -109,6 +109,12 @@ struct Problem {
   unsigned int* pair_list;      // [pair_cap] (a << 16 | b), a < b: positions of two candidates that share a row
   int pair_cap;
   int sm_count;
+  // sampling ahead (one scheduler): the draw of round t + 1 is made during round t from the priorities of its start
+  // and corrected for the coefficients that round t updates (k_sample_patch)
+  const unsigned long long* round_ptr;   // the sampler's round index is *round_ptr + round_ahead
+  int round_ahead;
+  unsigned long long* keys_out;          // sampler: if set, the winners' keys in rank order go here too
+  float* delta_prev;                     // [n_keep] delta of the kept coefficients before this round's update
   // scheduler threads: this Problem is scheduler part_index of part_count and owns { j : j mod part_count == part_index }
   int part_count, part_index;
 };
@@ -318,6 +324,9 @@ cudaError_t launch_init_scheduler(const Problem& p, const Problem& first, cudaSt
 cudaError_t launch_objective(const Problem& p, cudaStream_t s);
 cudaError_t prepare_sample(const Problem& p);
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
+// Candidates of the round at hand from a draw made one round ahead (`ahead`: its keys in rank order, ahead.n_cand of
+// them) and the coefficients the last update changed (p.kept, p.delta_prev, p.delta).
+cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s);
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_gram_dense_tc();
 cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);

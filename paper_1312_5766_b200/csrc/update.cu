@@ -38,6 +38,7 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
   }
   const double d = (double)b_new - (double)b_old;        // the change that beta (FP32) really makes
   p.beta[j] = b_new;
+  p.delta_prev[a] = p.delta[j];
   p.delta[j] = (float)fabs(d);
   p.dbeta[a] = (float)d;
   p.dbeta64[a] = d;
@@ -114,7 +115,7 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
 // quarter-warps are added in a fixed order.
 // proposals = 1: the changes were formed by the pack kernel for every candidate (cand_dbeta64 / cand_bnew by
 // position in the list, src.index = positions of the kept ones); this kernel then also does the bookkeeping of
-// the kept coefficients (beta, delta, dbeta), spread over its CTAs.  Nothing here reads beta or delta.
+// the kept coefficients (beta, delta, dbeta), spread over its CTAs.  No other thread reads beta or delta here.
 constexpr int kRowsPerCta = 32;
 constexpr int kColSlots = kThreads / 8;    // quarter-warps per CTA
 constexpr int kStageCols = 2048;           // kept columns staged per pass (24 KB of shared memory)
@@ -177,6 +178,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
       const int pos = src.index[a], j = kept[a];
       const double d = p.cand_dbeta64[pos];
       p.beta[j] = p.cand_bnew[pos];
+      p.delta_prev[a] = p.delta[j];
       p.delta[j] = (float)fabs(d);
       p.dbeta[a] = (float)d;
       p.dbeta64[a] = d;

@@ -500,3 +500,52 @@ def test_graph_replay_equals_round_by_round(name, n_keep, n_cand):
         assert torch.equal(x, y)
     assert a.totals() == b.totals() and a.totals()["kept"] == kept_total
     assert a.status()[0] == 0 and b.status()[0] == 0
+
+
+# --------------------------------------------------------------------------------------------------
+# sampling ahead: strads_run (one scheduler) draws the candidates of round t + 1 during round t and corrects the
+# list for the coefficients round t updates.  The result must be the list a draw made at the round's start
+# gives: state after mixed sequences of strads_run and other calls == the same rounds one by one (strads_round
+# draws at the round's start and is itself checked against the oracle above).
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("name,cfg_over,flags", [
+    ("dense", dict(n_cols=1500, n_candidates=256, n_keep=64), 0),          # the first sweep ends after ~24 rounds
+    ("dense", dict(n_cols=300, n_candidates=256, n_keep=64), 0),           # P' + P > J: the early list is everything
+    ("dense_grouped", dict(n_candidates=512, n_keep=120), 0),              # heavy rejection, whole-list retries
+    ("csc", dict(n_cols=6000, n_candidates=1000, n_keep=128), 0),
+    ("csc_zipf", dict(), 0),
+    ("dense", dict(n_cols=1500, n_candidates=256, n_keep=64), "uniform"),
+])
+def test_sampling_ahead_equals_round_by_round(name, cfg_over, flags):
+    b = _binding()
+    cfg = dict(_small_problems()[name], **cfg_over)
+    cfg["n_true"] = min(cfg["n_true"], cfg["n_cols"] // 10)
+    p = wl.make_problem(cfg, seed=21)
+    kw = dict(flags=b.FLAG_UNIFORM_DRAW) if flags == "uniform" else {}
+    a, ref = _solver(p, **kw), _solver(p, **kw)
+    done = 0
+
+    def check():
+        assert a.get_round() == ref.get_round() == done
+        for x, y in ((a.beta, ref.beta), (a.resid, ref.resid), (a.delta, ref.delta)):
+            assert torch.equal(x, y), (name, done)
+
+    # runs of several lengths; between them calls that leave the early list stale or unusable
+    for step in (3, 1, 40, "round", 2, "filter", 25, "set_round", 30, "round_host", 12):
+        if step == "round":
+            a.round(); n = 1
+        elif step == "filter":
+            a.filter(torch.arange(p.n_candidates, dtype=torch.int32, device="cuda")); n = 0   # overwrites kept / counts
+        elif step == "set_round":
+            a.set_round(done); n = 0
+        elif step == "round_host":
+            hb, hr, hd = (t.cpu().pin_memory() for t in (a.beta, a.resid, a.delta))
+            a.round_host(hb, hr, hd); n = 1
+        else:
+            a.run(step); n = step
+        for _ in range(n):
+            ref.round()
+        done += n
+        check()
+    assert a.totals() == ref.totals()
+    assert a.status()[0] == 0 and ref.status()[0] == 0
