@@ -50,6 +50,7 @@ namespace {
 constexpr int kProfEvents = 6;   // per round: start, after sample, pack, Gram, walk, update
 constexpr int kGraphTurns = 16;  // S > 1: turns of every scheduler in the captured sequence
 constexpr int kGraphRoundsAhead = 8;  // one scheduler, sampling ahead: rounds in the captured sequence
+constexpr int kEdgeCap = 8192;        // conflicting pairs the Gram kernels can list for the walk (32 KB)
 constexpr int kAheadMaxKeep = 4096;   // sampling ahead: the patch kernel holds 2 P keys in shared memory
 
 Scheduler& on_turn(strads_lasso_s* h) { return h->sch[h->round_host % h->n_sched]; }
@@ -72,7 +73,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev,
+      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary;
   long long ldc;
@@ -145,6 +146,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_pairs = take(sizeof(unsigned int) * (size_t)L.pair_cap);
   L.off_resid_acc = take(csc ? sizeof(long long) * (size_t)c->n_rows : 0);
   L.off_delta_prev = take(sizeof(float) * (size_t)c->n_keep);
+  L.off_edges = take(sizeof(unsigned int) * kEdgeCap);
   // sampling ahead (one scheduler, P <= kAheadMaxKeep): a second set of sampler buffers for P' + P winners.
   // Dense layouts only: measured on CSC workloads, whose rounds contain a cooperative kernel, a draw running
   // beside the round made it slower (c4: 140 -> 203 us), not faster.
@@ -343,6 +345,8 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.round_ptr = &p.st->round; p.round_ahead = 0;
   p.keys_out = nullptr;
   p.delta_prev = reinterpret_cast<float*>(ws + L.off_delta_prev);
+  p.edges = reinterpret_cast<unsigned int*>(ws + L.off_edges);
+  p.cap_edges = kEdgeCap;
 }
 
 // The early draw's view: everything of scheduler 0, except its own sampler state and buffers, P' + P winners with

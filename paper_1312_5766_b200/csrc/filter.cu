@@ -16,6 +16,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kRange = 64;                       // positions decided per step of the walk
+constexpr int kSparsePasses = 24;                // passes of the walk from the pair list before the bit rows take over
 constexpr size_t kResidentBytes = 200 * 1024;    // conflict rows of the whole list in shared memory up to this
 
 __host__ __device__ inline int words_of(int n_cand) { return (n_cand + 31) >> 5; }
@@ -33,11 +34,11 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
     // dense window whose TF32 screen left more borderline pairs than the list holds: its bits are incomplete;
     // the whole-list retry (which has the 3xTF32 fallback) takes over
-    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; }
+    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; p.st->edge_count = 0; p.st->edges_off = 0; }
     return;
   }
   if (p.layout == STRADS_CSC && n_cand < n_total && window_skipped(p)) {
-    if (threadIdx.x == 0) p.st->window_short = 1;    // window attempt skipped: go straight to the whole-list walk
+    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->edge_count = 0; p.st->edges_off = 0; }   // window attempt skipped: go straight to the whole-list walk
     return;
   }
   extern __shared__ unsigned int sm[];
@@ -50,34 +51,108 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   __shared__ int s_kept, s_examined, s_done;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
-  for (int w = tid; w < Wn + 2; w += kThreads) blocked[w] = 0u;
   if (tid == 0) { s_kept = 0; s_examined = n_cand; s_done = 0; }
 
   if (p.flags & STRADS_FLAG_NO_FILTER) {
     const int nk = min(n_cand, p.n_keep);
     for (int i = tid; i < p.n_keep; i += kThreads) kept_out[i] = i < nk ? cand[i] : -1;
-    if (tid == 0) { p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; p.st->window_short = 0; }
+    if (tid == 0) {
+      p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; p.st->window_short = 0;
+      p.st->edge_count = 0; p.st->edges_off = 0;
+    }
     return;
   }
-  for (int i = tid; i < n_cand; i += kThreads) s_cand[i] = cand[i];
+
+  // ---- The walk from the list of conflicting pairs, when the Gram kernels listed all of them. ----
+  // Conflicts are few, so the first-fit rule "keep b unless an earlier kept a conflicts with it" is settled in
+  // passes over the pairs: a candidate with a kept earlier neighbour is out, one whose earlier neighbours are all
+  // decided and out is kept (a candidate without earlier neighbours at once).  The number of passes is the longest
+  // chain of such dependencies, two or three in practice; if it exceeds kSparsePasses the walk over the bit rows
+  // below takes over.  Stopping at P is a cut of the kept sequence at its P-th member: no decision depends on a
+  // later position.
+  bool settled = false;
+  const unsigned int n_edges = p.st->edge_count;
+  if (!p.st->edges_off && n_edges <= (unsigned)p.cap_edges) {
+    unsigned char* state = reinterpret_cast<unsigned char*>(sm);          // 0 undecided, 1 kept, 2 out
+    unsigned char* hit = state + ((n_cand + 15) & ~15);                   // has a kept earlier neighbour
+    unsigned char* pend = hit + ((n_cand + 15) & ~15);                    // has an undecided earlier neighbour
+    unsigned int* e = reinterpret_cast<unsigned int*>(pend + ((n_cand + 15) & ~15));
+    for (int i = tid; i < n_cand; i += kThreads) { state[i] = 0; hit[i] = 0; pend[i] = 0; }
+    for (unsigned int k = tid; k < n_edges; k += kThreads) e[k] = __ldcg(p.edges + k);
+    __syncthreads();
+    for (int pass = 0; pass < kSparsePasses && !settled; ++pass) {
+      for (unsigned int k = tid; k < n_edges; k += kThreads) {
+        const int a = (int)(e[k] >> 16), b = (int)(e[k] & 0xffffu);
+        if (state[b] == 0) {
+          const unsigned char sa = state[a];
+          if (sa == 1) hit[b] = 1;                     // (several threads may store the same value: benign)
+          else if (sa == 0) pend[b] = 1;
+        }
+      }
+      __syncthreads();
+      int open = 0;
+      for (int i = tid; i < n_cand; i += kThreads) {
+        if (state[i] == 0) {
+          if (hit[i]) state[i] = 2;
+          else if (!pend[i]) state[i] = 1;
+          else open = 1;
+          pend[i] = 0;
+        }
+      }
+      settled = __syncthreads_or(open) == 0;
+    }
+    if (settled) {
+      // kept members in order: thread t counts its contiguous chunk, the chunks are scanned, and every thread
+      // writes its kept members at their ranks, up to P
+      __shared__ int s_scan[kThreads];
+      const int chunk = (n_cand + kThreads - 1) / kThreads;
+      const int i0 = min(tid * chunk, n_cand), i1 = min(i0 + chunk, n_cand);
+      int mine = 0;
+      for (int i = i0; i < i1; ++i) mine += state[i] == 1;
+      s_scan[tid] = mine;
+      __syncthreads();
+      for (int o = 1; o < kThreads; o <<= 1) {
+        const int v = tid >= o ? s_scan[tid - o] : 0;
+        __syncthreads();
+        s_scan[tid] += v;
+        __syncthreads();
+      }
+      int rank = s_scan[tid] - mine;
+      const int total = s_scan[kThreads - 1];
+      for (int i = i0; i < i1 && rank < p.n_keep; ++i) {
+        if (state[i] == 1) {
+          kept_out[rank] = cand[i];
+          p.kept_pos[rank] = i;
+          if (rank == p.n_keep - 1) s_examined = i + 1;          // the walk stops here
+          ++rank;
+        }
+      }
+      if (tid == 0) s_kept = min(total, p.n_keep);
+    }
+    __syncthreads();
+  }
+
+  for (int w = tid; w < Wn + 2 && !settled; w += kThreads) blocked[w] = 0u;
+  const int n_rows = settled ? 0 : n_cand;             // (settled: nothing left for the walk over the bit rows)
+  for (int i = tid; i < n_rows; i += kThreads) s_cand[i] = cand[i];
   if (resident && (W & 3) == 0 && Wn <= 64) {
     // all rows at once, 128-bit loads: 8 or 16 lanes per row (one per group of four words), sixteen rows in
     // flight per thread, loads before stores
     const int quads = (Wn + 3) >> 2;                   // (W % 4 == 0: 4 * quads <= W)
     const int lpr_log = quads <= 8 ? 3 : 4, lpr = 1 << lpr_log;
     const int c = tid & (lpr - 1), rstep = kThreads >> lpr_log;
-    for (int r0 = tid >> lpr_log; r0 < n_cand; r0 += 16 * rstep) {
+    for (int r0 = tid >> lpr_log; r0 < n_rows; r0 += 16 * rstep) {
       uint4 v[16];
 #pragma unroll
       for (int u = 0; u < 16; ++u) {
         const int r = r0 + u * rstep;
         v[u] = make_uint4(0u, 0u, 0u, 0u);
-        if (r < n_cand && c < quads) v[u] = __ldcg(reinterpret_cast<const uint4*>(p.conflict + (long long)r * W) + c);
+        if (r < n_rows && c < quads) v[u] = __ldcg(reinterpret_cast<const uint4*>(p.conflict + (long long)r * W) + c);
       }
 #pragma unroll
       for (int u = 0; u < 16; ++u) {
         const int r = r0 + u * rstep;
-        if (r < n_cand && c < quads) {
+        if (r < n_rows && c < quads) {
           unsigned int* dst = rows + r * Wp + 4 * c;
           dst[0] = v[u].x;
           if (4 * c + 1 < Wn) dst[1] = v[u].y;
@@ -88,7 +163,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     }
   } else if (resident) {
     // all rows at once: independent loads, eight in flight per thread, before any store
-    const int total = n_cand * Wn;
+    const int total = n_rows * Wn;
     for (int i0 = tid; i0 < total; i0 += 8 * kThreads) {
       unsigned int v[8];
       int at[8];
@@ -106,7 +181,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   }
   __syncthreads();
 
-  for (int cur = 0; cur < n_cand; cur += kRange) {
+  for (int cur = 0; cur < n_rows; cur += kRange) {
     const int m = min(kRange, n_cand - cur);
     const int w0 = cur >> 5;                           // even: the range is words w0, w0 + 1 of every mask
     const unsigned long long valid = m >= 64 ? ~0ull : ((1ull << m) - 1ull);
@@ -245,6 +320,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   for (int i = nk + tid; i < p.n_keep; i += kThreads) kept_out[i] = -1;
   if (tid == 0) {
     p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0;
+    p.st->edge_count = 0; p.st->edges_off = 0;         // the next Gram starts a new list
     p.st->window_short = (!only_if_short && nk < p.n_keep && n_cand < n_total) ? 1 : 0;
     if (!only_if_short && n_cand < n_total) {          // a window attempt: remember how it went
       if (p.st->window_short) p.st->walk_streak = min(p.st->walk_streak + 1, 16);
@@ -273,7 +349,9 @@ cudaError_t prepare_filter(const Problem&) {
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s) {
   bool resident;
-  const size_t smem = filter_smem_bytes(n_cand, &resident);
+  size_t smem = filter_smem_bytes(n_cand, &resident);
+  const size_t sparse = 3 * (((size_t)n_cand + 15) & ~(size_t)15) + sizeof(unsigned int) * (size_t)p.cap_edges;   // walk from the pair list
+  if (smem < sparse) smem = sparse;
   return launch_chained(k_filter, 1, kThreads, smem, s, p, cand, n_cand, n_total, only_if_short ? 1 : 0, resident ? 1 : 0,
                         kept_out);
 }

@@ -110,8 +110,10 @@ __global__ void __launch_bounds__(kThreads) k_csc_pair_bits(Problem p, const int
     const long long a0 = p.xptr[ja];
     const float dot = sparse_dot(p.xrow + a0, p.xv + a0, (int)(p.xptr[ja + 1] - a0), p, jb);
     const double den = sqrt(p.n2[ja] * p.n2[jb]);
-    if (den > 0.0 && fabs((double)dot) >= rho * den)
+    if (den > 0.0 && fabs((double)dot) >= rho * den) {
       atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+      list_conflict(p, a, b);                             // (a pair listed twice is listed twice here too: harmless)
+    }
   }
 }
 
@@ -127,6 +129,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
     if (blockIdx.x == 0 && threadIdx.x == 0 && used) p.st->bucket_avoid = failed;   // (nobody reads it in this kernel)
     if (used && !failed) return;
   }
+  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->edges_off = 1;     // this kernel sets bits without listing the pairs
   __shared__ int arow[kStage];
   __shared__ float aval[kStage];
   const int a = blockIdx.x;

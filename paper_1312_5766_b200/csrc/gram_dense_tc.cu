@@ -141,6 +141,7 @@ __device__ __forceinline__ uint32_t decide_word(const Problem& p, const uint32_t
       const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
       if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
     }
+    if (hit && b > a) list_conflict(p, a, b);
     word |= (uint32_t)hit << j;
   }
   return word;
@@ -512,6 +513,7 @@ __global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int 
       const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
       if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
     }
+    if (hit && b > a) list_conflict(p, a, b);
     nib |= (unsigned int)hit << k;
   }
   unsigned int word = nib << ((lane & 7) * 4);         // 8 lanes make one 32-column mask word
@@ -551,8 +553,10 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_sho
     for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
     if (lane == 0) {
       const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
-      if (den > 0.0 && fabs(acc) >= (double)p.rho * den)
+      if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
         atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+        list_conflict(p, a, b);
+      }
     }
   }
 }

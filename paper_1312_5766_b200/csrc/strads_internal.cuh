@@ -41,6 +41,8 @@ struct DeviceState {
   int sample_redo;              // sampler: the guided first pass found too few keys; the plain pass behind it runs
   int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
+  unsigned int edge_count;      // conflicting pairs listed by the Gram kernels of this round (may exceed the list)
+  int edges_off;                // a kernel that sets bits without listing pairs has run: the list is not complete
   unsigned int pad;
 };
 
@@ -115,10 +117,20 @@ struct Problem {
   int round_ahead;
   unsigned long long* keys_out;          // sampler: if set, the winners' keys in rank order go here too
   float* delta_prev;                     // [n_keep] delta of the kept coefficients before this round's update
+  // Conflicts are normally few (a handful per hundred candidates), so the Gram kernels also list the conflicting
+  // pairs (a << 16 | b, a < b, positions in the list) and the walk works from that list when it is complete.
+  unsigned int* edges;                   // [cap_edges]
+  int cap_edges;
   // scheduler threads: this Problem is scheduler part_index of part_count and owns { j : j mod part_count == part_index }
   int part_count, part_index;
 };
 static constexpr int kObjBlocks = 296;
+
+// A Gram kernel found candidates a < b (positions in the list) in conflict.
+__device__ __forceinline__ void list_conflict(const Problem& p, int a, int b) {
+  const unsigned int slot = atomicAdd(&p.st->edge_count, 1u);
+  if (slot < (unsigned)p.cap_edges) p.edges[slot] = ((unsigned int)a << 16) | (unsigned int)b;
+}
 
 // CSC: whether this round leaves the candidate window out and goes straight to the on-demand walk: after a
 // window that was too short, the next attempt comes 64 rounds (of this scheduler) later, and twice as late
