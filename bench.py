@@ -31,9 +31,9 @@ from paper_1312_5766_b200 import workloads as wl  # noqa: E402
 METRIC = "coordinate updates/sec and % of HBM roofline per STRADS round (1xB200)"
 UNIT = "coordinate updates/s"
 # DRAM bytes (read + write) per launch of the window-Gram kernels from ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum; profiles/k_gram_dense_tc_window_c2.md), keyed by (workload, window).  The capture was made
+# dram__bytes_write.sum; profiles/ncu_full_round_kernels_c2_J20000.md), keyed by (workload, window).  The capture was made
 # with J cut to 20,000; the window kernels read the packed window only, so their traffic does not depend on J.
-GRAM_WINDOW_TRAFFIC = {("c2", 512): 20.6e6}
+GRAM_WINDOW_TRAFFIC = {("c2", 512): 20.5e6}
 
 
 def measured_peaks():

@@ -42,6 +42,11 @@ struct strads_lasso_s {
   Problem ahead;             // the early draw's view of the problem: own sampler state and buffers, P' + P winners
   cudaStream_t ahead_stream;
   cudaEvent_t ahead_fork, ahead_done;
+  // ... and the whole-list retry of the dense Gram (launches that return at once unless the window was too short)
+  // goes to a branch of its own, ending in its own gated copy of the update, instead of standing between the
+  // window's walk and the update
+  cudaStream_t retry_stream;
+  cudaEvent_t retry_fork, retry_done;
   long long ahead_round;     // the round whose early list is in place (-1: none)
 };
 
@@ -191,8 +196,12 @@ int window_of(const Problem& p, int n_cand) {
   return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
 }
 
+// retry_stream (with retry_fork): where the whole-list retry of a dense window goes instead of `s`; *branched tells
+// the caller that it did, and that the update has to be enqueued on both streams, gated either way.
 int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, float* gram_dbg,
-                    cudaEvent_t after_pack = nullptr, cudaEvent_t after_gram = nullptr) {
+                    cudaEvent_t after_pack = nullptr, cudaEvent_t after_gram = nullptr, cudaStream_t retry_stream = nullptr,
+                    cudaEvent_t retry_fork = nullptr, bool* branched = nullptr) {
+  if (branched) *branched = false;
   const Problem& p = sc.p;
   if (p.flags & STRADS_FLAG_NO_FILTER) {
     if (after_pack) CK(cudaEventRecord(after_pack, s));
@@ -209,8 +218,15 @@ int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_
       // whole list, conflict rows formed only for the candidates the walk keeps
       CK(launch_walk_csc(p, cand, n_cand, sc.walk_grid, true, p.kept, s));
     } else {
-      CK(launch_gram(sc, s, cand, n_cand, nullptr, true));
-      CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, s));
+      cudaStream_t rs = s;
+      if (retry_stream != nullptr && branched != nullptr) {
+        CK(cudaEventRecord(retry_fork, s));
+        CK(cudaStreamWaitEvent(retry_stream, retry_fork, 0));
+        rs = retry_stream;
+        *branched = true;
+      }
+      CK(launch_gram(sc, rs, cand, n_cand, nullptr, true));
+      CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, rs));
     }
   }
   return STRADS_OK;
@@ -258,10 +274,21 @@ int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
   CK(cudaStreamWaitEvent(h->ahead_stream, h->ahead_fork, 0));
   CK(launch_sample(h->ahead, h->ahead.cand, h->ahead_stream));
   CK(cudaEventRecord(h->ahead_done, h->ahead_stream));
-  const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr);
+  const bool can_branch = update_reads_packed(p, false) && p.proposals;     // (the gated update is the single-kernel one)
+  bool branched = false;
+  const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr, nullptr, nullptr, can_branch ? h->retry_stream : nullptr,
+                                 h->retry_fork, &branched);
   if (rc) return rc;
   CK(cudaStreamWaitEvent(main, h->ahead_done, 0));
-  CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+  if (branched) {
+    CK(launch_update(p, p.kept, 1, true, main, 1));                          // runs if the window sufficed
+    CK(cudaStreamWaitEvent(h->retry_stream, h->ahead_done, 0));
+    CK(launch_update(p, p.kept, 1, true, h->retry_stream, 2));               // runs behind the retry otherwise
+    CK(cudaEventRecord(h->retry_done, h->retry_stream));
+    CK(cudaStreamWaitEvent(main, h->retry_done, 0));
+  } else {
+    CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+  }
   h->round_host += 1;
   h->ahead_round = h->round_host;
   return STRADS_OK;
@@ -374,6 +401,9 @@ void release(strads_lasso_s* h) {
   if (h->ahead_stream != nullptr) cudaStreamDestroy(h->ahead_stream);
   if (h->ahead_fork != nullptr) cudaEventDestroy(h->ahead_fork);
   if (h->ahead_done != nullptr) cudaEventDestroy(h->ahead_done);
+  if (h->retry_stream != nullptr) cudaStreamDestroy(h->retry_stream);
+  if (h->retry_fork != nullptr) cudaEventDestroy(h->retry_fork);
+  if (h->retry_done != nullptr) cudaEventDestroy(h->retry_done);
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
   if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
   if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
@@ -442,7 +472,10 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
     if ((e = cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest)) != cudaSuccess) return fail(cuda_fail(e, "priority range"));
     if ((e = cudaStreamCreateWithPriority(&h->ahead_stream, cudaStreamNonBlocking, prio_least)) != cudaSuccess ||
         (e = cudaEventCreateWithFlags(&h->ahead_fork, cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&h->ahead_done, cudaEventDisableTiming)) != cudaSuccess)
+        (e = cudaEventCreateWithFlags(&h->ahead_done, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaStreamCreateWithPriority(&h->retry_stream, cudaStreamNonBlocking, prio_least)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->retry_fork, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->retry_done, cudaEventDisableTiming)) != cudaSuccess)
       return fail(cuda_fail(e, "sampling-ahead stream"));
   }
   for (int s = 0; s < S; ++s) {

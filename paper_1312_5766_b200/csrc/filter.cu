@@ -321,7 +321,8 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   if (tid == 0) {
     p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0;
     p.st->edge_count = 0; p.st->edges_off = 0;         // the next Gram starts a new list
-    p.st->window_short = (!only_if_short && nk < p.n_keep && n_cand < n_total) ? 1 : 0;
+    // (the whole-list retry leaves the flag as the window's walk set it: kernels of a parallel branch may still read it)
+    if (!only_if_short) p.st->window_short = (nk < p.n_keep && n_cand < n_total) ? 1 : 0;
     if (!only_if_short && n_cand < n_total) {          // a window attempt: remember how it went
       if (p.st->window_short) p.st->walk_streak = min(p.st->walk_streak + 1, 16);
       else { p.st->prefer_walk = 0; p.st->walk_streak = 0; }

@@ -435,8 +435,8 @@ __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand
 // keys): exactly the list a draw made now would give.  Rank of an element of L at index i:
 // i - #(old keys of updated coefficients below it) + #(new keys below it); of a new key: its insertion point in L
 // instead of i.  (An old key below an element of L is itself on L, L being a prefix of the full ranking; a new key
-// beyond the end of a list shorter than J ranks >= P' and is left out.)  A thread per element; the <= P old and
-// new keys are recomputed by every CTA into shared memory and counted against by brute force.
+// beyond the end of a list shorter than J ranks >= P' and is left out.)  The <= P old and new keys are recomputed by
+// every CTA into shared memory and counted against by brute force.
 __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned long long* __restrict__ list, int n_list,
                                                       int* __restrict__ cand_out) {
   chain_begin();
@@ -456,23 +456,30 @@ __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned 
   }
   __syncthreads();
   if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
-  const int item = blockIdx.x * 256 + threadIdx.x;
+  // CTAs 0 .. list_ctas - 1: a thread per element of the list.  The CTAs behind them: a warp per new key, whose
+  // insertion point is counted over the whole list by the 32 lanes (independent, coalesced loads instead of the
+  // dependent probes of a binary search).
+  const int list_ctas = (n_list + 255) / 256;
   unsigned long long key;
   int at;                                              // elements of L below the key
-  if (item < n_list) {
+  bool from_list;
+  if ((int)blockIdx.x < list_ctas) {
+    const int item = blockIdx.x * 256 + threadIdx.x;
+    if (item >= n_list) return;
     key = list[item];
     at = item;
-  } else if (item - n_list < nk) {
-    key = new_k[item - n_list];
-    int lo = 0, hi = n_list;
-    while (lo < hi) {
-      const int mid = (lo + hi) >> 1;
-      if (list[mid] < key) lo = mid + 1; else hi = mid;
-    }
-    if (lo == n_list && (long long)n_list < p.J) return;
-    at = lo;
+    from_list = true;
   } else {
-    return;
+    const int a = ((int)blockIdx.x - list_ctas) * 8 + (int)(threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (a >= nk) return;
+    key = new_k[a];
+    int below = 0;
+    for (int i = lane; i < n_list; i += 32) below += list[i] < key;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
+    if (lane != 0 || (below == n_list && (long long)n_list < p.J)) return;
+    at = below;
+    from_list = false;
   }
   int below_old = 0, below_new = 0;
   bool is_old = false;
@@ -482,7 +489,7 @@ __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned 
     is_old |= o == key;
     below_new += new_k[a] < key;
   }
-  if (item < n_list && is_old) return;                 // an updated coefficient: its new key stands in for it
+  if (from_list && is_old) return;                     // an updated coefficient: its new key stands in for it
   const int rank = at - below_old + below_new;
   if (rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
 }
@@ -495,8 +502,8 @@ cudaError_t prepare_sample(const Problem&) {
 }
 
 cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s) {
-  const int items = ahead.n_cand + p.n_keep;
-  return launch_chained(k_sample_patch, (items + 255) / 256, 256, 2 * sizeof(unsigned long long) * (size_t)p.n_keep, s, p,
+  const int ctas = (ahead.n_cand + 255) / 256 + (p.n_keep + 7) / 8;      // list elements by thread, new keys by warp
+  return launch_chained(k_sample_patch, ctas, 256, 2 * sizeof(unsigned long long) * (size_t)p.n_keep, s, p,
                         (const unsigned long long*)ahead.keys_out, ahead.n_cand, cand_out);
 }
 

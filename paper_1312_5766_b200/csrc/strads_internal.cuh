@@ -356,7 +356,7 @@ cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int g
                             cudaStream_t s);
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s);
-cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s);
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s, int gate = 0);
 cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s);
 cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,
                           cudaStream_t s);

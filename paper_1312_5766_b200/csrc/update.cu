@@ -120,9 +120,12 @@ constexpr int kRowsPerCta = 32;
 constexpr int kColSlots = kThreads / 8;    // quarter-warps per CTA
 constexpr int kStageCols = 2048;           // kept columns staged per pass (24 KB of shared memory)
 
+// gate: 0 always; 1 only if the candidate window sufficed; 2 only if it did not (the update is then enqueued
+// twice, behind the window's walk and behind the whole-list retry on a branch of its own, and exactly one runs).
 __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* __restrict__ kept, ColumnSource src,
-                                                          int advance, int proposals) {
+                                                          int advance, int proposals, int gate) {
   chain_begin();
+  if (gate != 0 && (p.st->window_short != 0) != (gate == 2)) return;
   __shared__ double part[kColSlots][kRowsPerCta];
   __shared__ double s_d[kStageCols];
   __shared__ long long s_off[kStageCols];
@@ -293,17 +296,18 @@ __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta
 
 // from_packed: the kept columns are rows p.kept_pos[.] of the packed candidate buffer (dense, after a
 // tensor-core Gram of this round); otherwise they are read from X.
-cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s) {
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s, int gate) {
   if (p.layout == STRADS_DENSE_COLMAJOR) {
     ColumnSource src;
     if (from_packed) { src.base = p.xc; src.pitch = p.ldc; src.index = p.kept_pos; }
     else { src.base = p.xv; src.pitch = p.ld; src.index = kept; }
     cudaError_t e;
     const int proposals = from_packed && p.proposals ? 1 : 0;     // the pack kernel of this round left the changes
+    if (gate != 0 && !proposals) return cudaErrorInvalidValue;    // (only the single-kernel update is gated)
     if (!proposals && (e = launch_chained(k_dot_dense, dim3(p.dot_parts, p.n_keep), kThreads, 0, s, p, kept, src)) != cudaSuccess)
       return e;
     return launch_chained(k_apply_dense, (unsigned)((p.N + kRowsPerCta - 1) / kRowsPerCta), kThreads, 0, s, p, kept, src,
-                          advance, proposals);
+                          advance, proposals, gate);
   } else {
     cudaError_t e;
     if ((e = launch_chained(k_dot_csc, (p.n_keep * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, kept)) != cudaSuccess) return e;
