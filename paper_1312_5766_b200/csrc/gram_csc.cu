@@ -94,85 +94,25 @@ __global__ void __launch_bounds__(kThreads) k_csc_bucket_pairs(Problem p) {
       }
 }
 
-// Step 3: the listed pairs' inner products, eight lanes per pair (four pairs per warp).  Walking the two sorted
-// lists in step is a chain of ~100 dependent loads per pair; instead every lane takes entries of column a (four
-// at a time, 32 entries per trip of the group) and finds each one's row in column b by binary search, the four
-// searches of a lane interleaved.  The products are then added in ascending row order -- entry order of a, which
-// the ballots below restore -- with one fma each starting from zero: the sum sparse_dot forms, bit for bit.
-// The pair's conflict bit goes to the row of the earlier candidate (a pair that shares several rows is listed
-// as often and gives the same bit each time).
+// Step 3: a thread per listed pair merges the two columns and sets the pair's conflict bit in the row of the
+// earlier candidate (a pair that shares several rows is listed as often and gives the same bit each time).
 __global__ void __launch_bounds__(kThreads) k_csc_pair_bits(Problem p, const int* __restrict__ cand) {
   chain_begin();
   const DeviceState* st = p.st;
   if (!st->bucket_used || st->bucket_failed) return;
   const unsigned int n = st->pair_count;
   const double rho = (double)p.rho;
-  const unsigned int full = 0xffffffffu;
-  const int lane = threadIdx.x & 31, grp = lane >> 3, l8 = lane & 7;
-  const unsigned int groups_total = gridDim.x * (unsigned)(kThreads / 8);
-  // (a warp stays together: its four groups run the same number of trips, idle groups with an empty pair)
-  for (unsigned int i0 = (blockIdx.x * (unsigned)kThreads + threadIdx.x - lane) >> 3; i0 < n; i0 += groups_total) {
-    const unsigned int i = i0 + grp;
-    int a = 0, b = 0;
-    long long a0 = 0, b0 = 0;
-    int na = 0, nb = 0, ja = 0, jb = 0;
-    if (i < n) {
-      const unsigned int pr = __ldcg(p.pair_list + i);
-      a = (int)(pr >> 16); b = (int)(pr & 0xffffu);
-      if (a != b) {                                     // (a row never lists a column twice; defensive)
-        ja = cand[a]; jb = cand[b];
-        a0 = p.xptr[ja]; na = (int)(p.xptr[ja + 1] - a0);
-        b0 = p.xptr[jb]; nb = (int)(p.xptr[jb + 1] - b0);
-      }
-    }
-    const int na_max = max(max(__shfl_sync(full, na, 0), __shfl_sync(full, na, 8)),
-                           max(__shfl_sync(full, na, 16), __shfl_sync(full, na, 24)));
-    float dot = 0.f;
-    for (int c = 0; c < na_max; c += 32) {
-      int ra[4], lo[4], hi[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const int e = c + l8 + 8 * u;
-        ra[u] = e < na ? __ldg(p.xrow + a0 + e) : -1;
-        lo[u] = 0; hi[u] = ra[u] >= 0 ? nb : 0;
-      }
-      bool going = true;
-      while (going) {                                   // four lower-bound searches in step
-        going = false;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (lo[u] < hi[u]) {
-            const int mid = (lo[u] + hi[u]) >> 1;
-            if (__ldg(p.xrow + b0 + mid) < ra[u]) lo[u] = mid + 1; else hi[u] = mid;
-            going = true;
-          }
-        }
-      }
-      float av[4], bv[4];
-      bool hit[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        hit[u] = ra[u] >= 0 && lo[u] < nb && __ldg(p.xrow + b0 + lo[u]) == ra[u];
-        av[u] = hit[u] ? __ldg(p.xv + a0 + c + l8 + 8 * u) : 0.f;
-        bv[u] = hit[u] ? __ldg(p.xv + b0 + lo[u]) : 0.f;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {                     // entries c + 8u .. c + 8u + 7 in order: lanes 0 .. 7 of the group
-        unsigned int bits = (__ballot_sync(full, hit[u]) >> (grp * 8)) & 0xffu;
-        while (__any_sync(full, bits != 0u)) {
-          const int src = bits ? (grp * 8 + __ffs((int)bits) - 1) : lane;
-          const float x = __shfl_sync(full, av[u], src), y = __shfl_sync(full, bv[u], src);
-          if (bits) dot = fmaf(x, y, dot);
-          bits &= bits - 1u;
-        }
-      }
-    }
-    if (l8 == 0 && i < n && a != b) {
-      const double den = sqrt(p.n2[ja] * p.n2[jb]);
-      if (den > 0.0 && fabs((double)dot) >= rho * den) {
-        atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
-        list_conflict(p, a, b);                         // (a pair listed twice is listed twice here too: harmless)
-      }
+  for (unsigned int i = blockIdx.x * (unsigned)kThreads + threadIdx.x; i < n; i += gridDim.x * (unsigned)kThreads) {
+    const unsigned int pr = __ldcg(p.pair_list + i);
+    const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
+    if (a == b) continue;                               // (a row never lists a column twice; defensive)
+    const int ja = cand[a], jb = cand[b];
+    const long long a0 = p.xptr[ja];
+    const float dot = sparse_dot(p.xrow + a0, p.xv + a0, (int)(p.xptr[ja + 1] - a0), p, jb);
+    const double den = sqrt(p.n2[ja] * p.n2[jb]);
+    if (den > 0.0 && fabs((double)dot) >= rho * den) {
+      atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+      list_conflict(p, a, b);                             // (a pair listed twice is listed twice here too: harmless)
     }
   }
 }
