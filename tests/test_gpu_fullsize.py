@@ -95,3 +95,30 @@ def test_full_size_rounds(name):
     assert tot["rounds"] == t and tot["kept"] >= sum(k for k, _ in stats)
     del s, p
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["c2", "c3"])
+def test_full_size_run_equals_rounds(name):
+    """strads_run at full size (captured sequences of eight rounds, candidates drawn one round ahead and corrected,
+    whole-list retry on its own branch) leaves the bits of the same rounds run one by one with strads_round, whose
+    rounds the test above checks against the oracle."""
+    from paper_1312_5766_b200 import binding
+    free, _ = torch.cuda.mem_get_info()
+    need = {"c2": 8e9, "c3": 26e9}[name]
+    if free < need:
+        pytest.skip(f"{name} needs {need / 1e9:.0f} GB of device memory")
+    p = wl.make_problem(name, seed=0, device="cuda")
+    a = binding.StradsLasso.from_problem(p, device="cuda")        # (both handles read the same X on the device)
+    b = binding.StradsLasso.from_problem(p, device="cuda")
+    done = 0
+    for n in (19, 8, 6):                                           # a first round drawn on the spot, whole sequences, a tail
+        a.run(n)
+        for _ in range(n):
+            b.round()
+        done += n
+        assert a.get_round() == b.get_round() == done
+        for x, y in ((a.beta, b.beta), (a.resid, b.resid), (a.delta, b.delta)):
+            assert torch.equal(x, y), (name, done)
+    assert a.totals() == b.totals() and a.status()[0] == 0 and b.status()[0] == 0
+    del a, b, p
+    torch.cuda.empty_cache()
