@@ -176,9 +176,18 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
   const long long groups = (p.J + 3) >> 2;
   const float cut = mode == 1 ? p.st->t_cut : 0.f;
   const unsigned int cut_bin = cut > 0.f ? (__float_as_uint(cut) >> (32 - kHistBits)) : (unsigned)kHistBins;   // bins below it are complete
+  // Guided pass: the keys below the cutoff (a few times P' of them) are also saved, so that the collect pass can
+  // take the winners from those instead of going through all J coefficients again.
+  const bool save = cut > 0.f && p.survivors != nullptr;
   auto count = [&](unsigned long long key) {
     const unsigned int bin = (unsigned int)(key >> (64 - kHistBits));
-    if (bin < cut_bin) atomicAdd(&sh[bin], 1u);
+    if (bin < cut_bin) {
+      atomicAdd(&sh[bin], 1u);
+      if (save) {
+        const unsigned int at = atomicAdd(&p.st->surv_count, 1u);
+        if (at < (unsigned)p.cap_survivors) p.survivors[at] = key;
+      }
+    }
   };
   if (cut > 0.f) {
     __shared__ uint2 s_queue[kThreads / 32][kQueue];
@@ -224,12 +233,14 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
     atomicAdd(&s_total, mine);
     __syncthreads();
     if (s_total < (unsigned)p.n_cand) {
-      if (tid == 0) { p.st->hist_ticket = 0; p.st->sample_redo = 1; p.st->t_cut = 0.f; }
+      if (tid == 0) { p.st->hist_ticket = 0; p.st->sample_redo = 1; p.st->t_cut = 0.f; p.st->surv_valid = 0; }
       return;
     }
   }
   find_bin(sh, kHistBins, p.n_cand, &s_bin, &s_before);
   if (tid == 0) {
+    // (every CTA's appends are done and visible: they precede its ticket)
+    p.st->surv_valid = (save && __ldcg(&p.st->surv_count) <= (unsigned)p.cap_survivors) ? 1 : 0;
     p.st->sample_redo = 0;
     // next round's cutoff: four times the upper edge of this boundary bin (none if that is not a finite number)
     const unsigned int edge = ((unsigned int)s_bin + 1u) << (32 - kHistBits);
@@ -290,6 +301,12 @@ __global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
     }
   };
   const int tid = threadIdx.x;
+  if (p.st->surv_valid) {                              // every key below the first pass's cutoff is at hand
+    const unsigned int n = p.st->surv_count;
+    for (unsigned int i = blockIdx.x * (unsigned)kThreads + tid; i < n; i += gridDim.x * (unsigned)kThreads)
+      take(__ldcg(p.survivors + i));
+    return;
+  }
   if (cut > 0.f) {
     __shared__ uint2 s_queue[kThreads / 32][kQueue];
     KeyQueue q = {s_queue[tid >> 5], 0};
@@ -371,7 +388,7 @@ __global__ void __launch_bounds__(512) k_sample_rank(Problem p, int* cand_out) {
   __shared__ unsigned long long other[kChunk];
   const SelectState sel = p.st->sel;
   const ChunkRef ch = chunk_of(p, sel, blockIdx.x);
-  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
+  if (blockIdx.x == 0 && threadIdx.x == 0) { p.st->counts[0] = p.n_cand; p.st->surv_count = 0; }
   if (ch.n == 0) return;
   const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
   const unsigned long long* buf = ch.is_sure ? p.sure : p.boundary;
@@ -402,7 +419,7 @@ __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand
   chain_begin();
   __shared__ unsigned long long all[kDirectMax];
   const SelectState sel = p.st->sel;
-  if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
+  if (blockIdx.x == 0 && threadIdx.x == 0) { p.st->counts[0] = p.n_cand; p.st->surv_count = 0; }
   const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
   const int sure_ctas = (p.cap_sure + kDirectKeys - 1) / kDirectKeys;
   const bool is_sure = (int)blockIdx.x < sure_ctas;
@@ -517,7 +534,7 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   cudaError_t e;
   // many coefficients: the first pass leaves out the keys far above the last boundary (and a second launch
   // repeats it in full in the rare round where that boundary was a bad guide)
-  const bool guided = p.J >= (1 << 22);     // (below that the passes are bound by latency, not by arithmetic)
+  const bool guided = p.J >= (1 << 19);     // (below that the passes are bound by latency, not by arithmetic)
   if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, guided ? 1 : 0)) != cudaSuccess) return e;
   if (guided && (e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, 2)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;

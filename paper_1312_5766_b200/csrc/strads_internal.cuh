@@ -41,6 +41,8 @@ struct DeviceState {
   int sample_redo;              // sampler: the guided first pass found too few keys; the plain pass behind it runs
   int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
+  unsigned int surv_count;      // sampler: keys the guided first pass found below its cutoff and saved (append cursor)
+  int surv_valid;               // ... they are all there (no overflow, no repeat): the collect pass reads them, not delta[J]
   unsigned int edge_count;      // conflicting pairs listed by the Gram kernels of this round (may exceed the list)
   int edges_off;                // a kernel that sets bits without listing pairs has run: the list is not complete
   unsigned int pad;
@@ -116,6 +118,8 @@ struct Problem {
   const unsigned long long* round_ptr;   // the sampler's round index is *round_ptr + round_ahead
   int round_ahead;
   unsigned long long* keys_out;          // sampler: if set, the winners' keys in rank order go here too
+  unsigned long long* survivors;         // sampler: [cap_survivors] keys below the guided first pass's cutoff (null: not kept)
+  int cap_survivors;
   float* delta_prev;                     // [n_keep] delta of the kept coefficients before this round's update
   // Conflicts are normally few (a handful per hundred candidates), so the Gram kernels also list the conflicting
   // pairs (a << 16 | b, a < b, positions in the list) and the walk works from that list when it is complete.
