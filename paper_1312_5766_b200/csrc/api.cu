@@ -78,7 +78,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_survivors,
+      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
   long long ldc;
@@ -155,6 +155,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   // keys the sampler's guided first pass saves for its collect pass (many coefficients only): 8 P' of them
   L.cap_survivors = c->n_cols >= (1 << 19) ? 8 * c->n_candidates : 0;
   L.off_survivors = take(sizeof(unsigned long long) * (size_t)L.cap_survivors);
+  L.off_bin_off = take(sizeof(int) * (kHistBins + 1));
+  L.off_bin_cur = take(sizeof(unsigned int) * kHistBins);
   // sampling ahead (one scheduler, P <= kAheadMaxKeep): a second set of sampler buffers for P' + P winners.
   // Dense layouts only: measured on CSC workloads, whose rounds contain a cooperative kernel, a draw running
   // beside the round made it slower (c4: 140 -> 203 us), not faster.
@@ -168,6 +170,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_ahead_boundary = take(sizeof(unsigned long long) * (size_t)L.cap_ahead_boundary);
   L.off_ahead_keys = take(sizeof(unsigned long long) * (size_t)L.n_ahead);
   L.off_ahead_idx = take(sizeof(int) * (size_t)L.n_ahead);
+  L.off_ahead_bin_off = take(ahead ? sizeof(int) * (kHistBins + 1) : 0);
+  L.off_ahead_bin_cur = take(ahead ? sizeof(unsigned int) * kHistBins : 0);
   L.total = o;
   return L;
 }
@@ -375,6 +379,8 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.round_ptr = &p.st->round; p.round_ahead = 0;
   p.keys_out = nullptr;
   p.delta_prev = reinterpret_cast<float*>(ws + L.off_delta_prev);
+  p.bin_off = reinterpret_cast<int*>(ws + L.off_bin_off);
+  p.bin_cur = reinterpret_cast<unsigned int*>(ws + L.off_bin_cur);
   p.survivors = L.cap_survivors ? reinterpret_cast<unsigned long long*>(ws + L.off_survivors) : nullptr;
   p.cap_survivors = L.cap_survivors;
   p.edges = reinterpret_cast<unsigned int*>(ws + L.off_edges);
@@ -394,6 +400,8 @@ void fill_ahead(Problem& a, const Problem& p0, const Layout& L, char* ws) {
   a.cand = reinterpret_cast<int*>(ws + L.off_ahead_idx);
   a.keys_out = reinterpret_cast<unsigned long long*>(ws + L.off_ahead_keys);
   a.round_ptr = &p0.st->round; a.round_ahead = 1;
+  a.bin_off = reinterpret_cast<int*>(ws + L.off_ahead_bin_off);
+  a.bin_cur = reinterpret_cast<unsigned int*>(ws + L.off_ahead_bin_cur);
   a.survivors = nullptr; a.cap_survivors = 0;         // (the early draw is off the round's path: it keeps to the plain passes)
 }
 

@@ -254,6 +254,41 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
     s_sel.n_boundary = (int)sh[s_bin];
   }
   __syncthreads();
+  if (p.bin_off != nullptr) {
+    // Where the sure keys of every bin below the boundary bin start in the `sure` buffer (exclusive prefix of the
+    // counts; the boundary bin's own sure keys, if it gets refined, follow at s_before), and the bins' cursors:
+    // the collect pass then leaves the winners grouped by their top 12 bits, and ordering them is a matter of
+    // ranking every key inside its own small group.
+    __shared__ unsigned int s_wtot[kThreads / 32];
+    constexpr int kPer = kHistBins / kThreads;
+    const int b0 = tid * kPer, lane = tid & 31, wid = tid >> 5;
+    unsigned int mine = 0u;
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) mine += (b0 + u < s_bin) ? sh[b0 + u] : 0u;
+    unsigned int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) s_wtot[wid] = incl;
+    __syncthreads();
+    unsigned int run = incl - mine;
+    for (int w = 0; w < wid; ++w) run += s_wtot[w];
+#pragma unroll
+    for (int u = 0; u < kPer; ++u) {                   // counts -> offsets in place (nobody needs the counts any more)
+      const unsigned int c = (b0 + u < s_bin) ? sh[b0 + u] : 0u;
+      sh[b0 + u] = run;
+      run += c;
+    }
+    if (tid == kThreads - 1) p.bin_off[kHistBins] = (int)run;
+    __syncthreads();
+    for (int b = tid; b < kHistBins; b += kThreads) {  // coalesced
+      p.bin_off[b] = (int)sh[b];
+      p.bin_cur[b] = 0u;
+    }
+    __syncthreads();
+  }
   // Rare: the boundary bin does not fit the buffer -> refine digit by digit with this CTA alone.
   while (s_sel.n_boundary > p.cap_boundary && s_sel.bits < 64) {
     const int bits = s_sel.bits;
@@ -290,10 +325,17 @@ __global__ void __launch_bounds__(kThreads) k_sample_collect(Problem p) {
   // keys certainly above the boundary's upper edge are not computed
   unsigned long long edge = sel.bits <= 32 ? ((sel.prefix + 1ull) << (32 - sel.bits)) : (sel.prefix >> (sel.bits - 32));
   const float cut = edge < 0x7f800000ull && edge > 0ull ? __uint_as_float((unsigned int)edge) : 0.f;
+  const unsigned int top_bin = (unsigned int)(sel.prefix >> (sel.bits - kHistBits));   // the boundary bin of the first pass
   auto take = [&](unsigned long long key) {
     const unsigned long long pfx = key >> shift;
     if (pfx < sel.prefix) {
-      const unsigned int i = atomicAdd(&p.st->sure_count, 1u);
+      unsigned int i;
+      if (p.bin_off != nullptr) {                      // into the group of its histogram bin
+        const unsigned int bin = min((unsigned int)(key >> (64 - kHistBits)), top_bin);
+        i = (unsigned int)p.bin_off[bin] + atomicAdd(&p.bin_cur[bin], 1u);
+      } else {
+        i = atomicAdd(&p.st->sure_count, 1u);
+      }
       if (i < (unsigned)p.cap_sure) p.sure[i] = key;
     } else if (pfx == sel.prefix) {
       const unsigned int i = atomicAdd(&p.st->boundary_count, 1u);
@@ -444,6 +486,49 @@ __global__ void __launch_bounds__(256) k_sample_rank_direct(Problem p, int* cand
   }
 }
 
+// Ordering the winners when the collect pass grouped them by histogram bin (bin_off): bins are in key order, so a
+// sure key's rank is the start of its bin's group plus the number of smaller keys inside the group -- a few
+// hundred keys (an exponential race spreads the winners over dozens of bins, at most ~P' / 16 in one) -- and a
+// boundary key's is n_sure plus the number of smaller boundary keys.  Eight threads per key, all in one kernel.
+__global__ void __launch_bounds__(256) k_sample_rank_bins(Problem p, int* cand_out) {
+  chain_begin();
+  const SelectState sel = p.st->sel;
+  if (blockIdx.x == 0 && threadIdx.x == 0) { p.st->counts[0] = p.n_cand; p.st->surv_count = 0; }
+  const int n_sure = min(sel.n_sure, p.cap_sure), n_bnd = min(sel.n_boundary, p.cap_boundary);
+  const int i = (blockIdx.x * 256 + threadIdx.x) >> 3, slice = threadIdx.x & 7;    // eight threads per key
+  const unsigned long long* buf = p.sure;
+  unsigned long long key = 0ull;
+  int first = 0, count = 0, base = 0;
+  if (i < n_sure) {
+    const int top_bin = (int)(sel.prefix >> (sel.bits - kHistBits));
+    key = p.sure[i];
+    const int bin = min((int)(key >> (64 - kHistBits)), top_bin);
+    first = p.bin_off[bin];
+    count = (bin < top_bin ? p.bin_off[bin + 1] : n_sure) - first;
+    base = first;
+  } else if (i - n_sure < n_bnd) {
+    key = p.boundary[i - n_sure];
+    count = n_bnd; buf = p.boundary; base = n_sure;
+  }
+  // thread `slice` looks at keys slice, slice + 8, ... of the group: the eight threads read 64 consecutive bytes
+  int b0 = 0, b1 = 0, b2 = 0, b3 = 0;
+  int j = slice;
+  for (; j + 24 < count; j += 32) {
+    b0 += buf[first + j] < key; b1 += buf[first + j + 8] < key;
+    b2 += buf[first + j + 16] < key; b3 += buf[first + j + 24] < key;
+  }
+  for (; j < count; j += 8) b0 += buf[first + j] < key;
+  int below = b0 + b1 + b2 + b3;
+  below += __shfl_xor_sync(0xffffffffu, below, 1);
+  below += __shfl_xor_sync(0xffffffffu, below, 2);
+  below += __shfl_xor_sync(0xffffffffu, below, 4);
+  const int rank = base + below;
+  if (slice == 0 && count > 0 && rank < p.n_cand) {
+    cand_out[rank] = (int)(key & 0xffffffffull);
+    if (p.keys_out) p.keys_out[rank] = key;
+  }
+}
+
 // Sampling ahead.  The draw of round t is made during round t - 1 (beside its Gram and walk) from the delta of
 // that round's start, for P' + P winners instead of P'; the update of round t - 1 then changes delta for at most P
 // coefficients.  Every other coefficient keeps its key, and one of them that belongs to the true P' smallest has
@@ -538,6 +623,8 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, guided ? 1 : 0)) != cudaSuccess) return e;
   if (guided && (e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, 2)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
+  if (p.bin_off != nullptr)
+    return launch_chained(k_sample_rank_bins, (unsigned)((p.cap_sure + p.cap_boundary + 31) / 32), 256, 0, s, p, cand_out);
   if (p.cap_sure <= kDirectMax && p.cap_boundary <= kDirectMax) {
     const int ctas = (p.cap_sure + kDirectKeys - 1) / kDirectKeys + (p.cap_boundary + kDirectKeys - 1) / kDirectKeys;
     return launch_chained(k_sample_rank_direct, ctas, 256, 0, s, p, cand_out);

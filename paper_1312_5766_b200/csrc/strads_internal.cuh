@@ -118,6 +118,8 @@ struct Problem {
   const unsigned long long* round_ptr;   // the sampler's round index is *round_ptr + round_ahead
   int round_ahead;
   unsigned long long* keys_out;          // sampler: if set, the winners' keys in rank order go here too
+  int* bin_off;                          // sampler: [kHistBins + 1] where the sure keys of a histogram bin start in `sure` (null: appended in any order)
+  unsigned int* bin_cur;                 // sampler: [kHistBins] append cursor of every bin
   unsigned long long* survivors;         // sampler: [cap_survivors] keys below the guided first pass's cutoff (null: not kept)
   int cap_survivors;
   float* delta_prev;                     // [n_keep] delta of the kept coefficients before this round's update
