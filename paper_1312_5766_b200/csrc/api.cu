@@ -78,7 +78,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
+      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
   long long ldc;
@@ -152,6 +152,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_resid_acc = take(csc ? sizeof(long long) * (size_t)c->n_rows : 0);
   L.off_delta_prev = take(sizeof(float) * (size_t)c->n_keep);
   L.off_edges = take(sizeof(unsigned int) * kEdgeCap);
+  L.off_patch_keys = take(sizeof(unsigned long long) * 2 * (size_t)c->n_keep);
+  L.off_cand_keys = take(dense ? sizeof(unsigned long long) * 2 * (size_t)c->n_candidates : 0);
   // keys the sampler's guided first pass saves for its collect pass (many coefficients only): 8 P' of them
   L.cap_survivors = c->n_cols >= (1 << 19) ? 8 * c->n_candidates : 0;
   L.off_survivors = take(sizeof(unsigned long long) * (size_t)L.cap_survivors);
@@ -384,6 +386,8 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.survivors = L.cap_survivors ? reinterpret_cast<unsigned long long*>(ws + L.off_survivors) : nullptr;
   p.cap_survivors = L.cap_survivors;
   p.edges = reinterpret_cast<unsigned int*>(ws + L.off_edges);
+  p.patch_keys = reinterpret_cast<unsigned long long*>(ws + L.off_patch_keys);
+  p.cand_keys = reinterpret_cast<unsigned long long*>(ws + L.off_cand_keys);
   p.cap_edges = kEdgeCap;
 }
 

@@ -237,8 +237,10 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
       const double m = fabs(z) - (double)p.lambda / n;
       b_new = (float)(m <= 0.0 ? 0.0 : (z > 0.0 ? m : -m));
     }
+    const double d = isfinite(g) ? (double)b_new - (double)b_old : g - g;      // a non-finite product shows as NaN
     p.cand_bnew[a] = b_new;
-    p.cand_dbeta64[a] = isfinite(g) ? (double)b_new - (double)b_old : g - g;   // a non-finite product shows as NaN
+    p.cand_dbeta64[a] = d;
+    next_round_keys(p, (uint32_t)j, p.delta[j], (float)fabs(d), &p.cand_keys[a], &p.cand_keys[p.n_cand + a]);
   }
 }
 

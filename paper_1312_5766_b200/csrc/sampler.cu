@@ -537,8 +537,8 @@ __global__ void __launch_bounds__(256) k_sample_rank_bins(Problem p, int* cand_o
 // keys): exactly the list a draw made now would give.  Rank of an element of L at index i:
 // i - #(old keys of updated coefficients below it) + #(new keys below it); of a new key: its insertion point in L
 // instead of i.  (An old key below an element of L is itself on L, L being a prefix of the full ranking; a new key
-// beyond the end of a list shorter than J ranks >= P' and is left out.)  The <= P old and new keys are recomputed by
-// every CTA into shared memory and counted against by brute force.
+// beyond the end of a list shorter than J ranks >= P' and is left out.)  The <= P old and new keys were left by the
+// update (patch_keys); every CTA holds them in shared memory and counts against them by brute force.
 __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned long long* __restrict__ list, int n_list,
                                                       int* __restrict__ cand_out) {
   chain_begin();
@@ -546,52 +546,50 @@ __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned 
   const int nk = p.st->counts[2];                      // coefficients the last update touched
   unsigned long long* old_k = s_keys;
   unsigned long long* new_k = s_keys + p.n_keep;
-  const unsigned long long t = *p.round_ptr + (unsigned long long)p.round_ahead;
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
-  for (int a = threadIdx.x; a < nk; a += 256) {
-    const uint32_t j = (uint32_t)p.kept[a];
-    uint32_t w[4];
-    philox4x32_10(j >> 2, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
-    const uint32_t word = w[j & 3u];
-    old_k[a] = race_key64(p.delta_prev[a], p.eta, word, j, uniform);
-    new_k[a] = race_key64(p.delta[j], p.eta, word, j, uniform);
+  for (int a = threadIdx.x; a < nk; a += 256) {        // (left by the update, which knew both priorities)
+    old_k[a] = p.patch_keys[a];
+    new_k[a] = p.patch_keys[p.n_keep + a];
   }
   __syncthreads();
   if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
-  // CTAs 0 .. list_ctas - 1: a thread per element of the list.  The CTAs behind them: a warp per new key, whose
-  // insertion point is counted over the whole list by the 32 lanes (independent, coalesced loads instead of the
-  // dependent probes of a binary search).
-  const int list_ctas = (n_list + 255) / 256;
-  unsigned long long key;
-  int at;                                              // elements of L below the key
-  bool from_list;
+  const unsigned int full = 0xffffffffu;
+  const int list_ctas = (n_list + 31) / 32;            // eight threads per element of the list
   if ((int)blockIdx.x < list_ctas) {
-    const int item = blockIdx.x * 256 + threadIdx.x;
-    if (item >= n_list) return;
-    key = list[item];
-    at = item;
-    from_list = true;
-  } else {
-    const int a = ((int)blockIdx.x - list_ctas) * 8 + (int)(threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (a >= nk) return;
-    key = new_k[a];
-    int below = 0;
-    for (int i = lane; i < n_list; i += 32) below += list[i] < key;
+    const int item = (blockIdx.x * 256 + threadIdx.x) >> 3, slice = threadIdx.x & 7;
+    const unsigned long long key = item < n_list ? list[item] : 0ull;
+    int below_old = 0, below_new = 0, is_old = 0;
+    for (int a = slice; a < nk; a += 8) {
+      const unsigned long long o = old_k[a];
+      below_old += o < key;
+      is_old |= o == key;
+      below_new += new_k[a] < key;
+    }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
-    if (lane != 0 || (below == n_list && (long long)n_list < p.J)) return;
-    at = below;
-    from_list = false;
+    for (int o = 1; o < 8; o <<= 1) {
+      below_old += __shfl_xor_sync(full, below_old, o);
+      below_new += __shfl_xor_sync(full, below_new, o);
+      is_old |= __shfl_xor_sync(full, is_old, o);
+    }
+    if (slice != 0 || item >= n_list || is_old) return;   // (an updated coefficient: its new key stands in for it)
+    const int rank = item - below_old + below_new;
+    if (rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
+    return;
   }
-  int below_old = 0, below_new = 0;
-  bool is_old = false;
-  for (int a = 0; a < nk; ++a) {
-    const unsigned long long o = old_k[a];
-    below_old += o < key;
-    is_old |= o == key;
-    below_new += new_k[a] < key;
+  // The CTAs behind them: a warp per new key; its insertion point is counted over the whole list by the 32 lanes
+  // (independent, coalesced loads instead of the dependent probes of a binary search).
+  const int a = ((int)blockIdx.x - list_ctas) * 8 + (int)(threadIdx.x >> 5), lane = threadIdx.x & 31;
+  if (a >= nk) return;
+  const unsigned long long key = new_k[a];
+  int at = 0, below_old = 0, below_new = 0;
+  for (int i = lane; i < n_list; i += 32) at += list[i] < key;
+  for (int b = lane; b < nk; b += 32) { below_old += old_k[b] < key; below_new += new_k[b] < key; }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    at += __shfl_xor_sync(full, at, o);
+    below_old += __shfl_xor_sync(full, below_old, o);
+    below_new += __shfl_xor_sync(full, below_new, o);
   }
-  if (from_list && is_old) return;                     // an updated coefficient: its new key stands in for it
+  if (lane != 0 || (at == n_list && (long long)n_list < p.J)) return;
   const int rank = at - below_old + below_new;
   if (rank < p.n_cand) cand_out[rank] = (int)(key & 0xffffffffull);
 }
@@ -604,7 +602,7 @@ cudaError_t prepare_sample(const Problem&) {
 }
 
 cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s) {
-  const int ctas = (ahead.n_cand + 255) / 256 + (p.n_keep + 7) / 8;      // list elements by thread, new keys by warp
+  const int ctas = (ahead.n_cand + 31) / 32 + (p.n_keep + 7) / 8;        // list elements by eight threads, new keys by warp
   return launch_chained(k_sample_patch, ctas, 256, 2 * sizeof(unsigned long long) * (size_t)p.n_keep, s, p,
                         (const unsigned long long*)ahead.keys_out, ahead.n_cand, cand_out);
 }

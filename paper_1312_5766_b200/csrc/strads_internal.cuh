@@ -123,6 +123,8 @@ struct Problem {
   unsigned long long* survivors;         // sampler: [cap_survivors] keys below the guided first pass's cutoff (null: not kept)
   int cap_survivors;
   float* delta_prev;                     // [n_keep] delta of the kept coefficients before this round's update
+  unsigned long long* patch_keys;        // [2][n_keep] their race keys of the NEXT round, before and after the update
+  unsigned long long* cand_keys;         // dense, proposals: [2][n_cand] the same for every candidate, by position
   // Conflicts are normally few (a handful per hundred candidates), so the Gram kernels also list the conflicting
   // pairs (a << 16 | b, a < b, positions in the list) and the walk works from that list when it is complete.
   unsigned int* edges;                   // [cap_edges]
@@ -213,6 +215,19 @@ __device__ __forceinline__ unsigned long long race_key64(float delta_j, float et
   const float w = uniform ? 1.0f : __fmaf_rn(delta_j, delta_j, eta);
   const float T = __fdiv_rn(unit_exponential_rn(word), w);
   return ((unsigned long long)__float_as_uint(T) << 32) | j;
+}
+
+// The race keys coefficient j has in this scheduler's next round with its priority before (d_old) and after (d_new)
+// an update: what k_sample_patch needs to correct a draw made ahead of the update.
+__device__ __forceinline__ void next_round_keys(const Problem& p, uint32_t j, float d_old, float d_new,
+                                                unsigned long long* key_old, unsigned long long* key_new) {
+  const unsigned long long t = p.st->round + (unsigned long long)p.part_count;
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  uint32_t w[4];
+  philox4x32_10(j >> 2, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
+  const uint32_t word = (j & 2u) ? ((j & 1u) ? w[3] : w[2]) : ((j & 1u) ? w[1] : w[0]);
+  *key_old = race_key64(d_old, p.eta, word, j, uniform);
+  *key_new = race_key64(d_new, p.eta, word, j, uniform);
 }
 
 // x_a^T x_b of two CSC columns (ascending rows): a given as arrays (possibly staged in shared memory), b read

@@ -38,8 +38,10 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
   }
   const double d = (double)b_new - (double)b_old;        // the change that beta (FP32) really makes
   p.beta[j] = b_new;
-  p.delta_prev[a] = p.delta[j];
-  p.delta[j] = (float)fabs(d);
+  const float d_old = p.delta[j], d_new = (float)fabs(d);
+  p.delta_prev[a] = d_old;
+  p.delta[j] = d_new;
+  next_round_keys(p, (uint32_t)j, d_old, d_new, &p.patch_keys[a], &p.patch_keys[p.n_keep + a]);   // (the round advances in a later kernel)
   p.dbeta[a] = (float)d;
   p.dbeta64[a] = d;
   if (d != 0.0) atomicAdd(&p.st->counts[3], 1);
@@ -183,6 +185,8 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
       p.beta[j] = p.cand_bnew[pos];
       p.delta_prev[a] = p.delta[j];
       p.delta[j] = (float)fabs(d);
+      p.patch_keys[a] = p.cand_keys[pos];              // formed by the pack kernel (this kernel advances the round)
+      p.patch_keys[p.n_keep + a] = p.cand_keys[p.n_cand + pos];
       p.dbeta[a] = (float)d;
       p.dbeta64[a] = d;
       if (d != 0.0) {                                    // counted here and in the running total: CTA 0 may be done already
