@@ -183,6 +183,13 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
   double n = 0.0;
   float b_old = 0.f;
   if (threadIdx.x == 0) { n = p.n2[j]; b_old = p.beta[j]; }   // two far gathers, under way while the column streams
+  // the candidate's unit exponential of the next round and its key with the present priority, by one thread of
+  // another warp while the column streams (the key with the new priority follows from the change, at the end)
+  __shared__ float s_E;
+  if (threadIdx.x == 32) {
+    s_E = next_round_exponential(p, (uint32_t)j);
+    p.cand_keys[a] = race_key_from(s_E, p.delta[j], p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
+  }
   float h0 = 0.f, l0 = 0.f, h1 = 0.f, l1 = 0.f;
   constexpr int kU = 4;                                 // column loads in flight per thread
   for (long long g0 = threadIdx.x; g0 < n4; g0 += (long long)kU * blockDim.x) {
@@ -240,7 +247,7 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
     const double d = isfinite(g) ? (double)b_new - (double)b_old : g - g;      // a non-finite product shows as NaN
     p.cand_bnew[a] = b_new;
     p.cand_dbeta64[a] = d;
-    next_round_keys(p, (uint32_t)j, p.delta[j], (float)fabs(d), &p.cand_keys[a], &p.cand_keys[p.n_cand + a]);
+    p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
   }
 }
 

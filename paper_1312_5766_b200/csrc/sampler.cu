@@ -617,7 +617,7 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   cudaError_t e;
   // many coefficients: the first pass leaves out the keys far above the last boundary (and a second launch
   // repeats it in full in the rare round where that boundary was a bad guide)
-  const bool guided = p.J >= (1 << 19);     // (below that the passes are bound by latency, not by arithmetic)
+  const bool guided = p.J >= (1 << 22);     // (below that the passes are bound by latency, not by arithmetic)
   if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, guided ? 1 : 0)) != cudaSuccess) return e;
   if (guided && (e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, 2)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;

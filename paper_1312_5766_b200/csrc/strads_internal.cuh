@@ -210,24 +210,32 @@ __device__ __forceinline__ float unit_exponential_rn(uint32_t x) {
 
 // 64-bit ranking key of coefficient j: (bits of T_j) << 32 | j, T_j = E_j / (delta_j^2 + eta).
 // All keys are distinct; ascending key order = ascending T, ties to the smaller j.
+__device__ __forceinline__ unsigned long long race_key_from(float E, float delta_j, float eta, uint32_t j, bool uniform) {
+  const float w = uniform ? 1.0f : __fmaf_rn(delta_j, delta_j, eta);
+  const float T = __fdiv_rn(E, w);
+  return ((unsigned long long)__float_as_uint(T) << 32) | j;
+}
 __device__ __forceinline__ unsigned long long race_key64(float delta_j, float eta, uint32_t word, uint32_t j,
                                                          bool uniform) {
-  const float w = uniform ? 1.0f : __fmaf_rn(delta_j, delta_j, eta);
-  const float T = __fdiv_rn(unit_exponential_rn(word), w);
-  return ((unsigned long long)__float_as_uint(T) << 32) | j;
+  return race_key_from(unit_exponential_rn(word), delta_j, eta, j, uniform);
 }
 
 // The race keys coefficient j has in this scheduler's next round with its priority before (d_old) and after (d_new)
 // an update: what k_sample_patch needs to correct a draw made ahead of the update.
-__device__ __forceinline__ void next_round_keys(const Problem& p, uint32_t j, float d_old, float d_new,
-                                                unsigned long long* key_old, unsigned long long* key_new) {
+// (In two steps, because the unit exponential does not depend on the priorities: it can be had before the update.)
+__device__ __forceinline__ float next_round_exponential(const Problem& p, uint32_t j) {
   const unsigned long long t = p.st->round + (unsigned long long)p.part_count;
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
   uint32_t w[4];
   philox4x32_10(j >> 2, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
   const uint32_t word = (j & 2u) ? ((j & 1u) ? w[3] : w[2]) : ((j & 1u) ? w[1] : w[0]);
-  *key_old = race_key64(d_old, p.eta, word, j, uniform);
-  *key_new = race_key64(d_new, p.eta, word, j, uniform);
+  return unit_exponential_rn(word);
+}
+__device__ __forceinline__ void next_round_keys(const Problem& p, uint32_t j, float d_old, float d_new,
+                                                unsigned long long* key_old, unsigned long long* key_new) {
+  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  const float E = next_round_exponential(p, j);
+  *key_old = race_key_from(E, d_old, p.eta, j, uniform);
+  *key_new = race_key_from(E, d_new, p.eta, j, uniform);
 }
 
 // x_a^T x_b of two CSC columns (ascending rows): a given as arrays (possibly staged in shared memory), b read
