@@ -386,7 +386,9 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.survivors = L.cap_survivors ? reinterpret_cast<unsigned long long*>(ws + L.off_survivors) : nullptr;
   p.cap_survivors = L.cap_survivors;
   p.edges = reinterpret_cast<unsigned int*>(ws + L.off_edges);
-  p.patch_keys = reinterpret_cast<unsigned long long*>(ws + L.off_patch_keys);
+  // (only the draw made ahead needs them: one scheduler, dense)
+  p.patch_keys = (S == 1 && c->layout == STRADS_DENSE_COLMAJOR && c->n_keep <= kAheadMaxKeep)
+                     ? reinterpret_cast<unsigned long long*>(ws + L.off_patch_keys) : nullptr;
   p.cand_keys = reinterpret_cast<unsigned long long*>(ws + L.off_cand_keys);
   p.cap_edges = kEdgeCap;
 }

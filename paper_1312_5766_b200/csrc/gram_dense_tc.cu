@@ -186,7 +186,7 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
   // the candidate's unit exponential of the next round and its key with the present priority, by one thread of
   // another warp while the column streams (the key with the new priority follows from the change, at the end)
   __shared__ float s_E;
-  if (threadIdx.x == 32) {
+  if (threadIdx.x == 32 && p.patch_keys != nullptr) {
     s_E = next_round_exponential(p, (uint32_t)j);
     p.cand_keys[a] = race_key_from(s_E, p.delta[j], p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
   }
@@ -247,7 +247,8 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
     const double d = isfinite(g) ? (double)b_new - (double)b_old : g - g;      // a non-finite product shows as NaN
     p.cand_bnew[a] = b_new;
     p.cand_dbeta64[a] = d;
-    p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
+    if (p.patch_keys != nullptr)
+      p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
   }
 }
 

@@ -41,7 +41,8 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
   const float d_old = p.delta[j], d_new = (float)fabs(d);
   p.delta_prev[a] = d_old;
   p.delta[j] = d_new;
-  next_round_keys(p, (uint32_t)j, d_old, d_new, &p.patch_keys[a], &p.patch_keys[p.n_keep + a]);   // (the round advances in a later kernel)
+  if (p.patch_keys != nullptr)                           // (the round advances in a later kernel)
+    next_round_keys(p, (uint32_t)j, d_old, d_new, &p.patch_keys[a], &p.patch_keys[p.n_keep + a]);
   p.dbeta[a] = (float)d;
   p.dbeta64[a] = d;
   if (d != 0.0) atomicAdd(&p.st->counts[3], 1);
@@ -185,8 +186,10 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
       p.beta[j] = p.cand_bnew[pos];
       p.delta_prev[a] = p.delta[j];
       p.delta[j] = (float)fabs(d);
-      p.patch_keys[a] = p.cand_keys[pos];              // formed by the pack kernel (this kernel advances the round)
-      p.patch_keys[p.n_keep + a] = p.cand_keys[p.n_cand + pos];
+      if (p.patch_keys != nullptr) {                   // formed by the pack kernel (this kernel advances the round)
+        p.patch_keys[a] = p.cand_keys[pos];
+        p.patch_keys[p.n_keep + a] = p.cand_keys[p.n_cand + pos];
+      }
       p.dbeta[a] = (float)d;
       p.dbeta64[a] = d;
       if (d != 0.0) {                                    // counted here and in the running total: CTA 0 may be done already
