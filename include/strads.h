@@ -141,7 +141,16 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out);
  * the update of the current round runs, which is the paper's "each thread has S-fold more time" and gives
  * results identical to running the same rounds strictly one after another (strads_round does that).
  * Each scheduler has its own slice of the workspace.  On return every piece of work has been enqueued and
- * the configured stream waits for all of it. */
+ * the configured stream waits for all of it.
+ *
+ * One scheduler, dense X, n_keep <= 4096: the candidates of round t + 1 (Algorithm 1's draw) depend on
+ * round t only through the at most P priorities its update changes, so strads_run draws the P' + P best of
+ * round t + 1 during round t, on a stream of its own beside the Gram and the walk, from the priorities of
+ * round t's start, and round t + 1 starts from that list corrected for the coefficients round t updated
+ * (they are struck and entered again with their new keys; the P' smallest remain).  The candidates are
+ * exactly those of a draw made at the round's start; the state after strads_run equals that of the same
+ * rounds run with strads_round, bit for bit.  Eight rounds are replayed per captured launch sequence; the
+ * streams and events this needs belong to the handle (no device memory is allocated). */
 int strads_run(strads_handle_t h, int64_t n_rounds);
 
 /* The same round as strads_round for callers whose state lives in HOST memory: copies
