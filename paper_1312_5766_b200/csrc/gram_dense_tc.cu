@@ -161,11 +161,14 @@ __device__ __forceinline__ void dot_step(float x, float r, float& hi, float& lo)
   lo = __fadd_rn(lo, __fadd_rn(se, pe));
 }
 
+constexpr int kPackStream = 256;                 // threads that copy (and multiply) the column
+constexpr int kPackThreads = kPackStream + 32;   // + one warp with no streaming work, for the next round's keys
+
 // One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).  With p.proposals the column is
 // also multiplied into the residual as it streams by (fixed order: per-thread strided sums, lanes by shuffle
 // tree, warps in index order) and the candidate's would-be update follows from it at once (Eq. 2): the update
 // step then only has to apply the proposals of the kept candidates.
-__global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
+__global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
                                                          int only_if_short) {
   chain_begin();
   const int a = blockIdx.x;
@@ -183,25 +186,27 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
   double n = 0.0;
   float b_old = 0.f;
   if (threadIdx.x == 0) { n = p.n2[j]; b_old = p.beta[j]; }   // two far gathers, under way while the column streams
-  // the candidate's unit exponential of the next round and its key with the present priority, by one thread of
-  // another warp while the column streams (the key with the new priority follows from the change, at the end)
+  // the candidate's unit exponential of the next round and its key with the present priority, by a thread of the
+  // warp that streams nothing (~600 dependent instructions: in a streaming warp they would hold up its loads); the
+  // key with the new priority follows from the change, at the end
   __shared__ float s_E;
-  if (threadIdx.x == 32 && p.patch_keys != nullptr) {
+  if (threadIdx.x == kPackStream && p.patch_keys != nullptr) {
     s_E = next_round_exponential(p, (uint32_t)j);
     p.cand_keys[a] = race_key_from(s_E, p.delta[j], p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
   }
   float h0 = 0.f, l0 = 0.f, h1 = 0.f, l1 = 0.f;
   constexpr int kU = 4;                                 // column loads in flight per thread
-  for (long long g0 = threadIdx.x; g0 < n4; g0 += (long long)kU * blockDim.x) {
+  const long long first = threadIdx.x < kPackStream ? (long long)threadIdx.x : n4;      // (the extra warp: no trips)
+  for (long long g0 = first; g0 < n4; g0 += (long long)kU * kPackStream) {
     float4 xv[kU], rv[kU];
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-      const long long g = g0 + (long long)u * blockDim.x;
+      const long long g = g0 + (long long)u * kPackStream;
       xv[u] = g < n4 ? __ldg(src + g) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-      const long long g = g0 + (long long)u * blockDim.x;
+      const long long g = g0 + (long long)u * kPackStream;
       if (g < n4_full) {
         rv[u] = r4[g];
       } else if (g < n4) {                              // the last, partial group: rows past N do not exist
@@ -216,7 +221,7 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
     }
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
-      const long long g = g0 + (long long)u * blockDim.x;
+      const long long g = g0 + (long long)u * kPackStream;
       if (g < n4) dst[g] = xv[u];
       if (g >= n4_full) {                               // padding of the column (and groups past the end) stay out of the sum
         const long long i = g << 2;
@@ -233,11 +238,11 @@ __global__ void __launch_bounds__(256) k_pack_candidates(Problem p, const int* _
   double v = ((double)h0 + (double)l0) + ((double)h1 + (double)l1);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  if ((threadIdx.x & 31) == 0) wsum[threadIdx.x >> 5] = v;
+  if ((threadIdx.x & 31) == 0 && threadIdx.x < kPackStream) wsum[threadIdx.x >> 5] = v;
   __syncthreads();
   if (threadIdx.x == 0) {
     double g = 0.0;
-    for (int w = 0; w < 8; ++w) g += wsum[w];
+    for (int w = 0; w < kPackStream / 32; ++w) g += wsum[w];
     float b_new = b_old;
     if (n > 0.0) {
       const double z = (double)b_old + g / n;
@@ -480,9 +485,59 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   }
 }
 
+// Exact decision for one pair the TF32 screen could not call, by a whole warp: FP64 dot product of the packed
+// columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
+__device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, int lane) {
+  const long long n4 = (p.N + 3) >> 2;
+  const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
+  const float4* xa = reinterpret_cast<const float4*>(p.xc + (long long)a * p.ldc);
+  const float4* xb = reinterpret_cast<const float4*>(p.xc + (long long)b * p.ldc);
+  double acc = 0.0;
+  for (long long g = lane; g < n4; g += 32) {
+    const float4 u = xa[g], w = xb[g];
+    const long long i = g << 2;
+    acc += (double)u.x * w.x;
+    if (i + 1 < p.N) acc += (double)u.y * w.y;
+    if (i + 2 < p.N) acc += (double)u.z * w.z;
+    if (i + 3 < p.N) acc += (double)u.w * w.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
+    if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
+      atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+      list_conflict(p, a, b);
+    }
+  }
+}
+
+// The pairs the screen of a candidate window left open, by the CTA of the split-K reduce kernel that finishes last
+// (few pairs, normally none: this saves a launch on the round's path).  More than kInlineRecheck of them: the
+// window is handed to the whole-list retry, whose Gram has a recheck kernel of its own, by the overflow rule.
+constexpr unsigned int kInlineRecheck = 64;
+__device__ void recheck_by_last_cta(const Problem& p, unsigned int n_ctas) {
+  __shared__ int s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&p.st->gram_ticket, 1u) == n_ctas - 1u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const unsigned int n = __ldcg(&p.st->amb_count);
+  if (n > kInlineRecheck) {
+    if (threadIdx.x == 0 && n <= (unsigned)p.cap_amb) p.st->amb_count = (unsigned)p.cap_amb + 1u;   // "overflow"
+  } else {
+    const int lane = threadIdx.x & 31;
+    for (unsigned int e = threadIdx.x >> 5; e < n; e += blockDim.x >> 5) recheck_pair(p, __ldcg(p.amb_pairs + e), lane);
+  }
+  if (threadIdx.x == 0) p.st->gram_ticket = 0u;
+}
+
 // Split-K: sums the partial tiles of one output tile in split order and thresholds (screen rules).
 // One CTA per (tile, 8 rows); a warp owns one row, a lane four of its 128 columns.
-__global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short) {
+__global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short,
+                                                     int recheck_here) {
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
   const int tile = blockIdx.x >> 4, rgroup = blockIdx.x & 15;
@@ -532,10 +587,10 @@ __global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int 
   word |= __shfl_xor_sync(0xffffffffu, word, 4);
   const int widx = tj * (kTile / 32) + (lane >> 3);
   if ((lane & 7) == 0 && a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+  if (recheck_here) recheck_by_last_cta(p, gridDim.x);
 }
 
-// Exact decision for the pairs the TF32 screen could not call: one warp per pair, FP64 dot product of the
-// packed columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
+// All pairs the screen left open: one warp per pair.
 __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_short) {
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
@@ -544,31 +599,7 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_sho
   const int lane = threadIdx.x & 31;
   const unsigned int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const unsigned int n_warps = (gridDim.x * blockDim.x) >> 5;
-  const long long n4 = (p.N + 3) >> 2;
-  for (unsigned int e = warp; e < n; e += n_warps) {
-    const unsigned int pr = p.amb_pairs[e];
-    const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
-    const float4* xa = reinterpret_cast<const float4*>(p.xc + (long long)a * p.ldc);
-    const float4* xb = reinterpret_cast<const float4*>(p.xc + (long long)b * p.ldc);
-    double acc = 0.0;
-    for (long long g = lane; g < n4; g += 32) {
-      const float4 u = xa[g], w = xb[g];
-      const long long i = g << 2;
-      acc += (double)u.x * w.x;
-      if (i + 1 < p.N) acc += (double)u.y * w.y;
-      if (i + 2 < p.N) acc += (double)u.z * w.z;
-      if (i + 3 < p.N) acc += (double)u.w * w.w;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-    if (lane == 0) {
-      const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
-      if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
-        atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
-        list_conflict(p, a, b);
-      }
-    }
-  }
+  for (unsigned int e = warp; e < n; e += n_warps) recheck_pair(p, p.amb_pairs[e], lane);
 }
 
 }  // namespace
@@ -624,15 +655,18 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   q.cand_cur = cand;
   const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
   cudaError_t e;
-  if ((e = launch_chained(k_pack_candidates, n_cand, 256, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
+  if ((e = launch_chained(k_pack_candidates, n_cand, kPackThreads, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
   if (after_pack != nullptr && (e = cudaEventRecord(after_pack, s)) != cudaSuccess) return e;   // optional step timing
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
     if ((e = launch_chained(k_gram_dense_tc<false>, tiles * n_split, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, n_split,
                             ois)) != cudaSuccess)
       return e;
-    if (n_split > 1 && (e = launch_chained(k_gram_reduce, tiles * 16, 256, 0, s, q, n_cand, n_tiles, n_split, ois)) != cudaSuccess)
+    // a window with split K and a retry behind it: the reduce kernel's last CTA rechecks, no launch of its own
+    const int recheck_here = (n_split > 1 && fallback_elsewhere) ? 1 : 0;
+    if (n_split > 1 &&
+        (e = launch_chained(k_gram_reduce, tiles * 16, 256, 0, s, q, n_cand, n_tiles, n_split, ois, recheck_here)) != cudaSuccess)
       return e;
-    if ((e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
+    if (!recheck_here && (e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
   }
   if (!fallback_elsewhere || (p.flags & STRADS_FLAG_GRAM_3XTF32))
     return launch_chained(k_gram_dense_tc<true>, tiles, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, 1, ois);

@@ -43,6 +43,7 @@ struct DeviceState {
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int surv_count;      // sampler: keys the guided first pass found below its cutoff and saved (append cursor)
   int surv_valid;               // ... they are all there (no overflow, no repeat): the collect pass reads them, not delta[J]
+  unsigned int gram_ticket;     // dense Gram: CTAs of the split-K reduce kernel that are done (the last one rechecks)
   unsigned int edge_count;      // conflicting pairs listed by the Gram kernels of this round (may exceed the list)
   int edges_off;                // a kernel that sets bits without listing pairs has run: the list is not complete
   unsigned int pad;
