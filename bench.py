@@ -354,12 +354,17 @@ def main():
             return 4
         nt = (n + 127) // 128
         tiles = nt * (nt + 1) // 2
-        return 3 + (1 if tiles * 2 <= 148 else 0) + (0 if retry_follows else 1)
+        split = tiles * 2 <= 148
+        if retry_follows and split:
+            return 3                   # pack, screen, reduce (whose last CTA also rechecks the open pairs)
+        return 3 + (1 if split else 0) + (0 if retry_follows else 1)
     launches_per_round = 2 + (1 if p.n_cols >= (1 << 22) else 0) + 1 + (1 if p.layout == wl.DENSE else 3)
     sampling_ahead = p.layout == wl.DENSE and p.n_keep <= 4096
     if sampling_ahead:
         launches_per_round += 1        # the early list's correction; the early draw itself launches what a plain draw does
     if window < p.n_candidates:
+        if sampling_ahead:
+            launches_per_round += 1    # the update's gated copy at the end of the retry branch
         launches_per_round += gram_launches(window, True) + 1
         launches_per_round += (gram_launches(p.n_candidates, False) + 1) if p.layout == wl.DENSE else 1
     else:
