@@ -47,6 +47,10 @@ struct strads_lasso_s {
   // window's walk and the update
   cudaStream_t retry_stream;
   cudaEvent_t retry_fork, retry_done;
+  // strads_round_host: beta and the residual travel on a stream of their own while the draw (which reads only the
+  // priorities) already runs
+  cudaStream_t copy_stream;
+  cudaEvent_t copy_fork, copy_done;
   long long ahead_round;     // the round whose early list is in place (-1: none)
 };
 
@@ -247,13 +251,15 @@ bool update_reads_packed(const Problem& p, bool gram_exported) {
 }
 
 // One round, every step on the caller's stream, by the scheduler whose turn it is.
-int one_round(strads_lasso_s* h, const strads_round_out_t* out) {
+// before_gram: an event steps 2 and 3 have to wait for (state still on its way from the host; the draw needs only delta).
+int one_round(strads_lasso_s* h, const strads_round_out_t* out, cudaEvent_t before_gram = nullptr) {
   h->ahead_round = -1;                                 // delta changes without a new early list
   const Scheduler& sc = on_turn(h);
   const Problem& p = sc.p;
   cudaEvent_t* ev = (h->prof_events != nullptr && h->prof_rounds < h->prof_cap) ? h->prof_events + kProfEvents * h->prof_rounds : nullptr;
   if (ev) CK(cudaEventRecord(ev[0], h->stream));
   CK(launch_sample(p, p.cand, h->stream));
+  if (before_gram != nullptr) CK(cudaStreamWaitEvent(h->stream, before_gram, 0));
   if (ev) CK(cudaEventRecord(ev[1], h->stream));
   {
     const int rc = gram_and_filter(sc, h->stream, p.cand, p.n_cand, out ? out->gram : nullptr, ev ? ev[2] : nullptr,
@@ -424,6 +430,9 @@ void release(strads_lasso_s* h) {
   if (h->retry_stream != nullptr) cudaStreamDestroy(h->retry_stream);
   if (h->retry_fork != nullptr) cudaEventDestroy(h->retry_fork);
   if (h->retry_done != nullptr) cudaEventDestroy(h->retry_done);
+  if (h->copy_stream != nullptr) cudaStreamDestroy(h->copy_stream);
+  if (h->copy_fork != nullptr) cudaEventDestroy(h->copy_fork);
+  if (h->copy_done != nullptr) cudaEventDestroy(h->copy_done);
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
   if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
   if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
@@ -483,6 +492,10 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
   if ((e = prepare_gram_dense_tc()) != cudaSuccess) return fail(cuda_fail(e, "prepare_gram_dense_tc"));
   if ((e = launch_init(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_init"));
   if ((e = launch_resid_from_beta(p0, h->stream)) != cudaSuccess) return fail(cuda_fail(e, "launch_resid_from_beta"));
+  if ((e = cudaStreamCreateWithFlags(&h->copy_stream, cudaStreamNonBlocking)) != cudaSuccess ||
+      (e = cudaEventCreateWithFlags(&h->copy_fork, cudaEventDisableTiming)) != cudaSuccess ||
+      (e = cudaEventCreateWithFlags(&h->copy_done, cudaEventDisableTiming)) != cudaSuccess)
+    return fail(cuda_fail(e, "copy stream"));
   h->ahead_round = -1;
   h->ahead_ok = L.n_ahead > 0;
   if (h->ahead_ok) {
@@ -629,10 +642,15 @@ int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, fl
                       int32_t* kept_host, float* dbeta_host, int32_t* counts_host) {
   if (h == nullptr || !beta_host || !resid_host || !delta_host) return STRADS_ERR_INVALID_ARG;
   const Problem& p = on_turn(h).p;
-  CK(cudaMemcpyAsync(p.beta, beta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
-  CK(cudaMemcpyAsync(p.resid, resid_host, sizeof(float) * p.N, cudaMemcpyHostToDevice, h->stream));
+  // delta first, on the handle's stream: the draw can start as soon as it is there; beta and the residual follow on
+  // a second stream (behind whatever the handle's stream still has in flight) and are awaited before the Gram
+  CK(cudaEventRecord(h->copy_fork, h->stream));
+  CK(cudaStreamWaitEvent(h->copy_stream, h->copy_fork, 0));
   CK(cudaMemcpyAsync(p.delta, delta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->stream));
-  const int rc = one_round(h, nullptr);
+  CK(cudaMemcpyAsync(p.resid, resid_host, sizeof(float) * p.N, cudaMemcpyHostToDevice, h->copy_stream));
+  CK(cudaMemcpyAsync(p.beta, beta_host, sizeof(float) * p.J, cudaMemcpyHostToDevice, h->copy_stream));
+  CK(cudaEventRecord(h->copy_done, h->copy_stream));
+  const int rc = one_round(h, nullptr, h->copy_done);
   if (rc) return rc;
   CK(cudaMemcpyAsync(beta_host, p.beta, sizeof(float) * p.J, cudaMemcpyDeviceToHost, h->stream));
   CK(cudaMemcpyAsync(resid_host, p.resid, sizeof(float) * p.N, cudaMemcpyDeviceToHost, h->stream));
