@@ -515,7 +515,10 @@ __device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, 
 // The pairs the screen of a candidate window left open, by the CTA of the split-K reduce kernel that finishes last
 // (few pairs, normally none: this saves a launch on the round's path).  More than kInlineRecheck of them: the
 // window is handed to the whole-list retry, whose Gram has a recheck kernel of its own, by the overflow rule.
-constexpr unsigned int kInlineRecheck = 64;
+// "Few" is a budget of multiply-adds for this one CTA (2^21, some tens of microseconds at worst): short columns
+// leave many pairs open (their correlations scatter widely around rho) but each is cheap, long columns hardly any.
+constexpr unsigned int kInlineRecheck = 4096;
+constexpr long long kInlineRecheckWork = 1ll << 21;
 __device__ void recheck_by_last_cta(const Problem& p, unsigned int n_ctas) {
   __shared__ int s_last;
   __threadfence();
@@ -525,7 +528,7 @@ __device__ void recheck_by_last_cta(const Problem& p, unsigned int n_ctas) {
   if (!s_last) return;
   __threadfence();
   const unsigned int n = __ldcg(&p.st->amb_count);
-  if (n > kInlineRecheck) {
+  if (n > kInlineRecheck || (long long)n * p.N > kInlineRecheckWork) {
     if (threadIdx.x == 0 && n <= (unsigned)p.cap_amb) p.st->amb_count = (unsigned)p.cap_amb + 1u;   // "overflow"
   } else {
     const int lane = threadIdx.x & 31;
