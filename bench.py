@@ -255,13 +255,13 @@ def main():
         # exact recheck, timed together).  Algorithmic flops W(W-1)N: upper triangle, 2 flop per multiply-add.
         flops = float(window) * (window - 1) * p.n_rows
         achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
-        peak = peaks["bf16_tflops"] * 0.5                    # TF32 dense = half the BF16 rate (nominal 1.1 vs 2.25 PF)
+        peak = peaks["bf16_tflops"]                          # the screen multiplies BF16 roundings of the columns
         roofline = {"kernel": "k_gram_dense_tc<screen> (+ k_gram_reduce, k_gram_recheck)", "bound": "tensor",
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "traffic": GRAM_WINDOW_TRAFFIC.get((args.workload, window)),
                     "window": window, "launch_ms": step_ms["gram_ms"],
-                    "peak_source": f"{peaks['source']} BF16 burst x 0.5 (nominal TF32:BF16 ratio); the kernel is timed "
-                                   "alone between events"}
+                    "peak_source": f"{peaks['source']} BF16 burst (the screen's operands are BF16; pairs it cannot call "
+                                   "are decided exactly in FP64); the kernel is timed alone between events"}
     else:
         # dominant kernel: the pair merges of the window (k_gram_csc); bytes: each window column once
         nnz_col = p.nnz / p.n_cols

@@ -81,11 +81,11 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_xcb, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
       off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
-  long long ldc;
+  long long ldc, ldcb;
 };
 
 int n_sched_of(const strads_lasso_config_t* c) { return c->n_schedulers > 1 ? c->n_schedulers : 1; }
@@ -141,6 +141,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
   L.ldc = (c->n_rows + 3) / 4 * 4;
   L.off_xc = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(float) * (size_t)c->n_candidates * L.ldc : 0);
+  L.ldcb = (c->n_rows + 7) / 8 * 8;
+  L.off_xcb = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(unsigned short) * (size_t)c->n_candidates * L.ldcb : 0);
   L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)
   L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
@@ -366,6 +368,8 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.cap_amb = L.cap_amb;
   p.xc = reinterpret_cast<float*>(ws + L.off_xc);
   p.ldc = L.ldc;
+  p.xcb = reinterpret_cast<unsigned short*>(ws + L.off_xcb);
+  p.ldcb = L.ldcb;
   p.cand_dbeta64 = reinterpret_cast<double*>(ws + L.off_cand_dbeta64);
   p.cand_bnew = reinterpret_cast<float*>(ws + L.off_cand_bnew);
   // with one scheduler a round's steps follow one another on one stream, so r at pack time is r at update time;

@@ -1,18 +1,21 @@
 // SAP step 2, dense X, on the 5th-generation tensor cores: conflict bits of all candidate pairs from
 // G = X_C^T X_C, a genuine dense contraction (M = N' = P', K = the N samples).
 //
-//   k_pack_candidates   copies the P' candidate columns into one contiguous [P'][ldc] buffer.  The
-//                       candidates are scattered over the whole design matrix (one 2 MB page each for a
-//                       4 GB X); gathering them once makes every later access TLB- and TMA-friendly
-//                       (measured: the same GEMM runs 2x slower straight from scattered columns).
+//   k_pack_candidates   copies the P' candidate columns into one contiguous [P'][ldc] buffer, and a copy
+//                       rounded to BF16 beside it.  The candidates are scattered over the whole design
+//                       matrix (one 2 MB page each for a 4 GB X); gathering them once makes every later
+//                       access TLB- and TMA-friendly (measured: the same GEMM runs 2x slower straight
+//                       from scattered columns).
 //   k_gram_dense_tc<0>  "screen": one CTA per 128 x 128 tile of the upper triangle of tile pairs; one
-//                       thread feeds a 3-stage ring of 64 KB stages with TMA tile loads (128-byte
-//                       swizzle, zero fill past N and P'), one thread issues tcgen05.mma kind::tf32
-//                       on the raw FP32 bits into a 128 x 128 FP32 accumulator in tensor memory, four
-//                       warps read it back with tcgen05.ld, threshold in FP64 and write mask words.
-//                       A single-pass TF32 correlation is within 2^-9 of the exact one whatever the
-//                       data, so pairs further than the band from rho are decided for certain; the few
-//                       inside the band go to a list ...
+//                       thread feeds a 3-stage ring of 64 KB stages with TMA tile loads of the BF16 copy
+//                       (128-byte swizzle, zero fill past N and P'), one thread issues tcgen05.mma
+//                       kind::f16 into a 128 x 128 FP32 accumulator in tensor memory, four warps read
+//                       it back with tcgen05.ld, threshold in FP64 and write mask words.  The kernel is
+//                       bound by bringing operands from L2 to shared memory, so half-width operands
+//                       halve its main loop; the screen only has to be right about the pairs it calls:
+//                       a BF16 correlation is within 2^-8 of the exact one whatever the data, so pairs
+//                       further than the band from rho are decided for certain; the few inside the band
+//                       go to a list ...
 //   k_gram_recheck      ... and are decided exactly (FP64 dot product), so the decisions equal those of
 //                       an exact Gram.
 //   k_gram_dense_tc<1>  3xTF32 fallback, runs only if that list overflows (or on request): producer
@@ -22,6 +25,7 @@
 // Every wait has an iteration limit; on expiry the CTA raises STRADS_STATUS_WAIT_EXPIRED, stops issuing
 // work, and still frees its tensor memory.  No multicast anywhere.
 #include <cuda.h>
+#include <cuda_bf16.h>
 
 #include "strads_internal.cuh"
 
@@ -38,10 +42,12 @@ constexpr uint32_t kWaitLimit = 1u << 24;
 constexpr uint32_t kTmemCols = 128;
 constexpr size_t kRingBytes = 192 * 1024;
 constexpr size_t kDynSmem = kRingBytes + 1024;
-// Half-width of the "too close to call" band of the screen, relative to ||x_a|| ||x_b||: input
-// truncation costs at most 2^-9 (two operands, 11 significand bits each, Cauchy-Schwarz on the sum),
-// the N/8 FP32 accumulator updates at most 2^-23 each; doubled for margin.
-__device__ __forceinline__ double screen_band(long long N) { return 1.0 / 256.0 + (double)N * (1.0 / 33554432.0); }
+// Half-width of the "too close to call" band of the screen, relative to ||x_a|| ||x_b||.  The screen multiplies
+// BF16 roundings of the columns: each operand is off by at most 2^-9 relative (8 significand bits, round to nearest),
+// so the sum of products by at most 2^-8 (1 + 2^-10) ||x_a|| ||x_b|| (Cauchy-Schwarz); the FP32 accumulator updates
+// add at most 2^-24 each over N / 16 steps.  Doubled for margin.
+__device__ __forceinline__ double screen_band(long long N) { return 1.0 / 128.0 + (double)N * (1.0 / 33554432.0); }
+constexpr int kScreenK = 64;               // BF16 elements of K per sub-block of the screen = one 128-byte swizzle row
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -90,6 +96,15 @@ __device__ __forceinline__ void umma_tf32(uint32_t d_tmem, uint64_t a_desc, uint
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The same with BF16 inputs, K = 16.
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                          uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
@@ -161,6 +176,15 @@ __device__ __forceinline__ void dot_step(float x, float r, float& hi, float& lo)
   lo = __fadd_rn(lo, __fadd_rn(se, pe));
 }
 
+// Four consecutive elements of a packed column, rounded to BF16 (nearest even), as one 8-byte store.
+__device__ __forceinline__ void store_bf16x4(unsigned short* row, long long g, const float4& v) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 w;
+  w.x = *reinterpret_cast<const unsigned int*>(&lo);
+  w.y = *reinterpret_cast<const unsigned int*>(&hi);
+  reinterpret_cast<uint2*>(row)[g] = w;
+}
+
 constexpr int kPackStream = 256;                 // threads that copy (and multiply) the column
 constexpr int kPackThreads = kPackStream + 32;   // + one warp with no streaming work, for the next round's keys
 
@@ -177,8 +201,13 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
   const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)j * p.ld);
   float4* dst = reinterpret_cast<float4*>(p.xc + (long long)a * p.ldc);
   const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
+  unsigned short* dstb = p.xcb + (long long)a * p.ldcb;   // (ldcb >= ldc: every group of four has its place)
   if (!p.proposals) {
-    for (long long g = threadIdx.x; g < n4; g += blockDim.x) dst[g] = __ldg(src + g);
+    for (long long g = threadIdx.x; g < n4; g += blockDim.x) {
+      const float4 v = __ldg(src + g);
+      dst[g] = v;
+      store_bf16x4(dstb, g, v);
+    }
     return;
   }
   const float4* r4 = reinterpret_cast<const float4*>(p.resid);
@@ -222,7 +251,7 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
       const long long g = g0 + (long long)u * kPackStream;
-      if (g < n4) dst[g] = xv[u];
+      if (g < n4) { dst[g] = xv[u]; store_bf16x4(dstb, g, xv[u]); }
       if (g >= n4_full) {                               // padding of the column (and groups past the end) stay out of the sum
         const long long i = g << 2;
         if (i >= p.N) xv[u].x = 0.f;
@@ -309,7 +338,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const uint32_t tmem_base = s_tmem_base;
 
   const long long N = p.N;
-  const int n_st_all = (int)((N + (long long)kBlockK * kSub - 1) / ((long long)kBlockK * kSub));   // stages of K
+  constexpr int kBK = k3x ? kBlockK : kScreenK;        // elements of K per sub-block (128 bytes either way)
+  const int n_st_all = (int)((N + (long long)kBK * kSub - 1) / ((long long)kBK * kSub));   // stages of K
   const int per_split = (n_st_all + n_split - 1) / n_split;
   const int st_first = min(n_st_all, split * per_split);
   const int n_st = min(n_st_all, st_first + per_split) - st_first;     // this CTA's stages (may be 0)
@@ -329,7 +359,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
         mbar_arrive_expect_tx(bar, (uint32_t)kStageBytes);
 #pragma unroll
         for (int sub = 0; sub < kSub; ++sub) {
-          const int k = ((st_first + st) * kSub + sub) * kBlockK;    // past N the whole box is zero-filled
+          const int k = ((st_first + st) * kSub + sub) * kBK;        // past N the whole box is zero-filled
           tma_load_2d(sb + sub * kTileBytes, &tmap, k, ti * kTile, bar);
           tma_load_2d(sb + (kSub + sub) * kTileBytes, &tmap, k, tj * kTile, bar);
         }
@@ -398,7 +428,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     cp_async_wait<0>();
   } else if (warp == kMmaWarp) {
     // ------------------------------ MMA issuer (whole warp waits, one lane issues) ------------------------------
-    const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+    // instruction descriptor: FP32 accumulator; A and B both TF32 (3xTF32) or both BF16 (screen), K-major; N, M
+    constexpr uint32_t kFmt = k3x ? 2u : 1u;
+    const uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
     uint32_t acc = 0;
     for (int st = 0; st < n_st; ++st) {
       const int s = st % kStages;
@@ -416,7 +448,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       if (lane == 0) {
         const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes;
 #pragma unroll
-        for (int k8 = 0; k8 < kSub * kBlockK / 8; ++k8) {   // K = 8 per instruction: 32 bytes along the swizzled row
+        for (int k8 = 0; k8 < kSub * kBlockK / 8; ++k8) {   // 32 bytes of K per instruction (8 TF32 / 16 BF16) along the swizzled row
           const int sub = k8 / (kBlockK / 8);
           const uint64_t a_hi = umma_desc(sb + sub * kTileBytes), b_hi = umma_desc(sb + (kSub + sub) * kTileBytes);
           const uint64_t o = (uint64_t)((k8 % (kBlockK / 8)) * 2);
@@ -426,7 +458,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
             umma_tf32(tmem_base, a_hi + o, b_lo + o, idesc, 1u);
             umma_tf32(tmem_base, a_hi + o, b_hi + o, idesc, 1u);
           } else {
-            umma_tf32(tmem_base, a_hi + o, b_hi + o, idesc, acc);
+            umma_bf16(tmem_base, a_hi + o, b_hi + o, idesc, acc);
           }
           acc = 1;
         }
@@ -613,7 +645,7 @@ cudaError_t prepare_gram_dense_tc() {
   return cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
 }
 
-// Tensor map over the packed candidate buffer: [n_cand rows][N floats], row pitch ldc, box 32 x 128, 128-byte
+// Tensor map over the BF16 copy of the packed candidates: [n_cand rows][N elements], row pitch ldcb, box 64 x 128, 128-byte
 // swizzle, zero fill outside.  `out` is 128 bytes, 64-byte aligned (a CUtensorMap).
 cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
   static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
@@ -626,10 +658,10 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
   const cuuint64_t dims[2] = {(cuuint64_t)p.N, (cuuint64_t)p.n_cand};
-  const cuuint64_t strides[1] = {(cuuint64_t)p.ldc * sizeof(float)};
-  const cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)kTile};
+  const cuuint64_t strides[1] = {(cuuint64_t)p.ldcb * sizeof(unsigned short)};
+  const cuuint32_t box[2] = {(cuuint32_t)kScreenK, (cuuint32_t)kTile};
   const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = reinterpret_cast<EncodeFn>(fn)(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, p.xc,
+  const CUresult r = reinterpret_cast<EncodeFn>(fn)(static_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, p.xcb,
                                                     dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -648,7 +680,7 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   // few tiles (a candidate window): share each tile's K range among CTAs so that all SMs work
   int n_split = 1;
   if (tiles * 2 <= p.sm_count) {
-    const int n_st = (int)((p.N + 2 * kBlockK - 1) / (2 * kBlockK));
+    const int n_st = (int)((p.N + 2 * kScreenK - 1) / (2 * kScreenK));
     n_split = p.sm_count / tiles;
     if (n_split > n_st) n_split = n_st;
     if (n_split > p.partial_tiles / tiles) n_split = p.partial_tiles / tiles;

@@ -96,6 +96,8 @@ struct Problem {
   int cap_amb;
   float* xc;                    // dense: packed copy of the candidate columns, [n_cand][ldc]
   long long ldc;                // N rounded up to a multiple of 4
+  unsigned short* xcb;          // dense: the same columns rounded to BF16, [n_cand][ldcb]: operands of the Gram's screen
+  long long ldcb;               // N rounded up to a multiple of 8
   // dense, one scheduler: the pack kernel also forms x_c^T r and with it the change every candidate would
   // make if kept (valid while r is untouched between the pack and the update: same stream, same round)
   int proposals;                // 1: the pack kernel fills the two arrays below and the update applies them
