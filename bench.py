@@ -275,7 +275,7 @@ def main():
     # + r read and written)
     if p.layout == wl.DENSE:
         upd_bytes = 4.0 * p.n_rows * kept_per_round + 8.0 * p.n_rows + 16.0 * kept_per_round
-        pack_bytes = 8.0 * p.n_rows * window
+        pack_bytes = 6.0 * p.n_rows * window              # FP32 columns read, BF16 copies written
     else:
         upd_bytes = 8.0 * (p.nnz / p.n_cols) * kept_per_round + 8.0 * p.n_rows
         pack_bytes = 0.0

@@ -140,7 +140,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // borderline pairs of the TF32 screen (1 MB)
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
   L.ldc = (c->n_rows + 3) / 4 * 4;
-  L.off_xc = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(float) * (size_t)c->n_candidates * L.ldc : 0);
+  L.off_xc = take(0);                                                  // (no FP32 copy of the candidates is kept)
   L.ldcb = (c->n_rows + 7) / 8 * 8;
   L.off_xcb = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(unsigned short) * (size_t)c->n_candidates * L.ldcb : 0);
   L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)

@@ -199,14 +199,11 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
   if (a >= n_cand || (only_if_short && !p.st->window_short)) return;
   const int j = cand[a];
   const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)j * p.ld);
-  float4* dst = reinterpret_cast<float4*>(p.xc + (long long)a * p.ldc);
   const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
   unsigned short* dstb = p.xcb + (long long)a * p.ldcb;   // (ldcb >= ldc: every group of four has its place)
   if (!p.proposals) {
     for (long long g = threadIdx.x; g < n4; g += blockDim.x) {
-      const float4 v = __ldg(src + g);
-      dst[g] = v;
-      store_bf16x4(dstb, g, v);
+      store_bf16x4(dstb, g, __ldg(src + g));
     }
     return;
   }
@@ -251,7 +248,7 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
 #pragma unroll
     for (int u = 0; u < kU; ++u) {
       const long long g = g0 + (long long)u * kPackStream;
-      if (g < n4) { dst[g] = xv[u]; store_bf16x4(dstb, g, xv[u]); }
+      if (g < n4) store_bf16x4(dstb, g, xv[u]);
       if (g >= n4_full) {                               // padding of the column (and groups past the end) stay out of the sum
         const long long i = g << 2;
         if (i >= p.N) xv[u].x = 0.f;
@@ -377,8 +374,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     for (int i = 0; i < 8; ++i) {
       const int row = warp * 32 + i * 4 + rsub;
       const int ga = ti * kTile + row, gb = tj * kTile + row;
-      srcA[i] = ga < n_cand ? p.xc + (long long)ga * p.ldc : nullptr;
-      srcB[i] = gb < n_cand ? p.xc + (long long)gb * p.ldc : nullptr;
+      srcA[i] = ga < n_cand ? p.xv + (long long)p.cand_cur[ga] * p.ld : nullptr;   // (straight from X: the fallback is rare)
+      srcB[i] = gb < n_cand ? p.xv + (long long)p.cand_cur[gb] * p.ld : nullptr;
       dst_off[i] = (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
     }
     auto issue = [&](int st) {                         // all copies of one stage
@@ -388,9 +385,9 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       const uint32_t bytes = left >= 4 ? 16u : (left > 0 ? (uint32_t)left * 4u : 0u);
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        cp_async16(sb + dst_off[i], srcA[i] ? (const void*)(srcA[i] + (bytes ? k : 0)) : (const void*)p.xc,
+        cp_async16(sb + dst_off[i], srcA[i] ? (const void*)(srcA[i] + (bytes ? k : 0)) : (const void*)p.xv,
                    srcA[i] ? bytes : 0u);
-        cp_async16(sb + kTileBytes + dst_off[i], srcB[i] ? (const void*)(srcB[i] + (bytes ? k : 0)) : (const void*)p.xc,
+        cp_async16(sb + kTileBytes + dst_off[i], srcB[i] ? (const void*)(srcB[i] + (bytes ? k : 0)) : (const void*)p.xv,
                    srcB[i] ? bytes : 0u);
       }
     };
@@ -522,8 +519,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
 __device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, int lane) {
   const long long n4 = (p.N + 3) >> 2;
   const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
-  const float4* xa = reinterpret_cast<const float4*>(p.xc + (long long)a * p.ldc);
-  const float4* xb = reinterpret_cast<const float4*>(p.xc + (long long)b * p.ldc);
+  const float4* xa = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[a] * p.ld);
+  const float4* xb = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[b] * p.ld);
   double acc = 0.0;
   for (long long g = lane; g < n4; g += 32) {
     const float4 u = xa[g], w = xb[g];

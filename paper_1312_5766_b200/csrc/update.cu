@@ -140,9 +140,8 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
     const int n_here = min(kStageCols, n_kept - base);
     if (base > 0) __syncthreads();
     for (int a = threadIdx.x; a < n_here; a += kThreads) {
-      const int idx = src.index[base + a];
-      s_off[a] = (long long)idx * src.pitch;
-      s_d[a] = proposals ? p.cand_dbeta64[idx] : p.dbeta64[base + a];
+      s_off[a] = (long long)src.index[base + a] * src.pitch;
+      s_d[a] = proposals ? p.cand_dbeta64[p.kept_pos[base + a]] : p.dbeta64[base + a];
     }
     __syncthreads();
     if (i < p.N) {
@@ -181,7 +180,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
   if (proposals) {
     for (int a = blockIdx.x * kThreads + threadIdx.x; a < p.n_keep; a += gridDim.x * kThreads) {
       if (a >= n_kept) { p.dbeta[a] = 0.f; continue; }
-      const int pos = src.index[a], j = kept[a];
+      const int pos = p.kept_pos[a], j = kept[a];
       const double d = p.cand_dbeta64[pos];
       p.beta[j] = p.cand_bnew[pos];
       p.delta_prev[a] = p.delta[j];
@@ -306,8 +305,7 @@ __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta
 cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s, int gate) {
   if (p.layout == STRADS_DENSE_COLMAJOR) {
     ColumnSource src;
-    if (from_packed) { src.base = p.xc; src.pitch = p.ldc; src.index = p.kept_pos; }
-    else { src.base = p.xv; src.pitch = p.ld; src.index = kept; }
+    src.base = p.xv; src.pitch = p.ld; src.index = kept;           // the kept columns, from X itself
     cudaError_t e;
     const int proposals = from_packed && p.proposals ? 1 : 0;     // the pack kernel of this round left the changes
     if (gate != 0 && !proposals) return cudaErrorInvalidValue;    // (only the single-kernel update is gated)
