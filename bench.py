@@ -33,7 +33,7 @@ UNIT = "coordinate updates/s"
 # DRAM bytes (read + write) per launch of the window-Gram kernels from ncu (dram__bytes_read.sum +
 # dram__bytes_write.sum; profiles/ncu_full_round_kernels_c2_J20000.md), keyed by (workload, window).  The capture was made
 # with J cut to 20,000; the window kernels read the packed window only, so their traffic does not depend on J.
-GRAM_WINDOW_TRAFFIC = {("c2", 512): 20.5e6}
+GRAM_WINDOW_TRAFFIC = {("c2", 512): 10.3e6}
 
 
 def measured_peaks():
