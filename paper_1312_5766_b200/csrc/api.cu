@@ -13,7 +13,7 @@ using namespace strads;
 // One scheduler thread of Section 3: its coefficients (Problem::part_index), its slice of the workspace
 // (everything steps 1 and 2 write), and what orders its work against the updates.
 struct Scheduler {
-  alignas(64) unsigned char gram_tmap[128];   // tensor map over its packed candidate buffer (dense layouts)
+  alignas(64) unsigned char gram_tmap[128];   // tensor map over the BF16 copies of its candidates (dense layouts)
   Problem p;
   int walk_grid;             // CTAs of the cooperative on-demand walk (CSC)
   cudaStream_t stream;       // S > 1: steps 1 and 2 of its rounds are enqueued here
@@ -247,8 +247,9 @@ int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_
   return STRADS_OK;
 }
 
-// after a tensor-core Gram the kept columns are read from the packed candidate buffer
-bool update_reads_packed(const Problem& p, bool gram_exported) {
+// whether this round's pack kernel ran before the update (tensor-core Gram): with one scheduler it has then left the
+// would-be changes of all candidates
+bool update_after_pack(const Problem& p, bool gram_exported) {
   return p.layout == STRADS_DENSE_COLMAJOR && !(p.flags & (STRADS_FLAG_NO_FILTER | STRADS_FLAG_SIMT_GRAM)) && !gram_exported;
 }
 
@@ -269,7 +270,7 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out, cudaEvent_t befo
     if (rc) return rc;
   }
   if (ev) CK(cudaEventRecord(ev[4], h->stream));
-  CK(launch_update(p, p.kept, 1, update_reads_packed(p, out && out->gram), h->stream));
+  CK(launch_update(p, p.kept, 1, update_after_pack(p, out && out->gram), h->stream));
   if (ev) { CK(cudaEventRecord(ev[5], h->stream)); h->prof_rounds += 1; }
   h->round_host += 1;
   if (out != nullptr) {
@@ -291,7 +292,7 @@ int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
   CK(cudaStreamWaitEvent(h->ahead_stream, h->ahead_fork, 0));
   CK(launch_sample(h->ahead, h->ahead.cand, h->ahead_stream));
   CK(cudaEventRecord(h->ahead_done, h->ahead_stream));
-  const bool can_branch = update_reads_packed(p, false) && p.proposals;     // (the gated update is the single-kernel one)
+  const bool can_branch = update_after_pack(p, false) && p.proposals;     // (the gated update is the single-kernel one)
   bool branched = false;
   const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr, nullptr, nullptr, can_branch ? h->retry_stream : nullptr,
                                  h->retry_fork, &branched);
@@ -304,7 +305,7 @@ int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
     CK(cudaEventRecord(h->retry_done, h->retry_stream));
     CK(cudaStreamWaitEvent(main, h->retry_done, 0));
   } else {
-    CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+    CK(launch_update(p, p.kept, 1, update_after_pack(p, false), main));
   }
   h->round_host += 1;
   h->ahead_round = h->round_host;
@@ -332,7 +333,7 @@ int pipelined_rounds(strads_lasso_s* h, long long count, cudaStream_t main) {
     if (rc) return rc;
     CK(cudaEventRecord(sc.block_ready, sc.stream));
     CK(cudaStreamWaitEvent(main, sc.block_ready, 0));
-    CK(launch_update(p, p.kept, 1, update_reads_packed(p, false), main));
+    CK(launch_update(p, p.kept, 1, update_after_pack(p, false), main));
     CK(cudaEventRecord(sc.updated, main));
     h->round_host += 1;
   }

@@ -514,8 +514,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   }
 }
 
-// Exact decision for one pair the TF32 screen could not call, by a whole warp: FP64 dot product of the packed
-// columns.  Setting a bit is idempotent and order-independent, so the result is deterministic.
+// Exact decision for one pair the screen could not call, by a whole warp: FP64 dot product of the two columns of X.  Setting a bit is idempotent and order-independent, so the result is deterministic.
 __device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, int lane) {
   const long long n4 = (p.N + 3) >> 2;
   const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);

@@ -94,7 +94,7 @@ struct Problem {
   double* obj_partial;          // [2 * kObjBlocks]
   unsigned int* amb_pairs;      // [cap_amb] (a << 16 | b), positions in the candidate list
   int cap_amb;
-  float* xc;                    // dense: packed copy of the candidate columns, [n_cand][ldc]
+  float* xc;                    // (unused: no FP32 copy of the candidate columns is kept)
   long long ldc;                // N rounded up to a multiple of 4
   unsigned short* xcb;          // dense: the same columns rounded to BF16, [n_cand][ldcb]: operands of the Gram's screen
   long long ldcb;               // N rounded up to a multiple of 8
@@ -388,7 +388,7 @@ cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int g
                             cudaStream_t s);
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
                           cudaStream_t s);
-cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s, int gate = 0);
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool after_pack, cudaStream_t s, int gate = 0);
 cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s);
 cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,
                           cudaStream_t s);

@@ -52,12 +52,11 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
 // ------------------------------------------------------------------------------------------------
 // dense
 // ------------------------------------------------------------------------------------------------
-// Where the kept columns are read from.  After a tensor-core Gram they sit, contiguous and still in L2, in
-// the packed candidate buffer (row = position in the candidate list); otherwise in X itself.
+// Where the kept columns are read from: X itself.
 struct ColumnSource {
   const float* base;
   long long pitch;
-  const int* index;     // [n_kept]: packed: position in the candidate list; else: coefficient index
+  const int* index;     // [n_kept] coefficient index
 };
 
 __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __restrict__ kept, ColumnSource src) {
@@ -300,14 +299,14 @@ __global__ void k_export(Problem p, const int* kept, int* kept_out, float* dbeta
 
 }  // namespace
 
-// from_packed: the kept columns are rows p.kept_pos[.] of the packed candidate buffer (dense, after a
-// tensor-core Gram of this round); otherwise they are read from X.
-cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool from_packed, cudaStream_t s, int gate) {
+// after_pack: this round's pack kernel ran (dense, tensor-core Gram); with p.proposals it has left the changes of all
+// candidates, and p.kept_pos says where the kept ones are in the list.
+cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool after_pack, cudaStream_t s, int gate) {
   if (p.layout == STRADS_DENSE_COLMAJOR) {
     ColumnSource src;
     src.base = p.xv; src.pitch = p.ld; src.index = kept;           // the kept columns, from X itself
     cudaError_t e;
-    const int proposals = from_packed && p.proposals ? 1 : 0;     // the pack kernel of this round left the changes
+    const int proposals = after_pack && p.proposals ? 1 : 0;     // the pack kernel of this round left the changes
     if (gate != 0 && !proposals) return cudaErrorInvalidValue;    // (only the single-kernel update is gated)
     if (!proposals && (e = launch_chained(k_dot_dense, dim3(p.dot_parts, p.n_keep), kThreads, 0, s, p, kept, src)) != cudaSuccess)
       return e;
