@@ -109,16 +109,18 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
       const int i0 = min(tid * chunk, n_cand), i1 = min(i0 + chunk, n_cand);
       int mine = 0;
       for (int i = i0; i < i1; ++i) mine += state[i] == 1;
-      s_scan[tid] = mine;
-      __syncthreads();
-      for (int o = 1; o < kThreads; o <<= 1) {
-        const int v = tid >= o ? s_scan[tid - o] : 0;
-        __syncthreads();
-        s_scan[tid] += v;
-        __syncthreads();
+      int incl = mine;                                 // inclusive scan: lanes by shuffle, then the warps' totals
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
       }
-      int rank = s_scan[tid] - mine;
-      const int total = s_scan[kThreads - 1];
+      if (lane == 31) s_scan[warp] = incl;
+      __syncthreads();
+      int before = 0, total = 0;
+#pragma unroll
+      for (int w = 0; w < kThreads / 32; ++w) { const int v = s_scan[w]; if (w < warp) before += v; total += v; }
+      int rank = before + incl - mine;
       for (int i = i0; i < i1 && rank < p.n_keep; ++i) {
         if (state[i] == 1) {
           kept_out[rank] = cand[i];

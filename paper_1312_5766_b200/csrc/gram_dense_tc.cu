@@ -581,7 +581,14 @@ __global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int 
   const float4* src = reinterpret_cast<const float4*>(p.gram_partial + ((size_t)tile * n_split * kTile + la) * kTile) + lane;
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   int s = 0;
-  for (; s + 4 <= n_split; s += 4) {                   // four loads in flight, added in split order
+  for (; s + 8 <= n_split; s += 8) {                   // eight loads in flight, added in split order
+    float4 u[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) u[k] = __ldcg(src + (size_t)(s + k) * (kTile * kTile / 4));
+#pragma unroll
+    for (int k = 0; k < 8; ++k) { acc.x += u[k].x; acc.y += u[k].y; acc.z += u[k].z; acc.w += u[k].w; }
+  }
+  for (; s + 4 <= n_split; s += 4) {
     float4 u[4];
 #pragma unroll
     for (int k = 0; k < 4; ++k) u[k] = __ldcg(src + (size_t)(s + k) * (kTile * kTile / 4));
