@@ -549,3 +549,38 @@ def test_sampling_ahead_equals_round_by_round(name, cfg_over, flags):
         check()
     assert a.totals() == ref.totals()
     assert a.status()[0] == 0 and ref.status()[0] == 0
+
+
+# --------------------------------------------------------------------------------------------------
+# short columns: correlations scatter widely around rho, so the BF16 screen leaves many pairs open.  With few
+# of them the last CTA of the split-K reduce kernel rechecks them itself; beyond its budget the window is handed
+# to the whole-list retry, whose Gram has a recheck kernel (and, past its list, the 3xTF32 fallback).  Every path
+# must give the decisions of an exact Gram.
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n_rows,n_keep", [(64, 64), (64, 256), (300, 256), (24, 256)])
+def test_many_open_pairs_in_the_window(n_rows, n_keep):
+    b = _binding()
+    cfg = dict(kind="dense_iid", n_rows=n_rows, n_cols=4000, n_true=8, lam_frac=0.05, n_candidates=1024,
+               n_keep=n_keep, rho=0.1)
+    p = wl.make_problem(cfg, seed=17)
+    X = oracle_matrix(p)
+    n2 = oracle.colnorm2(X)
+    rho = float(np.float32(p.rho))
+    lazy, full = _solver(p), _solver(p, flags=b.FLAG_FULL_GRAM)
+    rng = np.random.default_rng(8)
+    for trial in range(3):
+        cand = rng.permutation(p.n_cols)[: p.n_candidates].astype(np.int32)
+        cd = torch.from_numpy(cand).cuda()
+        kept_l, counts_l = lazy.filter(cd)
+        kept_f, counts_f = full.filter(cd)
+        assert torch.equal(kept_l, kept_f) and torch.equal(counts_l, counts_f), (n_rows, n_keep, trial)
+        c = counts_l.cpu().numpy(); nk = int(c[2])
+        _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept_l.cpu().numpy()[:nk], int(c[1]))
+    assert lazy.status()[0] == 0 and full.status()[0] == 0
+    # and whole rounds through strads_run equal rounds one by one on such data too
+    a, ref = _solver(p), _solver(p)
+    a.run(20)
+    for _ in range(20):
+        ref.round()
+    for x, y in ((a.beta, ref.beta), (a.resid, ref.resid), (a.delta, ref.delta)):
+        assert torch.equal(x, y)
