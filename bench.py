@@ -345,7 +345,7 @@ def main():
                                   f"region ({sec:.1f} s, single thread; host has {os.cpu_count()} cores)"}
 
     # kernels launched per round (the library's fixed sequence; launches of the whole-list retry return at once when
-    # the window sufficed): sampler hist (+ its full repeat for J >= 2^22, returns at once) + collect (winners grouped by histogram bin) + ordering (ranks inside the groups);
+    # the window sufficed): sampler hist + collect (winners grouped by histogram bin) + ordering (ranks inside the groups);
     # dense Gram of n candidates: pack, screen, split-K reduce (few tiles only), recheck, and a 3xTF32 launch unless a
     # retry follows; CSC Gram: bucket fill, bucket pairs, pair bits, all-pairs fallback; walk 1; update: dense 1 (the
     # pack kernel has formed the changes), CSC 3
@@ -358,7 +358,7 @@ def main():
         if retry_follows and split:
             return 3                   # pack, screen, reduce (whose last CTA also rechecks the open pairs)
         return 3 + (1 if split else 0) + (0 if retry_follows else 1)
-    launches_per_round = 2 + (1 if p.n_cols >= (1 << 22) else 0) + 1 + (1 if p.layout == wl.DENSE else 3)
+    launches_per_round = 2 + 1 + (1 if p.layout == wl.DENSE else 3)
     sampling_ahead = p.layout == wl.DENSE and p.n_keep <= 4096
     if sampling_ahead:
         launches_per_round += 1        # the early list's correction; the early draw itself launches what a plain draw does

@@ -161,7 +161,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_patch_keys = take(sizeof(unsigned long long) * 2 * (size_t)c->n_keep);
   L.off_cand_keys = take(dense ? sizeof(unsigned long long) * 2 * (size_t)c->n_candidates : 0);
   // keys the sampler's guided first pass saves for its collect pass (many coefficients only): 8 P' of them
-  L.cap_survivors = c->n_cols >= (1 << 22) ? 8 * c->n_candidates : 0;
+  L.cap_survivors = c->n_cols >= (1 << 19) ? 8 * c->n_candidates : 0;
   L.off_survivors = take(sizeof(unsigned long long) * (size_t)L.cap_survivors);
   L.off_bin_off = take(sizeof(int) * (kHistBins + 1));
   L.off_bin_cur = take(sizeof(unsigned int) * kHistBins);

@@ -162,10 +162,9 @@ __device__ void find_bin(const unsigned int* h, int nbins, long long k_rem, int*
 
 // mode 0: plain.  mode 1: bins only the keys below a cutoff carried over from the previous round (four times that
 // round's boundary; the keys certainly above it are not even computed); if fewer than P' keys turn out to lie
-// below it, nothing is published and the launch behind (mode 2: plain, and only then) does the pass again.
+// below it, the last CTA redoes the pass in full by itself.
 __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
   chain_begin();
-  if (mode == 2 && !p.st->sample_redo) return;
   __shared__ unsigned int sh[kHistBins];
   __shared__ int s_last;
   __shared__ SelectState s_sel;
@@ -224,6 +223,7 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
   __syncthreads();
   __shared__ int s_bin;
   __shared__ long long s_before;
+  bool solo = false;
   if (cut > 0.f) {                                     // enough keys below the cutoff?
     __shared__ unsigned int s_total;
     if (tid == 0) s_total = 0u;
@@ -233,14 +233,22 @@ __global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
     atomicAdd(&s_total, mine);
     __syncthreads();
     if (s_total < (unsigned)p.n_cand) {
-      if (tid == 0) { p.st->hist_ticket = 0; p.st->sample_redo = 1; p.st->t_cut = 0.f; p.st->surv_valid = 0; }
-      return;
+      // The guide was too low (the weights collapsed since the last round: the end of the first sweep, say).  Rare,
+      // so this CTA redoes the pass alone and in full rather than the whole grid being launched a second time every
+      // round just in case: some milliseconds once, for 10^7 coefficients.
+      solo = true;
+      __syncthreads();
+      for (int b = tid; b < kHistBins; b += kThreads) sh[b] = 0;
+      __syncthreads();
+      for (long long g = tid; g < groups; g += kThreads)
+        for_keys_of_group(p, t, g, 0.f, [&](unsigned long long key) { atomicAdd(&sh[(unsigned int)(key >> (64 - kHistBits))], 1u); });
+      __syncthreads();
     }
   }
   find_bin(sh, kHistBins, p.n_cand, &s_bin, &s_before);
   if (tid == 0) {
     // (every CTA's appends are done and visible: they precede its ticket)
-    p.st->surv_valid = (save && __ldcg(&p.st->surv_count) <= (unsigned)p.cap_survivors) ? 1 : 0;
+    p.st->surv_valid = (save && !solo && __ldcg(&p.st->surv_count) <= (unsigned)p.cap_survivors) ? 1 : 0;
     p.st->sample_redo = 0;
     // next round's cutoff: four times the upper edge of this boundary bin (none if that is not a finite number)
     const unsigned int edge = ((unsigned int)s_bin + 1u) << (32 - kHistBits);
@@ -615,11 +623,10 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   cudaError_t e;
-  // many coefficients: the first pass leaves out the keys far above the last boundary (and a second launch
-  // repeats it in full in the rare round where that boundary was a bad guide)
-  const bool guided = p.J >= (1 << 22);     // (below that the passes are bound by latency, not by arithmetic)
+  // many coefficients: the first pass leaves out the keys far above the last boundary (its last CTA repeats it in
+  // full in the rare round where that boundary was a bad guide)
+  const bool guided = p.J >= (1 << 19);     // (below that the passes are bound by latency, not by arithmetic)
   if ((e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, guided ? 1 : 0)) != cudaSuccess) return e;
-  if (guided && (e = launch_chained(k_sample_hist, (unsigned)blocks, kThreads, 0, s, p, 2)) != cudaSuccess) return e;
   if ((e = launch_chained(k_sample_collect, (unsigned)blocks, kThreads, 0, s, p)) != cudaSuccess) return e;
   if (p.bin_off != nullptr)
     return launch_chained(k_sample_rank_bins, (unsigned)((p.cap_sure + p.cap_boundary + 31) / 32), 256, 0, s, p, cand_out);
