@@ -256,7 +256,7 @@ def main():
         flops = float(window) * (window - 1) * p.n_rows
         achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
         peak = peaks["bf16_tflops"]                          # the screen multiplies BF16 roundings of the columns
-        roofline = {"kernel": "k_gram_dense_tc<screen> (+ k_gram_reduce, k_gram_recheck)", "bound": "tensor",
+        roofline = {"kernel": "k_gram_dense_tc<screen> (+ k_gram_reduce, whose last CTA rechecks the open pairs)", "bound": "tensor",
                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                     "traffic": GRAM_WINDOW_TRAFFIC.get((args.workload, window)),
                     "window": window, "launch_ms": step_ms["gram_ms"],
