@@ -19,7 +19,8 @@
  *   - every array is allocated, owned and freed by the caller; the handle owns
  *     only host bookkeeping.  X and y are never written and must outlive the
  *     handle, as must beta, resid, delta and the workspace;
- *   - the library allocates no device memory;
+ *   - the library allocates no device memory (strads_sample_static keeps about 65 KB of scratch in a
+ *     fixed device array of its own instead of a workspace);
  *   - arguments are validated on the host before anything is launched; nothing
  *     traps, aborts or waits without a bound;
  *   - calls are asynchronous on the configured stream unless stated otherwise;
@@ -60,15 +61,20 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
 #define STRADS_FLAG_SIMT_GRAM     4u   /* dense Gram on the FP32 SIMT kernel instead of the
                                           tensor-core kernels                                  */
 #define STRADS_FLAG_GRAM_3XTF32   8u   /* dense Gram always by the 3xTF32 tensor-core kernel
-                                          (default: TF32 screen + exact recheck of the pairs
-                                          within 2^-8 of rho; 3xTF32 only if those overflow)   */
+                                          (default: a screen on BF16 roundings of the columns,
+                                          then an exact FP64 recheck of every pair whose
+                                          correlation it puts within 2^-7 + N 2^-25 of rho, so
+                                          that Algorithm 1's rho test is decided exactly;
+                                          3xTF32 only if the list of such pairs overflows)     */
 
 #define STRADS_FLAG_FULL_GRAM    16u   /* form the conflict bits of ALL P' candidates before the
                                           walk (default: of a leading window of 1.5 P + 128 first,
                                           of all P' only if the walk runs out of the window)    */
 
 /* limits */
-#define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (one CTA sorts the winners in shared memory) */
+#define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (positions in the candidate list are packed into 16 bits
+                                           in the lists of pairs; the walk holds P' / 32 mask words per CTA) */
+#define STRADS_MAX_C_INIT 1e18f         /* c_init^2 + eta must stay finite in binary32 */
 #define STRADS_MAX_SCHEDULERS 8
 
 typedef struct {
@@ -86,7 +92,7 @@ typedef struct {
   float    lambda;                      /* > = 0                                                    */
   float    eta;                         /* > 0   (paper: 1e-6 in the experiments)                   */
   float    rho;                         /* > 0   (paper: 0.1)                                       */
-  float    c_init;                      /* > 0, Algorithm 1's "very large" C; 1e4 recommended       */
+  float    c_init;                      /* 0 < C <= STRADS_MAX_C_INIT, Algorithm 1's "very large" C; 1e4 recommended */
   int32_t  n_candidates;                /* P': 1 <= P' <= min(J, STRADS_MAX_CANDIDATES)             */
   int32_t  n_keep;                      /* P : 1 <= P <= P'                                         */
   uint64_t seed;                        /* Philox key                                               */
@@ -179,7 +185,10 @@ int strads_filter(strads_handle_t h, const int32_t* cand_dev, int32_t n_cand,
 int strads_update(strads_handle_t h, const int32_t* kept_dev, int32_t n_kept, float* dbeta_dev);
 
 /* Round index t (0-based; the Philox counter).  With beta, resid, delta and the seed it is the
- * whole resumable state. */
+ * whole resumable state.  strads_run keeps the candidates it has drawn ahead for the next round; whoever
+ * writes beta, resid or delta directly (a restored checkpoint, priorities set by hand) must call
+ * strads_set_round afterwards -- with the current index if it is unchanged -- which discards that list, so
+ * that the next round draws from the state as it now is. */
 int strads_get_round(strads_handle_t h, int64_t* t_host_out);
 int strads_set_round(strads_handle_t h, int64_t t);
 
@@ -192,9 +201,31 @@ int strads_totals(strads_handle_t h, int64_t* totals_host_out /* [4] */);
 #define STRADS_STATUS_SAMPLER_REFINED 1u   /* informational: the sampler needed extra select passes */
 #define STRADS_STATUS_NONFINITE       2u   /* a gradient x_j^T r was NaN or Inf                     */
 #define STRADS_STATUS_WAIT_EXPIRED    4u   /* a bounded wait in a kernel gave up                     */
-#define STRADS_STATUS_GRAM_FALLBACK   8u   /* informational: the dense Gram's TF32 screen left more
+#define STRADS_STATUS_GRAM_FALLBACK   8u   /* informational: the dense Gram's BF16 screen left more
                                               borderline pairs than its list holds; 3xTF32 was used  */
 int strads_status(strads_handle_t h, uint32_t* bits_host_out);
+
+/* The error contract of the bounded waits ("nothing waits without a bound").  Every device-side wait of the
+ * round -- the mbarrier waits of the dense Gram's TMA / tensor-core pipeline (SAP step 2) and the grid-wide
+ * barrier of the CSC on-demand walk -- counts its iterations; past the limit the CTA raises
+ * STRADS_STATUS_WAIT_EXPIRED, stops issuing work, releases its tensor memory and returns, so the launch ends and
+ * strads_status reports STRADS_ERR_TIMEOUT.  From then on the round's outputs and beta / resid / delta are
+ * undefined, and the CSC walk does nothing on this handle, until strads_recover has been called:
+ *   restore beta, resid, delta from a copy of your own, strads_recover, strads_set_round, carry on.
+ * strads_set_wait_limit: iteration limit for all those waits on this handle (0 = the kernels' defaults, which
+ *   amount to seconds); synchronises the stream and drops the captured launch sequence of strads_run.
+ * strads_inject_stall: makes a wait of the NEXT launches run out, so that the path above can be exercised: with
+ *   STRADS_STALL_WALK_BARRIER the arrival counter of the CSC walk's barrier is set to a value no barrier completes
+ *   from; with STRADS_STALL_GRAM_LOADS the dense Gram's producer withholds its operand loads (until
+ *   strads_recover).  Nothing faults or hangs: the waits give up.  Refused (STRADS_ERR_INVALID_ARG) unless a
+ *   limit of at most STRADS_STALL_MAX_WAIT_LIMIT iterations is in force, so that giving up takes milliseconds.
+ * strads_recover: waits for the stream, clears the status word and the barrier state, ends an injected stall. */
+#define STRADS_STALL_WALK_BARRIER 1
+#define STRADS_STALL_GRAM_LOADS   2
+#define STRADS_STALL_MAX_WAIT_LIMIT 65536u
+int strads_set_wait_limit(strads_handle_t h, uint32_t iterations);
+int strads_inject_stall(strads_handle_t h, int32_t which);
+int strads_recover(strads_handle_t h);
 
 /* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);

@@ -23,13 +23,14 @@ FLAG_SIMT_GRAM = 4
 FLAG_GRAM_3XTF32 = 8
 FLAG_FULL_GRAM = 16
 MAX_CANDIDATES = 16384
+STALL_WALK_BARRIER, STALL_GRAM_LOADS = 1, 2
 
 EXPORTS = [
     "strads_workspace_bytes", "strads_lasso_init", "strads_round", "strads_run", "strads_round_host",
     "strads_objective", "strads_sample", "strads_filter", "strads_update", "strads_get_round",
     "strads_set_round", "strads_totals", "strads_status", "strads_colnorm2", "strads_destroy",
     "strads_error_string", "strads_last_cuda_error", "strads_profile_begin", "strads_profile_end",
-    "strads_sample_static",
+    "strads_sample_static", "strads_set_wait_limit", "strads_inject_stall", "strads_recover",
 ]
 
 
@@ -84,6 +85,9 @@ def load() -> C.CDLL:
         lib.strads_colnorm2.argtypes = [C.c_void_p, C.POINTER(C.c_void_p)]
         lib.strads_destroy.argtypes = [C.c_void_p]
         lib.strads_profile_begin.argtypes = [C.c_void_p, C.c_int64]
+        lib.strads_set_wait_limit.argtypes = [C.c_void_p, C.c_uint32]
+        lib.strads_inject_stall.argtypes = [C.c_void_p, C.c_int32]
+        lib.strads_recover.argtypes = [C.c_void_p]
         lib.strads_sample_static.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_uint64, C.c_uint64, C.c_int32,
                                              C.c_uint32, C.c_void_p, C.c_void_p]
         lib.strads_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -254,6 +258,15 @@ class StradsLasso:
         bits = C.c_uint32(0)
         rc = load().strads_status(self._h, C.byref(bits))
         return rc, int(bits.value)
+
+    def set_wait_limit(self, iterations: int) -> None:
+        _check(load().strads_set_wait_limit(self._h, int(iterations)), "strads_set_wait_limit")
+
+    def inject_stall(self, which: int) -> None:
+        _check(load().strads_inject_stall(self._h, int(which)), "strads_inject_stall")
+
+    def recover(self) -> None:
+        _check(load().strads_recover(self._h), "strads_recover")
 
     def colnorm2(self) -> torch.Tensor:
         """||x_j||^2 (FP64), a view into the workspace."""

@@ -81,7 +81,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xc, off_xcb, off_partial, off_walk_blocked, off_walk_rows, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xcb, off_partial, off_walk_blocked, off_walk_ctl,
       off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
@@ -137,17 +137,15 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_dot_partial = take(sizeof(double) * (size_t)c->n_keep * L.dot_parts);
   L.off_dot_ticket = take(sizeof(unsigned int) * (size_t)c->n_keep);
   L.off_obj = take(first ? sizeof(double) * 2 * kObjBlocks : 0);
-  L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // borderline pairs of the TF32 screen (1 MB)
+  L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // pairs the BF16 screen leaves to the exact recheck (1 MB)
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
   L.ldc = (c->n_rows + 3) / 4 * 4;
-  L.off_xc = take(0);                                                  // (no FP32 copy of the candidates is kept)
   L.ldcb = (c->n_rows + 7) / 8 * 8;
   L.off_xcb = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(unsigned short) * (size_t)c->n_candidates * L.ldcb : 0);
   L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)
   L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
-  L.off_walk_rows = take(0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
   // CSC Gram by row buckets: provided for while the buckets stay below 64 MB (N <= 2^20)
   const bool buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);
@@ -367,7 +365,6 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.obj_partial = first ? first->obj_partial : reinterpret_cast<double*>(ws + L.off_obj);
   p.amb_pairs = reinterpret_cast<unsigned int*>(ws + L.off_amb);
   p.cap_amb = L.cap_amb;
-  p.xc = reinterpret_cast<float*>(ws + L.off_xc);
   p.ldc = L.ldc;
   p.xcb = reinterpret_cast<unsigned short*>(ws + L.off_xcb);
   p.ldcb = L.ldcb;
@@ -378,7 +375,6 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.proposals = (c->layout == STRADS_DENSE_COLMAJOR && S == 1) ? 1 : 0;
   p.cand_cur = nullptr;
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
-  p.walk_rows = reinterpret_cast<unsigned int*>(ws + L.off_walk_rows);
   p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
   p.resid_acc = reinterpret_cast<long long*>(ws + L.off_resid_acc);
   p.pair_cap = L.pair_cap;
@@ -402,6 +398,7 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
                      ? reinterpret_cast<unsigned long long*>(ws + L.off_patch_keys) : nullptr;
   p.cand_keys = reinterpret_cast<unsigned long long*>(ws + L.off_cand_keys);
   p.cap_edges = kEdgeCap;
+  p.wait_limit = 0; p.stall = 0;
 }
 
 // The early draw's view: everything of scheduler 0, except its own sampler state and buffers, P' + P winners with
@@ -468,6 +465,9 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
     return STRADS_ERR_INVALID_ARG;
   if (!(c->lambda >= 0.f) || !(c->eta > 0.f) || !(c->rho > 0.f) || !(c->c_init > 0.f)) return STRADS_ERR_INVALID_ARG;
   if (!std::isfinite(c->lambda) || !std::isfinite(c->eta) || !std::isfinite(c->c_init)) return STRADS_ERR_INVALID_ARG;
+  // the weight C^2 + eta must stay finite in binary32, or every never-updated coefficient's race time is 0 and the
+  // first phase turns from a randomised sweep into one in index order
+  if (c->c_init > STRADS_MAX_C_INIT) return STRADS_ERR_INVALID_ARG;
   const int S = n_sched_of(c);
   const Layout L = carve(c), Lrest = carve(c, false);
   if (c->workspace_bytes < L.total + (size_t)(S - 1) * Lrest.total) return STRADS_ERR_WORKSPACE_TOO_SMALL;
@@ -559,7 +559,7 @@ static long long graph_rounds(const strads_lasso_s* h) {
 // the legacy default stream, which cannot be captured; nothing executes during capture).  With several
 // schedulers the sequence starts with scheduler 0.
 static int build_round_graph(strads_lasso_s* h) {
-  {
+  if (h->capture_stream == nullptr) {
     int prio_least = 0, prio_greatest = 0;
     CK(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
     CK(cudaStreamCreateWithPriority(&h->capture_stream, cudaStreamNonBlocking, prio_greatest));
@@ -749,6 +749,57 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
   if (bits_host_out) *bits_host_out = bits;
   if (bits & STRADS_STATUS_WAIT_EXPIRED) return STRADS_ERR_TIMEOUT;
   if (bits & STRADS_STATUS_NONFINITE) return STRADS_ERR_NUMERIC;
+  return STRADS_OK;
+}
+
+// The captured launch sequence holds copies of the kernels' arguments: drop it when one of them changes.
+static void drop_round_graph(strads_lasso_s* h) {
+  if (h->round_exec != nullptr) { cudaGraphExecDestroy(h->round_exec); h->round_exec = nullptr; }
+  if (h->round_graph != nullptr) { cudaGraphDestroy(h->round_graph); h->round_graph = nullptr; }
+}
+
+int strads_set_wait_limit(strads_handle_t h, uint32_t iterations) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->stream));
+  for (int s = 0; s < h->n_sched; ++s) h->sch[s].p.wait_limit = iterations;
+  h->ahead.wait_limit = iterations;
+  drop_round_graph(h);
+  return STRADS_OK;
+}
+
+int strads_inject_stall(strads_handle_t h, int32_t which) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  Scheduler& sc = on_turn(h);
+  // only with a short limit in force: the stalled wait then gives up within milliseconds
+  if (sc.p.wait_limit == 0 || sc.p.wait_limit > STRADS_STALL_MAX_WAIT_LIMIT) return STRADS_ERR_INVALID_ARG;
+  if (which == STRADS_STALL_WALK_BARRIER) {
+    if (sc.p.layout != STRADS_CSC) return STRADS_ERR_INVALID_ARG;
+    // an arrival count no barrier of the walk can complete from
+    CK(cudaMemsetAsync(&sc.p.walk_ctl->bar_count, 0x40, sizeof(unsigned int), h->stream));
+  } else if (which == STRADS_STALL_GRAM_LOADS) {
+    if (sc.p.layout != STRADS_DENSE_COLMAJOR) return STRADS_ERR_INVALID_ARG;
+    sc.p.stall = 1;
+    drop_round_graph(h);
+  } else {
+    return STRADS_ERR_INVALID_ARG;
+  }
+  return STRADS_OK;
+}
+
+int strads_recover(strads_handle_t h) {
+  if (h == nullptr) return STRADS_ERR_INVALID_ARG;
+  CK(cudaStreamSynchronize(h->stream));
+  bool had_stall = false;
+  for (int s = 0; s < h->n_sched; ++s) {
+    Problem& p = h->sch[s].p;
+    had_stall = had_stall || p.stall != 0;
+    p.stall = 0;
+    CK(cudaMemsetAsync(&p.st->status, 0, sizeof(unsigned int), h->stream));
+    if (p.layout == STRADS_CSC) CK(cudaMemsetAsync(p.walk_ctl, 0, sizeof(WalkControl), h->stream));
+  }
+  if (had_stall) drop_round_graph(h);
+  h->ahead_round = -1;                                   // (whatever was drawn ahead belongs to the abandoned rounds)
+  CK(cudaStreamSynchronize(h->stream));
   return STRADS_OK;
 }
 

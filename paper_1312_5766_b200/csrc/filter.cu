@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
   if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
-    // dense window whose TF32 screen left more borderline pairs than the list holds: its bits are incomplete;
+    // dense window whose BF16 screen left more borderline pairs than the list holds: its bits are incomplete;
     // the whole-list retry (which has the 3xTF32 fallback) takes over
     if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; p.st->edge_count = 0; p.st->edges_off = 0; }
     return;

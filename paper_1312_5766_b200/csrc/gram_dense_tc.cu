@@ -1,11 +1,11 @@
 // SAP step 2, dense X, on the 5th-generation tensor cores: conflict bits of all candidate pairs from
 // G = X_C^T X_C, a genuine dense contraction (M = N' = P', K = the N samples).
 //
-//   k_pack_candidates   copies the P' candidate columns into one contiguous [P'][ldc] buffer, and a copy
-//                       rounded to BF16 beside it.  The candidates are scattered over the whole design
+//   k_pack_candidates   writes the P' candidate columns, rounded to BF16, into one contiguous [P'][ldcb]
+//                       buffer: the screen's operands.  The candidates are scattered over the whole design
 //                       matrix (one 2 MB page each for a 4 GB X); gathering them once makes every later
 //                       access TLB- and TMA-friendly (measured: the same GEMM runs 2x slower straight
-//                       from scattered columns).
+//                       from scattered columns).  With one scheduler it also forms x_c^T r on the way.
 //   k_gram_dense_tc<0>  "screen": one CTA per 128 x 128 tile of the upper triangle of tile pairs; one
 //                       thread feeds a 3-stage ring of 64 KB stages with TMA tile loads of the BF16 copy
 //                       (128-byte swizzle, zero fill past N and P'), one thread issues tcgen05.mma
@@ -60,15 +60,15 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-// One TMA tile load: box {32 floats, 128 rows} at element coordinates (x = k, y = row) -> shared memory.
+// One TMA tile load: box {64 BF16 elements, 128 rows} at element coordinates (x = k, y = row) -> shared memory.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const void* tmap, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 // Bounded wait for the phase with the given parity; false = gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t it = 0; it < kWaitLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
@@ -305,6 +305,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && p.st->amb_count <= (unsigned)p.cap_amb) return;
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitLimit;
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && blockIdx.x == 0 && tid == 0)
     atomicOr(&p.st->status, STRADS_STATUS_GRAM_FALLBACK);
   // With n_split > 1 the K range of a tile is shared by n_split CTAs, each leaving an FP32 partial tile that
@@ -346,12 +347,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     for (int st = 0; st < n_st; ++st) {
       const int s = st % kStages;
       bool got = !s_abort;
-      if (got && st >= kStages) got = mbar_wait(empty0 + 8 * s, (uint32_t)(st / kStages - 1) & 1u);
+      if (got && st >= kStages) got = mbar_wait(empty0 + 8 * s, (uint32_t)(st / kStages - 1) & 1u, wait_limit);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
         break;
       }
-      if (lane == 0) {
+      if (lane == 0 && !p.stall) {                     // (stall: the loads are withheld and the MMA warp's wait runs out)
         const uint32_t sb = tiles0 + (uint32_t)s * kStageBytes, bar = full0 + 8 * s;
         mbar_arrive_expect_tx(bar, (uint32_t)kStageBytes);
 #pragma unroll
@@ -413,7 +414,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       const int nxt = st + kAhead;                     // refill the stage that st - 1 used
       if (nxt < n_st) {
         bool got = !s_abort;
-        if (got && nxt >= kStages) got = mbar_wait(empty0 + 8 * (nxt % kStages), (uint32_t)(nxt / kStages - 1) & 1u);
+        if (got && nxt >= kStages) got = mbar_wait(empty0 + 8 * (nxt % kStages), (uint32_t)(nxt / kStages - 1) & 1u, wait_limit);
         if (!__all_sync(0xffffffffu, got)) {
           if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
           break;
@@ -432,7 +433,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     for (int st = 0; st < n_st; ++st) {
       const int s = st % kStages;
       const uint32_t ph = (uint32_t)(st / kStages) & 1u;
-      const bool got = !s_abort && mbar_wait(full0 + 8 * s, ph);
+      const bool got = !s_abort && mbar_wait(full0 + 8 * s, ph, wait_limit);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
         break;
@@ -475,7 +476,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
       asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps see all of them
     }
-    bool ok = !s_abort && mbar_wait(done_bar, 0u);
+    bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
     ok = __all_sync(0xffffffffu, ok);
     if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

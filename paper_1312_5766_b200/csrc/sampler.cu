@@ -11,10 +11,14 @@
 //                    the rest).  For an exponential race the boundary bin holds < ~0.1 P' keys in
 //                    expectation whatever the weights are; if it ever exceeds the boundary buffer,
 //                    that CTA alone refines the boundary over further 12-bit digits (rare, exact).
-//   k_sample_collect pass 2: appends "sure" and "boundary" keys to two small buffers.
-//   k_sample_rank_direct (P' <= 2048)  orders the winners by counting, for every key, the smaller ones.
-//   k_sample_sort_chunks / k_sample_rank (larger P')  1024-key chunks sorted in shared memory by
-//                    one CTA each, then every key's rank by binary search in the other chunks.
+//   k_sample_collect pass 2: a "sure" key goes to the group of its histogram bin in the `sure` buffer (group
+//                    offsets from the first pass's counts), a "boundary" key to the boundary buffer.
+//   k_sample_rank_bins  (the default) orders the winners: bins are in key order already, so every key is
+//                    ranked inside its own group only, and the boundary keys among themselves.
+//   k_sample_patch   corrects a list drawn one round ahead for the coefficients the last update changed.
+//   k_sample_rank_direct (P' <= 2048) / k_sample_sort_chunks + k_sample_rank (larger P'): ordering without
+//                    group arrays (counting over the whole buffer; 1024-key chunk sorts in shared memory,
+//                    then ranks by binary search in the other chunks); used by strads_sample_static.
 #include <cstddef>
 #include <mutex>
 

@@ -29,7 +29,7 @@ struct DeviceState {
   double objective;             // result slot of the objective reduction
   float x_abs_max;              // max |x_ij| (CSC: bounds the fixed-point residual update)
   int beta0_nonzero;            // set at init when the starting beta has a non-zero entry
-  unsigned int amb_count;       // pairs the TF32 screen of the dense Gram left to the exact recheck
+  unsigned int amb_count;       // pairs the BF16 screen of the dense Gram left to the exact recheck
   int window_short;             // the filter ran out of its candidate window before P were kept: redo on all P'
   int prefer_walk;              // CSC: the last round needed the whole list, so skip the window attempt for a while
   unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
@@ -94,7 +94,6 @@ struct Problem {
   double* obj_partial;          // [2 * kObjBlocks]
   unsigned int* amb_pairs;      // [cap_amb] (a << 16 | b), positions in the candidate list
   int cap_amb;
-  float* xc;                    // (unused: no FP32 copy of the candidate columns is kept)
   long long ldc;                // N rounded up to a multiple of 4
   unsigned short* xcb;          // dense: the same columns rounded to BF16, [n_cand][ldcb]: operands of the Gram's screen
   long long ldcb;               // N rounded up to a multiple of 8
@@ -107,7 +106,6 @@ struct Problem {
   float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
   int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles
   unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words], OR-ed into by the whole grid
-  unsigned int* walk_rows;      // (unused)
   WalkControl* walk_ctl;
   long long* resid_acc;         // CSC: [N] fixed-point accumulators of the residual update (zero between rounds)
   // CSC Gram by row buckets (null / 0 when not provided for)
@@ -134,6 +132,10 @@ struct Problem {
   int cap_edges;
   // scheduler threads: this Problem is scheduler part_index of part_count and owns { j : j mod part_count == part_index }
   int part_count, part_index;
+  // bounded device-side waits: iteration limit of every spin (0: each kernel's own default), and, for exercising the
+  // expiry path, a launch whose operand loads are withheld so that a wait does run out (strads_inject_stall)
+  unsigned int wait_limit;
+  int stall;
 };
 static constexpr int kObjBlocks = 296;
 

@@ -42,7 +42,7 @@ __device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
 }
 
 // Grid-wide barrier.  Returns false when the wait gave up (or an earlier one did).
-__device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* status) {
+__device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* status, unsigned int limit) {
   __shared__ int s_ok;
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -56,7 +56,7 @@ __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* 
       atomicAdd(&c->bar_gen, 1u);
     } else {
       unsigned int it = 0;
-      while (*gen == g && ++it < kSpinLimit) {}
+      while (*gen == g && ++it < limit) {}
       if (*gen == g) { ok = false; atomicOr(status, STRADS_STATUS_WAIT_EXPIRED); c->failed = 1; }
     }
     __threadfence();
@@ -70,6 +70,10 @@ __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* 
 __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __restrict__ cand, int n_cand,
                                                         int only_if_short, int* __restrict__ kept_out) {
   if (only_if_short && !p.st->window_short) return;      // uniform over the grid: nobody reaches a barrier
+  // a wait that expired in an earlier launch left the barrier's counter where it was: nothing runs on this handle
+  // until strads_recover has cleared it (CTAs that disagree on this bit only meet a barrier that gives up)
+  if (p.st->status & STRADS_STATUS_WAIT_EXPIRED) return;
+  const unsigned int spin_limit = p.wait_limit ? p.wait_limit : kSpinLimit;
   __shared__ unsigned int blocked[kMaxWords];
   __shared__ int brow[kBatch][kColCap];
   __shared__ float bval[kBatch][kColCap];
@@ -91,7 +95,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
   if (blockIdx.x == 0)
     for (int w = tid; w < W; w += kThreads) blocked_g[w] = 0u;
   if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = n_cand; s_done = 0; }
-  bool ok = grid_barrier(c, n_ctas, &p.st->status);       // nobody ORs into the global mask before it is cleared
+  bool ok = grid_barrier(c, n_ctas, &p.st->status, spin_limit);       // nobody ORs into the global mask before it is cleared
 
   while (ok) {
     // ---- A: the next <= 32 candidates at or after the cursor that are not blocked (warp 0) ----
@@ -224,7 +228,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
         if (lane == 0 && word != 0u) atomicOr(&blocked_g[w], word);
       }
     }
-    ok = grid_barrier(c, n_ctas, &p.st->status);
+    ok = grid_barrier(c, n_ctas, &p.st->status, spin_limit);
     if (!ok) break;
     for (int w = tid; w < W; w += kThreads) blocked[w] = __ldcg(&blocked_g[w]);
     __syncthreads();

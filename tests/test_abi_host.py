@@ -92,7 +92,9 @@ def test_init_rejects_bad_pointers_and_parameters_without_touching_the_gpu(lib):
     for field, value, want in [("x_values", None, -1), ("y", None, -1), ("workspace", None, -1),
                                ("x_values", 0x10004, -1), ("delta", 0x10008, -1), ("workspace", 0x10010, -1),
                                ("eta", 0.0, -1), ("rho", -0.1, -1), ("lam", -1.0, -1), ("c_init", 0.0, -1),
-                               ("lam", float("nan"), -1), ("workspace_bytes", 16, -3), ("layout", 3, -2)]:
+                               ("lam", float("nan"), -1), ("workspace_bytes", 16, -3), ("layout", 3, -2),
+                               # C^2 + eta must stay finite in binary32 (else every first-phase race time is 0)
+                               ("c_init", 2e18, -1), ("c_init", float("inf"), -1)]:
         cfg = cfg_ok()
         setattr(cfg, field, value)
         assert lib.strads_lasso_init(C.byref(cfg), C.byref(h)) == want, field
@@ -104,3 +106,5 @@ def test_init_rejects_bad_pointers_and_parameters_without_touching_the_gpu(lib):
     # NULL handles
     assert lib.strads_round(None, None) == -1 and lib.strads_run(None, 1) == -1
     assert lib.strads_objective(None, None) == -1 and lib.strads_destroy(None) == -1
+    assert lib.strads_set_wait_limit(None, 10) == -1 and lib.strads_inject_stall(None, 1) == -1
+    assert lib.strads_recover(None) == -1

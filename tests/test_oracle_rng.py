@@ -11,7 +11,6 @@ import subprocess
 import sys
 
 import numpy as np
-import pytest
 
 import oracle
 
@@ -43,8 +42,8 @@ def _triton_philox(cases):
     env = dict(os.environ, TRITON_INTERPRET="1", CUDA_VISIBLE_DEVICES="")
     p = subprocess.run([sys.executable, "-c", _TRITON_SNIPPET, json.dumps(cases)], env=env,
                        capture_output=True, text=True, timeout=600)
-    if p.returncode != 0:
-        pytest.skip("Triton CPU interpreter unavailable: " + p.stderr[-300:])
+    # no skip: without this independent implementation the oracle's Philox would silently lose its pin
+    assert p.returncode == 0, "Triton's CPU interpreter (the independent Philox4x32-10) did not run: " + p.stderr[-600:]
     line = [ln for ln in p.stdout.splitlines() if ln.startswith("RESULT")][-1]
     return json.loads(line[len("RESULT"):])
 

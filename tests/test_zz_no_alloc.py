@@ -4,12 +4,13 @@ Some users of this library run where cudaMalloc is off limits -- inside another 
 or in a loop that must not touch the allocator -- so this entry point keeps its scratch memory in a fixed
 array inside the library.  It must give exactly the list the handle-based strads_sample gives, also when
 called twice in a row (the array keeps the previous call's contents), and refuse sizes its array cannot
-hold.  Collected last on purpose: a run that stops at the first failure has then run every other test.
+hold.  The list is also compared with the CPU oracle's ranking of all keys.  Collected last on purpose: a run that stops at the first failure has then run every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1312_5766_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -33,6 +34,7 @@ def test_static_sampler_matches_the_handle_based_one_twice_in_a_row():
         want = s.sample().clone()
         got = b.sample_static(delta, p.eta, seed, t, n_cand, out=out)
         assert torch.equal(got, want), (call, t)
+        assert np.array_equal(got.cpu().numpy(), oracle.sample(delta.cpu().numpy().astype(np.float64), p.eta, seed, t, n_cand))
         # and again, straight after, on the array the previous call left behind
         got2 = b.sample_static(delta, p.eta, seed, t, n_cand, out=out)
         assert torch.equal(got2, want), (call, t)
@@ -48,7 +50,9 @@ def test_static_sampler_matches_the_handle_based_one_twice_in_a_row():
     s300.set_round(1)
     want300 = s300.sample().clone()
     assert torch.equal(want300, want)
-    assert torch.equal(b.sample_static(delta, p.eta, seed, 1, 300), want300)
+    got300 = b.sample_static(delta, p.eta, seed, 1, 300)
+    assert torch.equal(got300, want300)
+    assert np.array_equal(got300.cpu().numpy(), oracle.sample(delta.cpu().numpy().astype(np.float64), p.eta, seed, 1, 300))
 
 
 def test_static_sampler_rejects_what_its_array_cannot_hold():
@@ -62,4 +66,4 @@ def test_static_sampler_rejects_what_its_array_cannot_hold():
     assert e.value.code == -1
     # the largest allowed size works
     got = b.sample_static(delta, 1e-6, 3, 4, b.STATIC_MAX_CANDIDATES)
-    assert len(set(got.cpu().tolist())) == b.STATIC_MAX_CANDIDATES
+    assert np.array_equal(got.cpu().numpy(), oracle.sample(np.ones(100_000), 1e-6, 3, 4, b.STATIC_MAX_CANDIDATES))
