@@ -35,6 +35,8 @@ struct strads_lasso_s {
   cudaStream_t capture_stream;
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
+  cudaGraph_t tail_graph;    // sampling ahead: one round from an early list, for what is left over of the sequences
+  cudaGraphExec_t tail_exec;
   cudaEvent_t fork;          // S > 1: where the schedulers' streams join the caller's stream
   // Sampling ahead (one scheduler; strads_run only): the draw of round t + 1 runs on its own stream beside the Gram
   // and walk of round t, and the round then starts from that list corrected for round t's update.
@@ -437,6 +439,8 @@ void release(strads_lasso_s* h) {
   if (h->copy_done != nullptr) cudaEventDestroy(h->copy_done);
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
   if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
+  if (h->tail_exec != nullptr) cudaGraphExecDestroy(h->tail_exec);
+  if (h->tail_graph != nullptr) cudaGraphDestroy(h->tail_graph);
   if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
   delete h;
 }
@@ -557,8 +561,8 @@ static long long graph_rounds(const strads_lasso_s* h) {
 
 // Captures the launch sequence of graph_rounds() rounds into a graph (on a private stream: the caller's may be
 // the legacy default stream, which cannot be captured; nothing executes during capture).  With several
-// schedulers the sequence starts with scheduler 0.
-static int build_round_graph(strads_lasso_s* h) {
+// schedulers the sequence starts with scheduler 0.  `tail`: one round from an early list instead (sampling ahead).
+static int build_round_graph(strads_lasso_s* h, bool tail = false) {
   if (h->capture_stream == nullptr) {
     int prio_least = 0, prio_greatest = 0;
     CK(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
@@ -574,18 +578,22 @@ static int build_round_graph(strads_lasso_s* h) {
     if (h->n_sched > 1) {
       rc = pipelined_rounds(h, graph_rounds(h), h->capture_stream);
     } else if (h->ahead_ok) {
-      for (long long i = 0; i < graph_rounds(h) && rc == STRADS_OK; ++i) rc = round_sampling_ahead(h, true, h->capture_stream);
+      const long long n = tail ? 1 : graph_rounds(h);
+      for (long long i = 0; i < n && rc == STRADS_OK; ++i) rc = round_sampling_ahead(h, true, h->capture_stream);
     } else {
       rc = one_round(h, nullptr);
     }
-    e = cudaStreamEndCapture(h->capture_stream, &h->round_graph);
+    e = cudaStreamEndCapture(h->capture_stream, tail ? &h->tail_graph : &h->round_graph);
     h->ahead_round = ahead_before;
   }
   h->stream = user;
   h->round_host = round_before;
   if (rc) return rc;
   if (e != cudaSuccess) return cuda_fail(e, "stream capture of a round");
-  CK(cudaGraphInstantiate(&h->round_exec, h->round_graph, 0));
+  // instantiated and uploaded now, so that the first launch does not pay for either
+  cudaGraphExec_t* exec = tail ? &h->tail_exec : &h->round_exec;
+  CK(cudaGraphInstantiate(exec, tail ? h->tail_graph : h->round_graph, 0));
+  CK(cudaGraphUpload(*exec, user));
   return STRADS_OK;
 }
 
@@ -619,6 +627,10 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
     const int rc = build_round_graph(h);
     if (rc) return rc;
   }
+  if (use_graph && h->ahead_ok && h->tail_exec == nullptr) {
+    const int rc = build_round_graph(h, true);
+    if (rc) return rc;
+  }
   const long long R = graph_rounds(h);
   for (int64_t i = 0; i < n_rounds; ++i) {
     if (use_graph && h->ahead_ok) {
@@ -628,8 +640,12 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
         h->round_host += R;
         h->ahead_round = h->round_host;
         i += R - 1;
-      } else {                                         // first round of a run (draw now, start drawing ahead), last few
-        const int rc = round_sampling_ahead(h, have_list, h->stream);
+      } else if (have_list) {                          // fewer rounds left than a sequence holds: one at a time
+        CK(cudaGraphLaunch(h->tail_exec, h->stream));
+        h->round_host += 1;
+        h->ahead_round = h->round_host;
+      } else {                                         // first round of a run: draw now, start drawing ahead
+        const int rc = round_sampling_ahead(h, false, h->stream);
         if (rc) return rc;
       }
     } else if (use_graph) {
@@ -756,6 +772,8 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
 static void drop_round_graph(strads_lasso_s* h) {
   if (h->round_exec != nullptr) { cudaGraphExecDestroy(h->round_exec); h->round_exec = nullptr; }
   if (h->round_graph != nullptr) { cudaGraphDestroy(h->round_graph); h->round_graph = nullptr; }
+  if (h->tail_exec != nullptr) { cudaGraphExecDestroy(h->tail_exec); h->tail_exec = nullptr; }
+  if (h->tail_graph != nullptr) { cudaGraphDestroy(h->tail_graph); h->tail_graph = nullptr; }
 }
 
 int strads_set_wait_limit(strads_handle_t h, uint32_t iterations) {
