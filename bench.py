@@ -192,12 +192,13 @@ def aggregate(units_local: float, ms_local: float, dist_ok: bool, device):
 
 def window_of(p: wl.LassoProblem) -> int:
     """The library's rule for the leading window of candidates whose Gram is formed first."""
-    w = (p.n_keep + p.n_keep // 2 + 128 + 127) // 128 * 128
+    slack = max(p.n_keep // 4, 64) if p.layout == wl.DENSE else p.n_keep // 2 + 128
+    w = (p.n_keep + slack + 127) // 128 * 128
     return w if 2 * w <= p.n_candidates else p.n_candidates
 
 
 def rooflines(p: wl.LassoProblem, workload: str, step_ms: dict, kept_per_round: float, examined_per_round: float,
-              ms_per_step: float, peaks: dict) -> dict:
+              moving_per_round: float, ms_per_step: float, peaks: dict) -> dict:
     """Roofline of the dominant kernel plus the streaming kernels against the measured HBM bandwidth."""
     window = window_of(p)
     out = {}
@@ -214,7 +215,8 @@ def rooflines(p: wl.LassoProblem, workload: str, step_ms: dict, kept_per_round: 
             "launch_ms": step_ms["gram_ms"], "algorithmic_flops_per_launch": flops,
             "peak_source": f"{peaks['source']} BF16 burst (the screen's operands are BF16; pairs it cannot call are decided "
                            "exactly in FP64); the kernel is timed alone between events"}
-        upd_bytes = 4.0 * p.n_rows * kept_per_round + 8.0 * p.n_rows + 16.0 * kept_per_round
+        # the update reads the columns of the kept coefficients that move (a null change needs no column) and r twice
+        upd_bytes = 4.0 * p.n_rows * moving_per_round + 8.0 * p.n_rows + 16.0 * kept_per_round
         pack_bytes = 6.0 * p.n_rows * window              # FP32 columns read, BF16 copies written
         ns_bytes = 4.0 * p.n_rows * (p.n_candidates + kept_per_round) + 8.0 * p.n_rows
         moved_bytes = 4.0 * p.n_rows * window + 8.0 * p.n_rows
@@ -317,6 +319,7 @@ def measure(workload: str, args, device, rank: int, world: int, dist_ok: bool, p
     n_timed = REPEATS * args.steps
     kept_per_round = (tot1["kept"] - tot0["kept"]) / n_timed
     examined_per_round = (tot1["examined"] - tot0["examined"]) / n_timed
+    moving_per_round = (tot1["nonzero"] - tot0["nonzero"]) / n_timed
     # per-step device times: the next rounds of the same run, launched kernel by kernel with events between the steps
     prof_rounds = min(max(args.steps, 100), 500)
     s.profile_begin(prof_rounds)
@@ -332,7 +335,7 @@ def measure(workload: str, args, device, rank: int, world: int, dist_ok: bool, p
         "ms_per_step_repeats": [m / args.steps for m in region_ms],
         "config": config_of(p, workload + (f" with J={args.n_cols}" if args.n_cols else ""), world),
         "rounds_per_s": world * args.steps / (ms * 1e-3), "kept_per_round": kept_per_round,
-        "examined_per_round": examined_per_round, "objective": objective, "status_bits": status_bits,
+        "examined_per_round": examined_per_round, "moving_per_round": moving_per_round, "objective": objective, "status_bits": status_bits,
         "step_ms": step_ms, "step_ms_rounds": prof["rounds"],
         "step_ms_note": "device time per step over the rounds right after the timed regions, launched kernel by kernel "
                         "with CUDA events between steps and a plain draw; the timed regions replay captured launch "
@@ -340,7 +343,8 @@ def measure(workload: str, args, device, rank: int, world: int, dist_ok: bool, p
         "sampling_ahead": p.layout == wl.DENSE and p.n_keep <= 4096,
         "clocks": clk,
     }
-    rec.update(rooflines(p, workload, step_ms, kept_per_round, examined_per_round, ms_local / args.steps, peaks))
+    rec.update(rooflines(p, workload, step_ms, kept_per_round, examined_per_round, moving_per_round, ms_local / args.steps,
+                         peaks))
 
     # ---- the same workload with S round-robin scheduler threads (blocks of later rounds prepared during updates) ----
     if with_round_robin and args.schedulers > 1 and p.n_candidates * args.schedulers <= p.n_cols:

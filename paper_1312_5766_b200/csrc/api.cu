@@ -83,10 +83,10 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xcb, off_partial, off_walk_blocked, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl,
       off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
-  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, partial_tiles, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
+  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
   long long ldc, ldcb;
 };
 
@@ -144,8 +144,6 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.ldc = (c->n_rows + 3) / 4 * 4;
   L.ldcb = (c->n_rows + 7) / 8 * 8;
   L.off_xcb = take(c->layout == STRADS_DENSE_COLMAJOR ? sizeof(unsigned short) * (size_t)c->n_candidates * L.ldcb : 0);
-  L.partial_tiles = c->layout == STRADS_DENSE_COLMAJOR ? 160 : 0;     // split-K partial tiles of a window Gram (10 MB)
-  L.off_partial = take(sizeof(float) * 128 * 128 * (size_t)L.partial_tiles);
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
@@ -188,9 +186,13 @@ bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) &
 
 // Conflict bits of all candidate pairs.  Dense: tensor-core kernel unless the FP32 Gram itself is wanted
 // (debug output) or the SIMT kernel is asked for.
-cudaError_t launch_gram(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, float* gram_dbg,
-                        bool only_if_short, bool window = false, cudaEvent_t after_pack = nullptr) {
+// n_total: length of the whole list (n_cand < n_total: a window).  *walked: the Gram kernel's last CTA also settles the
+// walk (dense tensor-core window), so that the walk kernel behind it only runs if that CTA leaves it the job.
+cudaError_t launch_gram(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, int n_total, float* gram_dbg,
+                        bool only_if_short, cudaEvent_t after_pack = nullptr, bool* walked = nullptr) {
   const Problem& p = sc.p;
+  const bool window = n_cand < n_total;
+  if (walked != nullptr) *walked = false;
   if (after_pack != nullptr && (p.layout == STRADS_CSC || gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM))) {
     const cudaError_t e = cudaEventRecord(after_pack, s);          // these paths have no pack kernel
     if (e != cudaSuccess) return e;
@@ -198,7 +200,7 @@ cudaError_t launch_gram(const Scheduler& sc, cudaStream_t s, const int* cand, in
   }
   if (p.layout == STRADS_CSC) return launch_gram_csc(p, cand, n_cand, gram_dbg, only_if_short, window, s);
   if (gram_dbg != nullptr || (p.flags & STRADS_FLAG_SIMT_GRAM)) return launch_gram_dense_simt(p, cand, n_cand, gram_dbg, s);
-  return launch_gram_dense_tc(p, sc.gram_tmap, cand, n_cand, only_if_short, window, after_pack, s);
+  return launch_gram_dense_tc(p, sc.gram_tmap, cand, n_cand, n_total, only_if_short, window, after_pack, s, walked);
 }
 
 // The greedy walk stops at P kept, so it normally looks at little more than the first P candidates: form the
@@ -207,7 +209,10 @@ cudaError_t launch_gram(const Scheduler& sc, cudaStream_t s, const int* cand, in
 // Gram + walk, enqueued behind it, runs (it is a no-op otherwise).  Same kept set either way.
 int window_of(const Problem& p, int n_cand) {
   if (p.flags & (STRADS_FLAG_FULL_GRAM | STRADS_FLAG_SIMT_GRAM)) return n_cand;
-  const long long w = ((long long)p.n_keep + p.n_keep / 2 + 128 + 127) / 128 * 128;
+  // dense: every window column is streamed and multiplied, so the window is cut closer (room for one candidate in five
+  // to be rejected); CSC: the window's cost is in the pairs that share a row, and a short window costs a whole-list walk
+  const long long slack = p.layout == STRADS_DENSE_COLMAJOR ? (p.n_keep / 4 > 64 ? p.n_keep / 4 : 64) : p.n_keep / 2 + 128;
+  const long long w = ((long long)p.n_keep + slack + 127) / 128 * 128;
   return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
 }
 
@@ -225,22 +230,26 @@ int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_
     return STRADS_OK;
   }
   const int window = gram_dbg != nullptr ? n_cand : window_of(p, n_cand);
-  CK(launch_gram(sc, s, cand, window, gram_dbg, false, window < n_cand, after_pack));
+  bool walked = false;
+  CK(launch_gram(sc, s, cand, window, n_cand, gram_dbg, false, after_pack, &walked));
   if (after_gram) CK(cudaEventRecord(after_gram, s));
-  CK(launch_filter(p, cand, window, n_cand, false, p.kept, s));
+  // the whole-list retry -- and, behind a Gram kernel that walks, the walk kernel it may leave the job to -- go to a
+  // branch of their own when the caller has one, so that launches that normally return at once do not stand between the
+  // window and the update
+  cudaStream_t rs = s;
+  if (walked && window < n_cand && retry_stream != nullptr && branched != nullptr) {
+    CK(cudaEventRecord(retry_fork, s));
+    CK(cudaStreamWaitEvent(retry_stream, retry_fork, 0));
+    rs = retry_stream;
+    *branched = true;
+  }
+  CK(launch_filter(p, cand, window, n_cand, false, p.kept, rs, walked));
   if (window < n_cand) {
     if (p.layout == STRADS_CSC) {
       // whole list, conflict rows formed only for the candidates the walk keeps
       CK(launch_walk_csc(p, cand, n_cand, sc.walk_grid, true, p.kept, s));
     } else {
-      cudaStream_t rs = s;
-      if (retry_stream != nullptr && branched != nullptr) {
-        CK(cudaEventRecord(retry_fork, s));
-        CK(cudaStreamWaitEvent(retry_stream, retry_fork, 0));
-        rs = retry_stream;
-        *branched = true;
-      }
-      CK(launch_gram(sc, rs, cand, n_cand, nullptr, true));
+      CK(launch_gram(sc, rs, cand, n_cand, n_cand, nullptr, true));
       CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, rs));
     }
   }
@@ -383,8 +392,6 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.bucket_count = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
   p.bucket_items = L.pair_cap ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;
   p.pair_list = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_pairs) : nullptr;
-  p.gram_partial = reinterpret_cast<float*>(ws + L.off_partial);
-  p.partial_tiles = L.partial_tiles;
   p.part_count = S; p.part_index = s;
   p.sm_count = first ? first->sm_count : 0;
   p.round_ptr = &p.st->round; p.round_ahead = 0;

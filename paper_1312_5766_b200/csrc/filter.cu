@@ -10,13 +10,13 @@
 // The conflict rows are read from shared memory: all of them are brought in once when they fit (a
 // candidate window does), otherwise the rows of the range's unblocked members are fetched per range.
 #include "strads_internal.cuh"
+#include "walk_pairs.cuh"
 
 namespace strads {
 namespace {
 
 constexpr int kThreads = 256;
 constexpr int kRange = 64;                       // positions decided per step of the walk
-constexpr int kSparsePasses = 24;                // passes of the walk from the pair list before the bit rows take over
 constexpr size_t kResidentBytes = 200 * 1024;    // conflict rows of the whole list in shared memory up to this
 
 __host__ __device__ inline int words_of(int n_cand) { return (n_cand + 31) >> 5; }
@@ -28,17 +28,19 @@ __host__ __device__ inline int rows_offset(int n_cand) { return cand_offset(n_ca
 // is final (the walk never looks further); otherwise window_short is raised and the caller's retry over
 // the whole list (launched with only_if_short) replaces the result.
 __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __restrict__ cand, int n_cand, int n_total,
-                                                      int only_if_short, int resident, int* __restrict__ kept_out) {
+                                                      int only_if_short, int resident, int only_if_pending,
+                                                      int* __restrict__ kept_out) {
   chain_begin();
   if (only_if_short && !p.st->window_short) return;
+  if (only_if_pending && !p.st->walk_pending) return;
   if (n_cand < n_total && p.st->amb_count > (unsigned)p.cap_amb) {
     // dense window whose BF16 screen left more borderline pairs than the list holds: its bits are incomplete;
     // the whole-list retry (which has the 3xTF32 fallback) takes over
-    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->amb_count = 0; p.st->edge_count = 0; p.st->edges_off = 0; }
+    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->route = 1; p.st->amb_count = 0; p.st->edge_count = 0; p.st->edges_off = 0; }
     return;
   }
   if (p.layout == STRADS_CSC && n_cand < n_total && window_skipped(p)) {
-    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->edge_count = 0; p.st->edges_off = 0; }   // window attempt skipped: go straight to the whole-list walk
+    if (threadIdx.x == 0) { p.st->window_short = 1; p.st->route = 1; p.st->edge_count = 0; p.st->edges_off = 0; }   // window attempt skipped: go straight to the whole-list walk
     return;
   }
   extern __shared__ unsigned int sm[];
@@ -58,79 +60,19 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     for (int i = tid; i < p.n_keep; i += kThreads) kept_out[i] = i < nk ? cand[i] : -1;
     if (tid == 0) {
       p.st->counts[1] = nk; p.st->counts[2] = nk; p.st->counts[3] = 0; p.st->amb_count = 0; p.st->window_short = 0;
+      p.st->route = 0; p.st->walk_pending = 0;
       p.st->edge_count = 0; p.st->edges_off = 0;
     }
     return;
   }
 
   // ---- The walk from the list of conflicting pairs, when the Gram kernels listed all of them. ----
-  // Conflicts are few, so the first-fit rule "keep b unless an earlier kept a conflicts with it" is settled in
-  // passes over the pairs: a candidate with a kept earlier neighbour is out, one whose earlier neighbours are all
-  // decided and out is kept (a candidate without earlier neighbours at once).  The number of passes is the longest
-  // chain of such dependencies, two or three in practice; if it exceeds kSparsePasses the walk over the bit rows
-  // below takes over.  Stopping at P is a cut of the kept sequence at its P-th member: no decision depends on a
-  // later position.
   bool settled = false;
   const unsigned int n_edges = p.st->edge_count;
   if (!p.st->edges_off && n_edges <= (unsigned)p.cap_edges) {
-    unsigned char* state = reinterpret_cast<unsigned char*>(sm);          // 0 undecided, 1 kept, 2 out
-    unsigned char* hit = state + ((n_cand + 15) & ~15);                   // has a kept earlier neighbour
-    unsigned char* pend = hit + ((n_cand + 15) & ~15);                    // has an undecided earlier neighbour
-    unsigned int* e = reinterpret_cast<unsigned int*>(pend + ((n_cand + 15) & ~15));
-    for (int i = tid; i < n_cand; i += kThreads) { state[i] = 0; hit[i] = 0; pend[i] = 0; }
-    for (unsigned int k = tid; k < n_edges; k += kThreads) e[k] = __ldcg(p.edges + k);
-    __syncthreads();
-    for (int pass = 0; pass < kSparsePasses && !settled; ++pass) {
-      for (unsigned int k = tid; k < n_edges; k += kThreads) {
-        const int a = (int)(e[k] >> 16), b = (int)(e[k] & 0xffffu);
-        if (state[b] == 0) {
-          const unsigned char sa = state[a];
-          if (sa == 1) hit[b] = 1;                     // (several threads may store the same value: benign)
-          else if (sa == 0) pend[b] = 1;
-        }
-      }
-      __syncthreads();
-      int open = 0;
-      for (int i = tid; i < n_cand; i += kThreads) {
-        if (state[i] == 0) {
-          if (hit[i]) state[i] = 2;
-          else if (!pend[i]) state[i] = 1;
-          else open = 1;
-          pend[i] = 0;
-        }
-      }
-      settled = __syncthreads_or(open) == 0;
-    }
-    if (settled) {
-      // kept members in order: thread t counts its contiguous chunk, the chunks are scanned, and every thread
-      // writes its kept members at their ranks, up to P
-      __shared__ int s_scan[kThreads];
-      const int chunk = (n_cand + kThreads - 1) / kThreads;
-      const int i0 = min(tid * chunk, n_cand), i1 = min(i0 + chunk, n_cand);
-      int mine = 0;
-      for (int i = i0; i < i1; ++i) mine += state[i] == 1;
-      int incl = mine;                                 // inclusive scan: lanes by shuffle, then the warps' totals
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (lane == 31) s_scan[warp] = incl;
-      __syncthreads();
-      int before = 0, total = 0;
-#pragma unroll
-      for (int w = 0; w < kThreads / 32; ++w) { const int v = s_scan[w]; if (w < warp) before += v; total += v; }
-      int rank = before + incl - mine;
-      for (int i = i0; i < i1 && rank < p.n_keep; ++i) {
-        if (state[i] == 1) {
-          kept_out[rank] = cand[i];
-          p.kept_pos[rank] = i;
-          if (rank == p.n_keep - 1) s_examined = i + 1;          // the walk stops here
-          ++rank;
-        }
-      }
-      if (tid == 0) s_kept = min(total, p.n_keep);
-    }
+    __syncthreads();                                                      // s_kept, s_examined are set
+    settled = walk_from_pair_list<kThreads>(p, cand, n_cand, n_edges, reinterpret_cast<unsigned char*>(sm), kept_out,
+                                            &s_kept, &s_examined);
     __syncthreads();
   }
 
@@ -325,6 +267,8 @@ __global__ void __launch_bounds__(kThreads) k_filter(Problem p, const int* __res
     p.st->edge_count = 0; p.st->edges_off = 0;         // the next Gram starts a new list
     // (the whole-list retry leaves the flag as the window's walk set it: kernels of a parallel branch may still read it)
     if (!only_if_short) p.st->window_short = (nk < p.n_keep && n_cand < n_total) ? 1 : 0;
+    if (!only_if_short && !only_if_pending) p.st->route = p.st->window_short;   // (left to it by the window's Gram: stays on the retry branch)
+    p.st->walk_pending = 0;
     if (!only_if_short && n_cand < n_total) {          // a window attempt: remember how it went
       if (p.st->window_short) p.st->walk_streak = min(p.st->walk_streak + 1, 16);
       else { p.st->prefer_walk = 0; p.st->walk_streak = 0; }
@@ -350,13 +294,13 @@ cudaError_t prepare_filter(const Problem&) {
 }
 
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
-                          cudaStream_t s) {
+                          cudaStream_t s, bool only_if_pending) {
   bool resident;
   size_t smem = filter_smem_bytes(n_cand, &resident);
-  const size_t sparse = 3 * (((size_t)n_cand + 15) & ~(size_t)15) + sizeof(unsigned int) * (size_t)p.cap_edges;   // walk from the pair list
+  const size_t sparse = walk_pairs_smem(n_cand, (unsigned)p.cap_edges);                                          // walk from the pair list
   if (smem < sparse) smem = sparse;
   return launch_chained(k_filter, 1, kThreads, smem, s, p, cand, n_cand, n_total, only_if_short ? 1 : 0, resident ? 1 : 0,
-                        kept_out);
+                        only_if_pending ? 1 : 0, kept_out);
 }
 
 }  // namespace strads

@@ -28,6 +28,7 @@
 #include <cuda_bf16.h>
 
 #include "strads_internal.cuh"
+#include "walk_pairs.cuh"
 
 namespace strads {
 namespace {
@@ -283,9 +284,93 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
   }
 }
 
+// Exact decision for one pair the screen could not call, by a whole warp: FP64 dot product of the two columns of X.  Setting a bit is idempotent and order-independent, so the result is deterministic.
+__device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, int lane) {
+  const long long n4 = (p.N + 3) >> 2;
+  const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
+  const float4* xa = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[a] * p.ld);
+  const float4* xb = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[b] * p.ld);
+  double acc = 0.0;
+  for (long long g = lane; g < n4; g += 32) {
+    const float4 u = xa[g], w = xb[g];
+    const long long i = g << 2;
+    acc += (double)u.x * w.x;
+    if (i + 1 < p.N) acc += (double)u.y * w.y;
+    if (i + 2 < p.N) acc += (double)u.z * w.z;
+    if (i + 3 < p.N) acc += (double)u.w * w.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  if (lane == 0) {
+    const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
+    if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
+      atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
+      list_conflict(p, a, b);
+    }
+  }
+}
+
+// What follows the window's Gram on the round's path, done by the CTA of the Gram kernel that finishes last
+// instead of by launches of their own:
+//   - the pairs the screen left open, normally a handful or none, are decided exactly.  "Few" is a budget of
+//     multiply-adds for this one CTA (2^21, some tens of microseconds at worst): short columns leave many pairs
+//     open (their correlations scatter widely around rho) but each is cheap, long columns hardly any.  Beyond the
+//     budget the window is handed to the whole-list retry, whose Gram has a recheck kernel of its own;
+//   - the greedy first-fit walk is settled from the list of conflicting pairs; if that list is incomplete or the
+//     chains of dependent decisions are too long, the walk kernel behind this one does it from the bit rows
+//     (walk_pending), otherwise that kernel returns at once.
+// DeviceState::route tells the update which of its two gated copies runs: 0 the one behind this kernel, 1 the one
+// at the end of the branch that holds the walk kernel and the whole-list retry.
+constexpr unsigned int kInlineRecheck = 4096;
+constexpr long long kInlineRecheckWork = 1ll << 21;
+__device__ void window_tail(const Problem& p, const int* __restrict__ cand, int n_cand, int n_total, unsigned char* sm) {
+  __shared__ int s_last, s_kept, s_examined;
+  DeviceState* st = p.st;
+  const int tid = threadIdx.x;
+  __threadfence();
+  __syncthreads();
+  if (tid == 0) s_last = atomicAdd(&st->gram_ticket, 1u) == gridDim.x - 1u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const unsigned int n_amb = __ldcg(&st->amb_count);
+  if (n_amb > (unsigned)p.cap_amb || n_amb > kInlineRecheck || (long long)n_amb * p.N > kInlineRecheckWork) {
+    if (tid == 0) {                                      // the whole-list retry takes over (it has the 3xTF32 fallback)
+      st->gram_ticket = 0u; st->window_short = 1; st->route = 1; st->walk_pending = 0;
+      st->amb_count = 0; st->edge_count = 0; st->edges_off = 0;
+    }
+    return;
+  }
+  for (unsigned int e = tid >> 5; e < n_amb; e += blockDim.x >> 5) recheck_pair(p, __ldcg(p.amb_pairs + e), tid & 31);
+  if (tid == 0) { s_kept = 0; s_examined = n_cand; }
+  __syncthreads();
+  const unsigned int n_edges = __ldcg(&st->edge_count);
+  bool settled = false;
+  if (!st->edges_off && n_edges <= (unsigned)p.cap_edges && walk_pairs_smem(n_cand, n_edges) <= kRingBytes)
+    settled = walk_from_pair_list<kThreads>(p, cand, n_cand, n_edges, sm, p.kept, &s_kept, &s_examined);
+  if (!settled) {
+    if (tid == 0) { st->gram_ticket = 0u; st->walk_pending = 1; st->route = 1; }
+    return;
+  }
+  const int nk = s_kept;
+  for (int i = nk + tid; i < p.n_keep; i += blockDim.x) p.kept[i] = -1;
+  if (tid == 0) {
+    st->gram_ticket = 0u;
+    st->counts[1] = s_examined; st->counts[2] = nk; st->counts[3] = 0; st->amb_count = 0;
+    st->edge_count = 0; st->edges_off = 0;               // the next Gram starts a new list
+    const int short_ = (nk < p.n_keep && n_cand < n_total) ? 1 : 0;
+    st->window_short = short_; st->route = short_; st->walk_pending = 0;
+  }
+}
+
+// n_split > 1: the launch is made of thread-block clusters of n_split CTAs that share one output tile, each taking
+// a slice of K (a window of few tiles would otherwise use few SMs); the partial tiles are combined through
+// distributed shared memory, in split order.  tail: 0 none; 1 the CTA of the grid that finishes last rechecks the
+// pairs the screen left open and settles the greedy walk from the list of conflicting pairs (window_tail).
 template <bool k3x>
 __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const __grid_constant__ CUtensorMap tmap,
-                                                                int n_cand, int n_tiles, int n_split, int only_if_short) {
+                                                                int n_cand, int n_total, int n_tiles, int n_split, int only_if_short,
+                                                                int tail) {
   chain_begin();
   // A stage holds kSub sub-blocks of 32 floats of K for A, the same for B [3xTF32: plus the two lo tiles].
   constexpr int kSub = k3x ? 1 : 2;
@@ -308,8 +393,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitLimit;
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && blockIdx.x == 0 && tid == 0)
     atomicOr(&p.st->status, STRADS_STATUS_GRAM_FALLBACK);
-  // With n_split > 1 the K range of a tile is shared by n_split CTAs, each leaving an FP32 partial tile that
-  // k_gram_reduce sums in split order (a window of few tiles would otherwise use few SMs).
+  // With n_split > 1 the K range of a tile is shared by the n_split CTAs of a cluster (consecutive block indices).
   const int tile = blockIdx.x / n_split, split = blockIdx.x - tile * n_split;
   int ti = 0, rem = tile;                              // linear index -> (ti, tj), ti <= tj
   while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
@@ -469,164 +553,115 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   }
 
   // ------------------------------ epilogue (warps 0..3: TMEM lanes 32 w .. 32 w + 31) ------------------------------
-  if (warp < kProducerWarps) {
-    if (n_split == 1) {                                // (screen: while the main loop runs) the norms of the tile
-      const int ga = ti * kTile + tid, gb = tj * kTile + tid;
-      normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
-      normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
-      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps see all of them
+  if (warp < kProducerWarps) {                           // (screen: while the main loop runs) the norms of the tile
+    const int ga = ti * kTile + tid, gb = tj * kTile + tid;
+    normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
+    normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
+    asm volatile("bar.sync 1, 128;" ::: "memory");       // the four epilogue warps see all of them
+  }
+  const double rho = (double)p.rho;
+  const double band = screen_band(N);
+  if (n_split == 1) {
+    if (warp < kProducerWarps) {
+      bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      if (ok) {
+        const int la = warp * 32 + lane;
+        const int a = ti * kTile + la;
+        const double norm_a = normA[la];
+#pragma unroll 1
+        for (int c = 0; c < kTile / 32; ++c) {
+          uint32_t v[32];
+          tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
+          const uint32_t word = decide_word<!k3x>(p, v, a, tj * kTile + c * 32, n_cand, norm_a, normB + c * 32, rho, band);
+          const int widx = tj * (kTile / 32) + c;
+          if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     }
-    bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
-    ok = __all_sync(0xffffffffu, ok);
-    if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (ok) {
+  } else {
+    // Split K inside a cluster.  Every CTA parks its partial tile in its own shared memory (the ring is drained:
+    // all stages this CTA asked for have been consumed), row r as 32 groups of four columns, group q at slot
+    // q ^ (r & 31) so that neither the row-per-thread stores nor the row-per-warp loads meet bank conflicts.
+    float* park = reinterpret_cast<float*>(tiles_ptr);
+    if (warp < kProducerWarps) {
+      bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int la = warp * 32 + lane;
-      const int a = ti * kTile + la;
-      const double norm_a = normA[la];
-      const double rho = (double)p.rho;
-      const double band = screen_band(N);
 #pragma unroll 1
       for (int c = 0; c < kTile / 32; ++c) {
         uint32_t v[32];
-        if (n_st > 0) {
+        if (ok && n_st > 0) {
           tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
-        } else {                                       // a split with no K of its own contributes zero
+        } else {                                         // a split with no K of its own (or one that gave up) adds zero
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = 0u;
         }
-        if (n_split > 1) {
-          uint4* dst = reinterpret_cast<uint4*>(p.gram_partial + (((size_t)tile * n_split + split) * kTile + la) * kTile + c * 32);
 #pragma unroll
-          for (int j = 0; j < 8; ++j) dst[j] = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-          continue;
+        for (int j = 0; j < 8; ++j) {
+          const int q = c * 8 + j;
+          *reinterpret_cast<uint4*>(park + la * kTile + ((q ^ (la & 31)) << 2)) = make_uint4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
         }
-        const uint32_t word = decide_word<!k3x>(p, v, a, tj * kTile + c * 32, n_cand, norm_a, normB + c * 32, rho, band);
-        const int widx = tj * (kTile / 32) + c;
-        if (a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    }
+    // every CTA of the cluster gets here, whatever happened above: the barriers are never left short of an arrival
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+    if (warp < kProducerWarps) {
+      // this CTA combines and thresholds its share of the tile's rows: a warp per row, a lane per four columns
+      const int row_lo = split * kTile / n_split, row_hi = (split + 1) * kTile / n_split;
+      const uint32_t park0 = smem_u32(park);
+      for (int la = row_lo + warp; la < row_hi; la += kProducerWarps) {
+        const uint32_t local = park0 + (uint32_t)(la * kTile + ((lane ^ (la & 31)) << 2)) * 4u;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int sp = 0; sp < n_split; ++sp) {             // in split order
+          uint32_t remote;
+          asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(sp));
+          float4 u;
+          asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(u.x), "=f"(u.y), "=f"(u.z), "=f"(u.w) : "r"(remote) : "memory");
+          acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
+        }
+        const int a = ti * kTile + la;
+        const double norm_a = normA[la];
+        const float g4[4] = {acc.x, acc.y, acc.z, acc.w};
+        unsigned int nib = 0u;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int b = tj * kTile + lane * 4 + k;
+          const double den = norm_a * normB[lane * 4 + k];
+          const double g = fabs((double)g4[k]);
+          const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
+          bool hit = live && g >= rho * den;
+          if (live && b > a && fabs(g - rho * den) <= band * den) {
+            hit = false;                                   // too close to call: decided exactly by the recheck
+            const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
+            if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
+          }
+          if (hit && b > a) list_conflict(p, a, b);
+          nib |= (unsigned int)hit << k;
+        }
+        unsigned int word = nib << ((lane & 7) * 4);       // 8 lanes make one 32-column mask word
+        word |= __shfl_xor_sync(0xffffffffu, word, 1);
+        word |= __shfl_xor_sync(0xffffffffu, word, 2);
+        word |= __shfl_xor_sync(0xffffffffu, word, 4);
+        const int widx = tj * (kTile / 32) + (lane >> 3);
+        if ((lane & 7) == 0 && a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
       }
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    // nobody leaves (and gives up its shared memory) while a neighbour may still be reading it
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
   }
   __syncthreads();
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
-}
-
-// Exact decision for one pair the screen could not call, by a whole warp: FP64 dot product of the two columns of X.  Setting a bit is idempotent and order-independent, so the result is deterministic.
-__device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, int lane) {
-  const long long n4 = (p.N + 3) >> 2;
-  const int a = (int)(pr >> 16), b = (int)(pr & 0xffffu);
-  const float4* xa = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[a] * p.ld);
-  const float4* xb = reinterpret_cast<const float4*>(p.xv + (long long)p.cand_cur[b] * p.ld);
-  double acc = 0.0;
-  for (long long g = lane; g < n4; g += 32) {
-    const float4 u = xa[g], w = xb[g];
-    const long long i = g << 2;
-    acc += (double)u.x * w.x;
-    if (i + 1 < p.N) acc += (double)u.y * w.y;
-    if (i + 2 < p.N) acc += (double)u.z * w.z;
-    if (i + 3 < p.N) acc += (double)u.w * w.w;
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-  if (lane == 0) {
-    const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
-    if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
-      atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
-      list_conflict(p, a, b);
-    }
-  }
-}
-
-// The pairs the screen of a candidate window left open, by the CTA of the split-K reduce kernel that finishes last
-// (few pairs, normally none: this saves a launch on the round's path).  More than kInlineRecheck of them: the
-// window is handed to the whole-list retry, whose Gram has a recheck kernel of its own, by the overflow rule.
-// "Few" is a budget of multiply-adds for this one CTA (2^21, some tens of microseconds at worst): short columns
-// leave many pairs open (their correlations scatter widely around rho) but each is cheap, long columns hardly any.
-constexpr unsigned int kInlineRecheck = 4096;
-constexpr long long kInlineRecheckWork = 1ll << 21;
-__device__ void recheck_by_last_cta(const Problem& p, unsigned int n_ctas) {
-  __shared__ int s_last;
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) s_last = atomicAdd(&p.st->gram_ticket, 1u) == n_ctas - 1u;
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const unsigned int n = __ldcg(&p.st->amb_count);
-  if (n > kInlineRecheck || (long long)n * p.N > kInlineRecheckWork) {
-    if (threadIdx.x == 0 && n <= (unsigned)p.cap_amb) p.st->amb_count = (unsigned)p.cap_amb + 1u;   // "overflow"
-  } else {
-    const int lane = threadIdx.x & 31;
-    for (unsigned int e = threadIdx.x >> 5; e < n; e += blockDim.x >> 5) recheck_pair(p, __ldcg(p.amb_pairs + e), lane);
-  }
-  if (threadIdx.x == 0) p.st->gram_ticket = 0u;
-}
-
-// Split-K: sums the partial tiles of one output tile in split order and thresholds (screen rules).
-// One CTA per (tile, 8 rows); a warp owns one row, a lane four of its 128 columns.
-__global__ void __launch_bounds__(256) k_gram_reduce(Problem p, int n_cand, int n_tiles, int n_split, int only_if_short,
-                                                     int recheck_here) {
-  chain_begin();
-  if (only_if_short && !p.st->window_short) return;
-  const int tile = blockIdx.x >> 4, rgroup = blockIdx.x & 15;
-  int ti = 0, rem = tile;
-  while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
-  const int tj = ti + rem;
-  const int lane = threadIdx.x & 31;
-  const int la = rgroup * 8 + (threadIdx.x >> 5);
-  const int a = ti * kTile + la;
-  const float4* src = reinterpret_cast<const float4*>(p.gram_partial + ((size_t)tile * n_split * kTile + la) * kTile) + lane;
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  int s = 0;
-  for (; s + 8 <= n_split; s += 8) {                   // eight loads in flight, added in split order
-    float4 u[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) u[k] = __ldcg(src + (size_t)(s + k) * (kTile * kTile / 4));
-#pragma unroll
-    for (int k = 0; k < 8; ++k) { acc.x += u[k].x; acc.y += u[k].y; acc.z += u[k].z; acc.w += u[k].w; }
-  }
-  for (; s + 4 <= n_split; s += 4) {
-    float4 u[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) u[k] = __ldcg(src + (size_t)(s + k) * (kTile * kTile / 4));
-#pragma unroll
-    for (int k = 0; k < 4; ++k) { acc.x += u[k].x; acc.y += u[k].y; acc.z += u[k].z; acc.w += u[k].w; }
-  }
-  for (; s < n_split; ++s) {
-    const float4 u = __ldcg(src + (size_t)s * (kTile * kTile / 4));
-    acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
-  }
-  const double norm_a = a < n_cand ? sqrt(p.n2[p.cand_cur[a]]) : 0.0;
-  const double rho = (double)p.rho, band = screen_band(p.N);
-  const float g4[4] = {acc.x, acc.y, acc.z, acc.w};
-  unsigned int nib = 0u;
-#pragma unroll
-  for (int k = 0; k < 4; ++k) {
-    const int b = tj * kTile + lane * 4 + k;
-    const double norm_b = b < n_cand ? sqrt(p.n2[p.cand_cur[b]]) : 0.0;
-    const double den = norm_a * norm_b;
-    const double g = fabs((double)g4[k]);
-    const bool live = a < n_cand && b < n_cand && a != b && den > 0.0;
-    bool hit = live && g >= rho * den;
-    if (live && b > a && fabs(g - rho * den) <= band * den) {
-      hit = false;                                     // too close to call: k_gram_recheck decides
-      const unsigned int slot = atomicAdd(&p.st->amb_count, 1u);
-      if (slot < (unsigned)p.cap_amb) p.amb_pairs[slot] = ((unsigned int)a << 16) | (unsigned int)b;
-    }
-    if (hit && b > a) list_conflict(p, a, b);
-    nib |= (unsigned int)hit << k;
-  }
-  unsigned int word = nib << ((lane & 7) * 4);         // 8 lanes make one 32-column mask word
-  word |= __shfl_xor_sync(0xffffffffu, word, 1);
-  word |= __shfl_xor_sync(0xffffffffu, word, 2);
-  word |= __shfl_xor_sync(0xffffffffu, word, 4);
-  const int widx = tj * (kTile / 32) + (lane >> 3);
-  if ((lane & 7) == 0 && a < n_cand && widx < p.mask_words) p.conflict[(long long)a * p.mask_words + widx] = word;
-  if (recheck_here) recheck_by_last_cta(p, gridDim.x);
+  if (tail) window_tail(p, p.cand_cur, n_cand, n_total, tiles_ptr);
 }
 
 // All pairs the screen left open: one warp per pair.
@@ -643,10 +678,32 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_sho
 
 }  // namespace
 
+// Clusters of up to kMaxSplit CTAs share a tile; how many clusters of each size the device can hold at once
+// (one CTA per SM: the ring takes nearly all of its shared memory) decides the split of a launch.
+constexpr int kMaxSplit = 16;
+static int g_max_clusters[kMaxSplit + 1];     // [size]; 0: size not available
+
 cudaError_t prepare_gram_dense_tc() {
   cudaError_t e = cudaFuncSetAttribute(k_gram_dense_tc<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+  e = cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
+  if (e != cudaSuccess) return e;
+  const bool beyond8 = cudaFuncSetAttribute(k_gram_dense_tc<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+  cudaGetLastError();
+  for (int size = 2; size <= kMaxSplit; ++size) {
+    g_max_clusters[size] = 0;
+    if (size > 8 && !beyond8) continue;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)size; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)size * 64); cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = kDynSmem;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    int n = 0;
+    if (cudaOccupancyMaxActiveClusters(&n, k_gram_dense_tc<false>, &cfg) == cudaSuccess) g_max_clusters[size] = n;
+    cudaGetLastError();                                  // (a size the device refuses is simply not used)
+  }
+  return cudaSuccess;
 }
 
 // Tensor map over the BF16 copy of the packed candidates: [n_cand rows][N elements], row pitch ldcb, box 64 x 128, 128-byte
@@ -672,23 +729,24 @@ cudaError_t encode_gram_tensor_map(const Problem& p, void* out) {
   return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
-// pack -> screen [-> split-K reduce] -> exact recheck of the borderline pairs -> (only if their list overflowed)
-// 3xTF32 over everything
-// `fallback_elsewhere`: the launch covers a window and a whole-list retry follows; an overflow of the borderline
-// list is then handled by that retry (the window's walk raises window_short), not by a 3xTF32 launch here.
-cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
-                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s) {
+// pack -> screen (K split inside clusters when the tiles are few) -> exact recheck of the borderline pairs -> (only
+// if their list overflowed) 3xTF32 over everything.
+// `fallback_elsewhere`: the launch covers a window (n_cand of n_total candidates) and a whole-list retry follows; an
+// overflow of the borderline list is then handled by that retry, not by a 3xTF32 launch here, and the last CTA of
+// the screen rechecks and walks (*walked = true: the caller's walk kernel need only run if walk_pending is raised).
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, int n_total, bool only_if_short,
+                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s, bool* walked) {
+  if (walked != nullptr) *walked = false;
   const int n_tiles = (n_cand + kTile - 1) / kTile;
   const int tiles = n_tiles * (n_tiles + 1) / 2;
   const int ois = only_if_short ? 1 : 0;
-  // few tiles (a candidate window): share each tile's K range among CTAs so that all SMs work
+  // few tiles (a candidate window): share each tile's K range among the CTAs of a cluster so that all SMs work; the
+  // largest cluster size of which the device holds `tiles` at once (one wave), and at least two stages of K each
   int n_split = 1;
   if (tiles * 2 <= p.sm_count) {
     const int n_st = (int)((p.N + 2 * kScreenK - 1) / (2 * kScreenK));
-    n_split = p.sm_count / tiles;
-    if (n_split > n_st) n_split = n_st;
-    if (n_split > p.partial_tiles / tiles) n_split = p.partial_tiles / tiles;
-    if (n_split < 1) n_split = 1;
+    for (int size = kMaxSplit; size >= 2; --size)
+      if (g_max_clusters[size] >= tiles && size * 2 <= n_st) { n_split = size; break; }
   }
   Problem q = p;
   q.cand_cur = cand;
@@ -697,18 +755,15 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   if ((e = launch_chained(k_pack_candidates, n_cand, kPackThreads, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
   if (after_pack != nullptr && (e = cudaEventRecord(after_pack, s)) != cudaSuccess) return e;   // optional step timing
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
-    if ((e = launch_chained(k_gram_dense_tc<false>, tiles * n_split, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, n_split,
-                            ois)) != cudaSuccess)
+    const int tail = (fallback_elsewhere && !only_if_short) ? 1 : 0;
+    if ((e = launch_chained_cluster(k_gram_dense_tc<false>, tiles * n_split, kThreads, kDynSmem, s, n_split, q, tm, n_cand, n_total,
+                                    n_tiles, n_split, ois, tail)) != cudaSuccess)
       return e;
-    // a window with split K and a retry behind it: the reduce kernel's last CTA rechecks, no launch of its own
-    const int recheck_here = (n_split > 1 && fallback_elsewhere) ? 1 : 0;
-    if (n_split > 1 &&
-        (e = launch_chained(k_gram_reduce, tiles * 16, 256, 0, s, q, n_cand, n_tiles, n_split, ois, recheck_here)) != cudaSuccess)
-      return e;
-    if (!recheck_here && (e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
+    if (tail && walked != nullptr) *walked = true;
+    if (!tail && (e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
   }
   if (!fallback_elsewhere || (p.flags & STRADS_FLAG_GRAM_3XTF32))
-    return launch_chained(k_gram_dense_tc<true>, tiles, kThreads, kDynSmem, s, q, tm, n_cand, n_tiles, 1, ois);
+    return launch_chained(k_gram_dense_tc<true>, tiles, kThreads, kDynSmem, s, q, tm, n_cand, n_total, n_tiles, 1, ois, 0);
   return cudaSuccess;
 }
 

@@ -43,10 +43,11 @@ struct DeviceState {
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int surv_count;      // sampler: keys the guided first pass found below its cutoff and saved (append cursor)
   int surv_valid;               // ... they are all there (no overflow, no repeat): the collect pass reads them, not delta[J]
-  unsigned int gram_ticket;     // dense Gram: CTAs of the split-K reduce kernel that are done (the last one rechecks)
+  unsigned int gram_ticket;     // dense window Gram: CTAs that are done (the last one rechecks and walks)
+  int walk_pending;             // ... that CTA could not settle the walk from the pair list: the walk kernel behind it does
+  int route;                    // ... which gated copy of the update runs: 0 the one behind the window, 1 the retry branch's
   unsigned int edge_count;      // conflicting pairs listed by the Gram kernels of this round (may exceed the list)
   int edges_off;                // a kernel that sets bits without listing pairs has run: the list is not complete
-  unsigned int pad;
 };
 
 struct WalkControl {            // shared by the CTAs of the cooperative on-demand walk (CSC)
@@ -103,8 +104,6 @@ struct Problem {
   double* cand_dbeta64;         // [n_cand] proposed change of candidate position a
   float* cand_bnew;             // [n_cand] proposed new beta
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
-  float* gram_partial;          // dense: split-K partial tiles [tile][split][128][128]
-  int partial_tiles;            // capacity of gram_partial in 128 x 128 tiles
   unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words], OR-ed into by the whole grid
   WalkControl* walk_ctl;
   long long* resid_acc;         // CSC: [N] fixed-point accumulators of the residual update (zero between rounds)
@@ -361,6 +360,21 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
   return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// The same for a kernel whose CTAs form thread-block clusters of cluster_x consecutive blocks (1: no clusters).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained_cluster(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, int cluster_x,
+                                   Args&&... args) {
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = (unsigned)cluster_x; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cfg.attrs = attr; cfg.numAttrs = cluster_x > 1 ? 2 : 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 // ---------------------------------------------------------------------------------------------
 // Launchers (one per step; all enqueue on `s` and return a cudaError_t).
 // ---------------------------------------------------------------------------------------------
@@ -378,8 +392,8 @@ cudaError_t prepare_gram_dense_tc();
 cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
 // `only_if_short`: the launch is the whole-list retry of a windowed round and does nothing unless the
 // window's filter set DeviceState::window_short.
-cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, bool only_if_short,
-                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s);
+cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* cand, int n_cand, int n_total, bool only_if_short,
+                                 bool fallback_elsewhere, cudaEvent_t after_pack, cudaStream_t s, bool* walked);
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
                             bool window, cudaStream_t s);
 cudaError_t prepare_filter(const Problem& p);
@@ -388,8 +402,10 @@ cudaError_t prepare_filter(const Problem& p);
 cudaError_t prepare_walk_csc(const Problem& p, int* grid_out);
 cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int grid, bool only_if_short, int* kept_out,
                             cudaStream_t s);
+// only_if_pending: the launch follows a window Gram whose last CTA walks; it does nothing unless that CTA left the
+// walk to it (DeviceState::walk_pending).
 cudaError_t launch_filter(const Problem& p, const int* cand, int n_cand, int n_total, bool only_if_short, int* kept_out,
-                          cudaStream_t s);
+                          cudaStream_t s, bool only_if_pending = false);
 cudaError_t launch_update(const Problem& p, const int* kept, int advance, bool after_pack, cudaStream_t s, int gate = 0);
 cudaError_t launch_set_counts(const Problem& p, int n_cand, int n_examined, int n_kept, cudaStream_t s);
 cudaError_t launch_export(const Problem& p, const int* kept, int* kept_out, float* dbeta_out, int* counts_out,

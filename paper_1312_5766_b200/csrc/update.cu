@@ -112,35 +112,74 @@ __global__ void __launch_bounds__(kThreads) k_dot_dense(Problem p, const int* __
 
 // r <- r - sum_a x_a dbeta_a with every row owned by one CTA: 32 rows per CTA, a quarter-warp per column
 // (8 lanes x float4 = one 128-byte line), so a warp reads four columns per instruction and the 32 quarter-warps
-// of the CTA take the kept columns round-robin, eight loads in flight each.  The kept columns' addresses and
-// changes are staged in shared memory first, so the column loads depend on nothing.  The per-row sums of the
-// quarter-warps are added in a fixed order.
+// of the CTA take the columns round-robin, eight loads in flight each: many small CTAs with shallow loops, which
+// measured as fast as streaming the same columns whole (16.4 us for c3's 41 MB from a cold cache; 128- to 512-row
+// blocks with a warp per column segment and the columns split into groups ran 1.4 to 6 times slower).
+// Only the kept columns whose change is not zero are read (a coefficient that stays where it is moves nothing):
+// their addresses and changes are compacted into shared memory first, in list order, so the column loads depend
+// on nothing.  The per-row sums of the quarter-warps are added in a fixed order.
 // proposals = 1: the changes were formed by the pack kernel for every candidate (cand_dbeta64 / cand_bnew by
-// position in the list, src.index = positions of the kept ones); this kernel then also does the bookkeeping of
+// position in the list, p.kept_pos = positions of the kept ones); this kernel then also does the bookkeeping of
 // the kept coefficients (beta, delta, dbeta), spread over its CTAs.  No other thread reads beta or delta here.
 constexpr int kRowsPerCta = 32;
 constexpr int kColSlots = kThreads / 8;    // quarter-warps per CTA
-constexpr int kStageCols = 2048;           // kept columns staged per pass (24 KB of shared memory)
+constexpr int kStageCols = 2048;           // moving columns staged per pass (32 KB of shared memory)
 
-// gate: 0 always; 1 only if the candidate window sufficed; 2 only if it did not (the update is then enqueued
-// twice, behind the window's walk and behind the whole-list retry on a branch of its own, and exactly one runs).
+// gate: 0 always; 1 only if the window's Gram kernel settled the walk and P were kept inside the window
+// (DeviceState::route == 0); 2 only otherwise (the update is then enqueued twice, behind the window's Gram and at the
+// end of the branch that holds the walk kernel and the whole-list retry, and exactly one runs).
 __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* __restrict__ kept, ColumnSource src,
                                                           int advance, int proposals, int gate) {
   chain_begin();
-  if (gate != 0 && (p.st->window_short != 0) != (gate == 2)) return;
+  if (gate != 0 && (p.st->route != 0) != (gate == 2)) return;
   __shared__ double part[kColSlots][kRowsPerCta];
   __shared__ double s_d[kStageCols];
   __shared__ long long s_off[kStageCols];
+  __shared__ int s_scan[kThreads / 32];
   const int n_kept = p.st->counts[2];
-  const int slot = threadIdx.x >> 3, l8 = threadIdx.x & 7;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int slot = tid >> 3, l8 = tid & 7;
   const long long i = (long long)blockIdx.x * kRowsPerCta + l8 * 4;
+
+  // ranks of the kept entries whose change is not zero: thread t owns the entries [t c, (t + 1) c)
+  const int per_thread = (n_kept + kThreads - 1) / kThreads;
+  const int a_lo = min(tid * per_thread, n_kept), a_hi = min(a_lo + per_thread, n_kept);
+  auto change_of = [&](int a) { return proposals ? p.cand_dbeta64[p.kept_pos[a]] : p.dbeta64[a]; };
+  double d_first[4] = {0.0, 0.0, 0.0, 0.0};               // the first four stay in registers (all of them up to P = 1,024)
+  int mine = 0;
+#pragma unroll
+  for (int k = 0; k < 4; ++k)
+    if (a_lo + k < a_hi) { d_first[k] = change_of(a_lo + k); mine += d_first[k] != 0.0; }
+  for (int a = a_lo + 4; a < a_hi; ++a) mine += change_of(a) != 0.0;
+  int incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_scan[warp] = incl;
+  __syncthreads();
+  int before = 0, n_moving = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) { const int v = s_scan[w]; if (w < warp) before += v; n_moving += v; }
+  const int rank0 = before + incl - mine;                 // rank of this thread's first moving entry
+
   double s0 = 0.0, s1 = 0.0, s2 = 0.0, s3 = 0.0;
-  for (int base = 0; base < n_kept; base += kStageCols) {
-    const int n_here = min(kStageCols, n_kept - base);
+  for (int base = 0; base < n_moving; base += kStageCols) {
+    const int n_here = min(kStageCols, n_moving - base);
     if (base > 0) __syncthreads();
-    for (int a = threadIdx.x; a < n_here; a += kThreads) {
-      s_off[a] = (long long)src.index[base + a] * src.pitch;
-      s_d[a] = proposals ? p.cand_dbeta64[p.kept_pos[base + a]] : p.dbeta64[base + a];
+    {
+      int rank = rank0;
+      auto place = [&](int a, double d) {
+        if (d != 0.0) {
+          if (rank >= base && rank < base + n_here) { s_d[rank - base] = d; s_off[rank - base] = (long long)src.index[a] * src.pitch; }
+          ++rank;
+        }
+      };
+#pragma unroll
+      for (int k = 0; k < 4; ++k)
+        if (a_lo + k < a_hi) place(a_lo + k, d_first[k]);
+      for (int a = a_lo + 4; a < a_hi; ++a) place(a, change_of(a));
     }
     __syncthreads();
     if (i < p.N) {
@@ -155,10 +194,8 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
         }
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-          if (d[u] != 0.0) {
-            s0 += (double)xv[u].x * d[u]; s1 += (double)xv[u].y * d[u];
-            s2 += (double)xv[u].z * d[u]; s3 += (double)xv[u].w * d[u];
-          }
+          s0 += (double)xv[u].x * d[u]; s1 += (double)xv[u].y * d[u];
+          s2 += (double)xv[u].z * d[u]; s3 += (double)xv[u].w * d[u];
         }
       }
     }
@@ -166,18 +203,19 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
   part[slot][l8 * 4 + 0] = s0; part[slot][l8 * 4 + 1] = s1;
   part[slot][l8 * 4 + 2] = s2; part[slot][l8 * 4 + 3] = s3;
   __syncthreads();
-  if (threadIdx.x < kRowsPerCta) {
-    const long long r = (long long)blockIdx.x * kRowsPerCta + threadIdx.x;
+  if (tid < kRowsPerCta) {
+    const long long r = (long long)blockIdx.x * kRowsPerCta + tid;
     if (r < p.N) {
       double s = 0.0;
 #pragma unroll
-      for (int w = 0; w < kColSlots; ++w) s += part[w][threadIdx.x];
+      for (int w = 0; w < kColSlots; ++w) s += part[w][tid];
       if (s != 0.0) p.resid[r] = (float)((double)p.resid[r] - s);
     }
   }
   DeviceState* st = p.st;
+  const int cta = blockIdx.x, n_ctas = gridDim.x;
   if (proposals) {
-    for (int a = blockIdx.x * kThreads + threadIdx.x; a < p.n_keep; a += gridDim.x * kThreads) {
+    for (int a = cta * kThreads + tid; a < p.n_keep; a += n_ctas * kThreads) {
       if (a >= n_kept) { p.dbeta[a] = 0.f; continue; }
       const int pos = p.kept_pos[a], j = kept[a];
       const double d = p.cand_dbeta64[pos];
@@ -197,7 +235,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
       if (!isfinite(d)) atomicOr(&st->status, STRADS_STATUS_NONFINITE);
     }
   }
-  if (blockIdx.x == 0 && threadIdx.x == 0 && advance) {
+  if (cta == 0 && tid == 0 && advance) {
     st->totals[0] += 1; st->totals[1] += st->counts[1]; st->totals[2] += st->counts[2];
     if (!proposals) st->totals[3] += st->counts[3];
     st->round += (unsigned long long)p.part_count;       // this scheduler's next turn
