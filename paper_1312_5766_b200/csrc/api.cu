@@ -49,6 +49,9 @@ struct strads_lasso_s {
   // window's walk and the update
   cudaStream_t retry_stream;
   cudaEvent_t retry_fork, retry_done;
+  // ... and the correction of the next round's early list, beside the update
+  cudaStream_t patch_stream;
+  cudaEvent_t patch_fork, patch_done;
   // strads_round_host: beta and the residual travel on a stream of their own while the draw (which reads only the
   // priorities) already runs
   cudaStream_t copy_stream;
@@ -289,33 +292,77 @@ int one_round(strads_lasso_s* h, const strads_round_out_t* out, cudaEvent_t befo
   return STRADS_OK;
 }
 
-// One round of strads_run with one scheduler, sampling ahead.  `main`: candidates (from the early list if there
-// is one for this round, else a draw made now), Gram, walk, update; `ahead_stream`: the early draw of the next
-// round, which reads delta and so lies between this round's candidates and its update.
+// What follows a window whose Gram kernel could not finish the job (its last CTA left the walk to the walk kernel,
+// or fewer than P were kept inside the window): the walk kernel on the window if asked for, the whole-list Gram and
+// walk if the window was short, then the gated copies of the correction of the early list and of the update.
+int retry_sequence(strads_lasso_s* h, const Scheduler& sc, int window, bool early_patch, cudaStream_t rs) {
+  const Problem& p = sc.p;
+  CK(launch_filter(p, p.cand, window, p.n_cand, false, p.kept, rs, true));
+  CK(launch_gram(sc, rs, p.cand, p.n_cand, p.n_cand, nullptr, true));
+  CK(launch_filter(p, p.cand, p.n_cand, p.n_cand, true, p.kept, rs));
+  if (early_patch) CK(launch_sample_patch(p, h->ahead, p.cand, rs, true, 2));
+  CK(launch_update(p, p.kept, 1, true, rs, 2));
+  return STRADS_OK;
+}
+
+// One round of strads_run with one scheduler, sampling ahead.  `main`: candidates, Gram (whose last CTA walks), update;
+// `ahead_stream`: the early draw of the next round, which reads delta and so lies between this round's candidates
+// and its update.
+// Where the pack kernel forms the keys of every candidate (dense tensor-core rounds), the early list of round t + 1 is
+// corrected as soon as round t's kept list stands, on `patch_stream` beside round t's update, and have_list says that
+// the candidates of this round are already in place.  Otherwise the correction opens round t + 1 (it needs the keys
+// the update leaves) and have_list says that the early list is there.
+// The retry of a window that did not suffice is a branch of its own (`retry_stream`) that ends in its own copies of
+// the correction and the update, gated on DeviceState::route like the copies on `main`, so that exactly one of each
+// runs.  (Tried and dropped: the branch as the body of a CUDA-graph IF node whose condition the window Gram's last CTA
+// sets -- c2 44.0 -> 42.4 us per round, c3 unchanged: evaluating the node costs about what the launches that return at
+// once do.)
 int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
   const Scheduler& sc = h->sch[0];
   const Problem& p = sc.p;
-  if (have_list) CK(launch_sample_patch(p, h->ahead, p.cand, main));
-  else CK(launch_sample(p, p.cand, main));
+  const bool early_patch = update_after_pack(p, false) && p.proposals;     // (also: the gated update is the single-kernel one)
+  if (!have_list) CK(launch_sample(p, p.cand, main));
+  else if (!early_patch) CK(launch_sample_patch(p, h->ahead, p.cand, main));
   CK(cudaEventRecord(h->ahead_fork, main));
   CK(cudaStreamWaitEvent(h->ahead_stream, h->ahead_fork, 0));
   CK(launch_sample(h->ahead, h->ahead.cand, h->ahead_stream));
   CK(cudaEventRecord(h->ahead_done, h->ahead_stream));
-  const bool can_branch = update_after_pack(p, false) && p.proposals;     // (the gated update is the single-kernel one)
-  bool branched = false;
-  const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr, nullptr, nullptr, can_branch ? h->retry_stream : nullptr,
-                                 h->retry_fork, &branched);
-  if (rc) return rc;
-  CK(cudaStreamWaitEvent(main, h->ahead_done, 0));
-  if (branched) {
-    CK(launch_update(p, p.kept, 1, true, main, 1));                          // runs if the window sufficed
-    CK(cudaStreamWaitEvent(h->retry_stream, h->ahead_done, 0));
-    CK(launch_update(p, p.kept, 1, true, h->retry_stream, 2));               // runs behind the retry otherwise
-    CK(cudaEventRecord(h->retry_done, h->retry_stream));
-    CK(cudaStreamWaitEvent(main, h->retry_done, 0));
-  } else {
+  const int window = window_of(p, p.n_cand);
+  if (!early_patch || window >= p.n_cand || (p.flags & STRADS_FLAG_GRAM_3XTF32)) {
+    // no window, or a Gram that does not walk: everything in a row
+    const int rc = gram_and_filter(sc, main, p.cand, p.n_cand, nullptr);
+    if (rc) return rc;
+    CK(cudaStreamWaitEvent(main, h->ahead_done, 0));
+    if (early_patch) {
+      CK(cudaEventRecord(h->patch_fork, main));
+      CK(cudaStreamWaitEvent(h->patch_stream, h->patch_fork, 0));
+      CK(launch_sample_patch(p, h->ahead, p.cand, h->patch_stream, true, 0));
+      CK(cudaEventRecord(h->patch_done, h->patch_stream));
+    }
     CK(launch_update(p, p.kept, 1, update_after_pack(p, false), main));
+    if (early_patch) CK(cudaStreamWaitEvent(main, h->patch_done, 0));
+    h->round_host += 1;
+    h->ahead_round = h->round_host;
+    return STRADS_OK;
   }
+  bool walked = false;
+  CK(launch_gram(sc, main, p.cand, window, p.n_cand, nullptr, false, nullptr, &walked));
+  if (!walked) return STRADS_ERR_INVALID_ARG;            // (early_patch implies the tensor-core screen, whose last CTA walks)
+  CK(cudaStreamWaitEvent(main, h->ahead_done, 0));         // the draw is over: delta may change, and the early list stands
+  CK(cudaEventRecord(h->retry_fork, main));
+  CK(cudaStreamWaitEvent(h->retry_stream, h->retry_fork, 0));
+  {
+    const int rc = retry_sequence(h, sc, window, early_patch, h->retry_stream);
+    if (rc) return rc;
+  }
+  CK(cudaEventRecord(h->retry_done, h->retry_stream));
+  CK(cudaEventRecord(h->patch_fork, main));
+  CK(cudaStreamWaitEvent(h->patch_stream, h->patch_fork, 0));
+  CK(launch_sample_patch(p, h->ahead, p.cand, h->patch_stream, true, 1));
+  CK(cudaEventRecord(h->patch_done, h->patch_stream));
+  CK(launch_update(p, p.kept, 1, true, main, 1));                            // runs if the window sufficed
+  CK(cudaStreamWaitEvent(main, h->patch_done, 0));
+  CK(cudaStreamWaitEvent(main, h->retry_done, 0));
   h->round_host += 1;
   h->ahead_round = h->round_host;
   return STRADS_OK;
@@ -441,6 +488,9 @@ void release(strads_lasso_s* h) {
   if (h->retry_stream != nullptr) cudaStreamDestroy(h->retry_stream);
   if (h->retry_fork != nullptr) cudaEventDestroy(h->retry_fork);
   if (h->retry_done != nullptr) cudaEventDestroy(h->retry_done);
+  if (h->patch_stream != nullptr) cudaStreamDestroy(h->patch_stream);
+  if (h->patch_fork != nullptr) cudaEventDestroy(h->patch_fork);
+  if (h->patch_done != nullptr) cudaEventDestroy(h->patch_done);
   if (h->copy_stream != nullptr) cudaStreamDestroy(h->copy_stream);
   if (h->copy_fork != nullptr) cudaEventDestroy(h->copy_fork);
   if (h->copy_done != nullptr) cudaEventDestroy(h->copy_done);
@@ -524,7 +574,10 @@ int strads_lasso_init(const strads_lasso_config_t* c, strads_handle_t* out_handl
         (e = cudaEventCreateWithFlags(&h->ahead_done, cudaEventDisableTiming)) != cudaSuccess ||
         (e = cudaStreamCreateWithPriority(&h->retry_stream, cudaStreamNonBlocking, prio_least)) != cudaSuccess ||
         (e = cudaEventCreateWithFlags(&h->retry_fork, cudaEventDisableTiming)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&h->retry_done, cudaEventDisableTiming)) != cudaSuccess)
+        (e = cudaEventCreateWithFlags(&h->retry_done, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaStreamCreateWithPriority(&h->patch_stream, cudaStreamNonBlocking, prio_greatest)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->patch_fork, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&h->patch_done, cudaEventDisableTiming)) != cudaSuccess)
       return fail(cuda_fail(e, "sampling-ahead stream"));
   }
   for (int s = 0; s < S; ++s) {

@@ -349,7 +349,9 @@ __device__ void window_tail(const Problem& p, const int* __restrict__ cand, int 
   if (!st->edges_off && n_edges <= (unsigned)p.cap_edges && walk_pairs_smem(n_cand, n_edges) <= kRingBytes)
     settled = walk_from_pair_list<kThreads>(p, cand, n_cand, n_edges, sm, p.kept, &s_kept, &s_examined);
   if (!settled) {
-    if (tid == 0) { st->gram_ticket = 0u; st->walk_pending = 1; st->route = 1; }
+    if (tid == 0) {
+      st->gram_ticket = 0u; st->walk_pending = 1; st->route = 1;
+    }
     return;
   }
   const int nk = s_kept;

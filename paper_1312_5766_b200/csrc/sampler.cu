@@ -551,16 +551,26 @@ __global__ void __launch_bounds__(256) k_sample_rank_bins(Problem p, int* cand_o
 // instead of i.  (An old key below an element of L is itself on L, L being a prefix of the full ranking; a new key
 // beyond the end of a list shorter than J ranks >= P' and is left out.)  The <= P old and new keys were left by the
 // update (patch_keys); every CTA holds them in shared memory and counts against them by brute force.
+// from_cand: the keys are taken from those the pack kernel formed for every candidate (by position in the list), so
+// that the correction can run beside the update of the same round instead of behind it.  gate: as for the update
+// (0 always; 1 / 2: only the copy on the branch that DeviceState::route names).
 __global__ void __launch_bounds__(256) k_sample_patch(Problem p, const unsigned long long* __restrict__ list, int n_list,
-                                                      int* __restrict__ cand_out) {
+                                                      int* __restrict__ cand_out, int from_cand, int gate) {
   chain_begin();
+  if (gate != 0 && (p.st->route != 0) != (gate == 2)) return;
   extern __shared__ unsigned long long s_keys[];       // [n_keep] old keys, then [n_keep] new keys
-  const int nk = p.st->counts[2];                      // coefficients the last update touched
+  const int nk = p.st->counts[2];                      // coefficients the update of this round touches
   unsigned long long* old_k = s_keys;
   unsigned long long* new_k = s_keys + p.n_keep;
-  for (int a = threadIdx.x; a < nk; a += 256) {        // (left by the update, which knew both priorities)
-    old_k[a] = p.patch_keys[a];
-    new_k[a] = p.patch_keys[p.n_keep + a];
+  for (int a = threadIdx.x; a < nk; a += 256) {
+    if (from_cand) {
+      const int pos = p.kept_pos[a];
+      old_k[a] = p.cand_keys[pos];
+      new_k[a] = p.cand_keys[p.n_cand + pos];
+    } else {                                           // left by the update, which knew both priorities
+      old_k[a] = p.patch_keys[a];
+      new_k[a] = p.patch_keys[p.n_keep + a];
+    }
   }
   __syncthreads();
   if (blockIdx.x == 0 && threadIdx.x == 0) p.st->counts[0] = p.n_cand;
@@ -613,10 +623,11 @@ cudaError_t prepare_sample(const Problem&) {
   return cudaFuncSetAttribute(k_sample_patch, cudaFuncAttributeMaxDynamicSharedMemorySize, 2 * 8 * 4096);
 }
 
-cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s) {
+cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s, bool from_cand,
+                                int gate) {
   const int ctas = (ahead.n_cand + 31) / 32 + (p.n_keep + 7) / 8;        // list elements by eight threads, new keys by warp
   return launch_chained(k_sample_patch, ctas, 256, 2 * sizeof(unsigned long long) * (size_t)p.n_keep, s, p,
-                        (const unsigned long long*)ahead.keys_out, ahead.n_cand, cand_out);
+                        (const unsigned long long*)ahead.keys_out, ahead.n_cand, cand_out, from_cand ? 1 : 0, gate);
 }
 
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {

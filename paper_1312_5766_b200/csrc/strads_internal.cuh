@@ -386,7 +386,10 @@ cudaError_t prepare_sample(const Problem& p);
 cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s);
 // Candidates of the round at hand from a draw made one round ahead (`ahead`: its keys in rank order, ahead.n_cand of
 // them) and the coefficients the last update changed (p.kept, p.delta_prev, p.delta).
-cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s);
+// from_cand: before this round's update, from the keys the pack kernel formed for every candidate (p.kept_pos, p.cand_keys);
+// gate: 0 always, 1 / 2 only on the branch DeviceState::route names (as launch_update).
+cudaError_t launch_sample_patch(const Problem& p, const Problem& ahead, int* cand_out, cudaStream_t s, bool from_cand = false,
+                                int gate = 0);
 cudaError_t launch_gram_dense_simt(const Problem& p, const int* cand, int n_cand, float* gram_dbg, cudaStream_t s);
 cudaError_t prepare_gram_dense_tc();
 cudaError_t encode_gram_tensor_map(const Problem& p, void* out_128_bytes);
