@@ -59,6 +59,8 @@ def _load():
             lib.so_unit_exponential_f32.argtypes = [C.c_uint32]
             lib.so_race_key.restype = C.c_float
             lib.so_race_key.argtypes = [C.c_float, C.c_float, C.c_uint32]
+            lib.so_race_key_mode.restype = C.c_float
+            lib.so_race_key_mode.argtypes = [C.c_float, C.c_float, C.c_uint32, C.c_int32]
             lib.so_draw_word.restype = C.c_uint32
             lib.so_draw_word.argtypes = [C.c_uint64, C.c_uint64, C.c_uint64]
             lib.so_corr.restype = C.c_double
@@ -127,11 +129,26 @@ def race_key(delta_j, eta, x):
     return float(_load().so_race_key(float(delta_j), float(eta), int(x) & 0xFFFFFFFF))
 
 
-def sample(delta, eta, seed, t, n_cand, return_keys=False):
+WEIGHT_MODES = {"square": 0, "abs": 1, "uniform": 2}     # p(j) ~ delta^2 + eta | |delta| + eta | 1
+FILTER_MODES = {"rho": 0, "none": 1, "dynamic": 2}        # Algorithm 1's test | first P candidates | dormant coefficients do not couple
+
+
+def race_key_mode(delta_j, eta, x, weight):
+    return float(_load().so_race_key_mode(float(delta_j), float(eta), int(x) & 0xFFFFFFFF, WEIGHT_MODES[weight]))
+
+
+def sample(delta, eta, seed, t, n_cand, return_keys=False, weight="square"):
     lib = _load()
     delta = _f64(delta)
     J = delta.shape[0]
     cand = np.empty(n_cand, dtype=np.int32)
+    if weight != "square":
+        assert not return_keys
+        rc = lib.so_sample_mode(C.c_int64(J), _p(delta), C.c_double(eta), C.c_uint64(seed), C.c_uint64(t),
+                                C.c_int32(n_cand), C.c_int32(WEIGHT_MODES[weight]), _p(cand))
+        if rc:
+            raise ValueError(f"so_sample_mode failed: {rc}")
+        return cand
     keys = np.empty(J, dtype=np.float32) if return_keys else None
     rc = lib.so_sample(C.c_int64(J), _p(delta), C.c_double(eta), C.c_uint64(seed), C.c_uint64(t),
                        C.c_int32(n_cand), _p(cand), _p(keys))
@@ -175,6 +192,18 @@ def filter(X: Matrix, n2, cand, n_keep, rho, follow=None, tol=0.0):
     return kept[: nk.value].copy(), ne.value, mm.value
 
 
+def filter_dynamic(X: Matrix, n2, cand, n_keep, rho, beta, delta):
+    """The filter with dependencies dropped at run time (a coefficient that is zero and whose last update left it
+    there couples with nobody).  Returns (kept, n_examined)."""
+    n2, beta, delta = _f64(n2), _f64(beta), _f64(delta)
+    cand = np.ascontiguousarray(cand, dtype=np.int32)
+    kept = np.full(n_keep, -1, dtype=np.int32)
+    nk, ne = C.c_int32(0), C.c_int32(0)
+    _load().so_filter_dynamic(X.ref, _p(n2), _p(cand), C.c_int32(len(cand)), C.c_int32(n_keep), C.c_double(rho),
+                              _p(beta), _p(delta), _p(kept), C.byref(nk), C.byref(ne))
+    return kept[: nk.value].copy(), ne.value
+
+
 def update(X: Matrix, n2, lam, kept, beta, resid, delta):
     """In-place Jacobi update of the kept coefficients; returns dbeta (float64)."""
     for a in (beta, resid, delta):
@@ -198,8 +227,10 @@ def init(X: Matrix, y, c_init):
     return n2, beta, resid, delta
 
 
-def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, delta, n_sched=1):
+def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, delta, n_sched=1, weight="square",
+          filter="rho"):
     """One round in place (round t is dispatched by scheduler thread t mod n_sched).
+    weight / filter: another schedule (WEIGHT_MODES, FILTER_MODES), one scheduler thread only.
     Returns dict(cand, kept, dbeta, counts)."""
     for a in (beta, resid, delta):
         assert a.dtype == np.float64 and a.flags.c_contiguous
@@ -208,7 +239,13 @@ def round(X: Matrix, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, resid, de
     kept = np.full(n_keep, -1, dtype=np.int32)
     dbeta = np.zeros(n_keep, dtype=np.float64)
     counts = np.zeros(4, dtype=np.int32)
-    if n_sched == 1:
+    if weight != "square" or filter != "rho":
+        assert n_sched == 1
+        rc = _load().so_round_mode(X.ref, _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
+                                   C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
+                                   C.c_int32(WEIGHT_MODES[weight]), C.c_int32(FILTER_MODES[filter]),
+                                   _p(beta), _p(resid), _p(delta), _p(cand), _p(kept), _p(dbeta), _p(counts))
+    elif n_sched == 1:
         rc = _load().so_round(X.ref, _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
                               C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
                               _p(beta), _p(resid), _p(delta), _p(cand), _p(kept), _p(dbeta), _p(counts))

@@ -177,6 +177,17 @@ float so_race_key(float delta_j, float eta, uint32_t x)
     return so_unit_exponential_f32(x) / w;
 }
 
+/* Other importance distributions p(j):
+ *   mode 0  w_j = delta_j^2 + eta   (Theorem 1; so_race_key)
+ *   mode 1  w_j = |delta_j| + eta   (Algorithm 1 as printed: p(j) ~ |beta_j^(t_j-2) - beta_j^(t_j-1)| + eta)
+ *   mode 2  w_j = 1                 (uniform draw: the static and the random scheduler of the comparison, Section 5.1) */
+float so_race_key_mode(float delta_j, float eta, uint32_t x, int32_t mode)
+{
+    if (mode == 0) return so_race_key(delta_j, eta, x);
+    const float w = mode == 1 ? fabsf(delta_j) + eta : 1.0f;
+    return so_unit_exponential_f32(x) / w;
+}
+
 typedef struct { uint32_t tbits; int32_t j; } so_keyed;
 
 static int keyed_less(const void *pa, const void *pb)
@@ -199,6 +210,24 @@ int so_sample(int64_t J, const double *delta, double eta, uint64_t seed, uint64_
         all[j].tbits = f32_bits(T);
         all[j].j = (int32_t)j;
         if (keys_out) keys_out[j] = T;
+    }
+    qsort(all, (size_t)J, sizeof(so_keyed), keyed_less);
+    for (int32_t a = 0; a < n_cand; ++a) cand[a] = all[a].j;
+    free(all);
+    return 0;
+}
+
+/* The same draw under another importance distribution (so_race_key_mode). */
+int so_sample_mode(int64_t J, const double *delta, double eta, uint64_t seed, uint64_t t,
+                   int32_t n_cand, int32_t mode, int32_t *cand)
+{
+    if (J <= 0 || n_cand < 0 || n_cand > J || mode < 0 || mode > 2) return -1;
+    so_keyed *all = (so_keyed *)malloc((size_t)J * sizeof(so_keyed));
+    if (!all) return -2;
+    for (int64_t j = 0; j < J; ++j) {
+        const float T = so_race_key_mode((float)delta[j], (float)eta, so_draw_word(seed, t, (uint64_t)j), mode);
+        all[j].tbits = f32_bits(T);
+        all[j].j = (int32_t)j;
     }
     qsort(all, (size_t)J, sizeof(so_keyed), keyed_less);
     for (int32_t a = 0; a < n_cand; ++a) cand[a] = all[a].j;
@@ -280,6 +309,38 @@ int so_filter(const so_matrix *X, const double *n2, const int32_t *cand, int32_t
     return 0;
 }
 
+/* The filter with dependencies dropped at run time (SAP step 4: "removing dependencies between
+ * variables that have reached zero"; Section 1, "Dynamic Block Structures": a coefficient that stays
+ * zero does not affect the update of another, however correlated the two columns are).
+ * A coefficient is dormant when it is zero and its last update left it there (beta_j = 0 and
+ * delta_j = 0; a coefficient never updated has delta_j = C and is not dormant).  The coupling
+ * d(x_j, x_k) of a pair with a dormant member is taken as 0: a dormant candidate is always kept and
+ * blocks nobody; the rho test applies among the others exactly as in so_filter. */
+int so_filter_dynamic(const so_matrix *X, const double *n2, const int32_t *cand, int32_t n_cand,
+                      int32_t n_keep, double rho, const double *beta, const double *delta,
+                      int32_t *kept, int32_t *n_kept_out, int32_t *n_examined_out)
+{
+    int32_t nk = 0, examined = 0;
+    for (int32_t a = 0; a < n_cand && nk < n_keep; ++a) {
+        const int32_t c = cand[a];
+        ++examined;
+        int keep = 1;
+        if (!(beta[c] == 0.0 && delta[c] == 0.0)) {
+            for (int32_t b = 0; b < nk; ++b) {
+                const int32_t k = kept[b];
+                if (beta[k] == 0.0 && delta[k] == 0.0) continue;
+                const double den = sqrt(n2[c] * n2[k]);
+                const double corr = den > 0.0 ? col_dot_col(X, c, k) / den : 0.0;
+                if (fabs(corr) >= rho) { keep = 0; break; }
+            }
+        }
+        if (keep) kept[nk++] = c;
+    }
+    *n_kept_out = nk;
+    *n_examined_out = examined;
+    return 0;
+}
+
 /* Correlation of two columns as the filter sees it (exposed for tests). */
 double so_corr(const so_matrix *X, const double *n2, int64_t j, int64_t k)
 {
@@ -356,6 +417,36 @@ int so_round(const so_matrix *X, const double *n2, double lambda, double eta, do
     if (rc) return rc;
     int32_t nk = 0, ne = 0;
     so_filter(X, n2, cand, n_cand, n_keep, rho, NULL, 0, 0.0, kept, &nk, &ne, NULL);
+    so_update(X, n2, lambda, kept, nk, beta, resid, delta, dbeta);
+    int32_t nz = 0;
+    for (int32_t a = 0; a < nk; ++a) nz += dbeta[a] != 0.0;
+    counts[0] = n_cand; counts[1] = ne; counts[2] = nk; counts[3] = nz;
+    return 0;
+}
+
+/* One round under another schedule: weight_mode as so_race_key_mode; filter_mode 0 the rho test of
+ * Algorithm 1, 1 none (the first P candidates: the random scheduler, which "does not perform
+ * dependency checking"), 2 the rho test with dependencies dropped at run time (so_filter_dynamic).
+ * weight_mode 2 with filter_mode 0 is the static scheduler of Section 5.1. */
+int so_round_mode(const so_matrix *X, const double *n2, double lambda, double eta, double rho,
+                  int32_t n_cand, int32_t n_keep, uint64_t seed, uint64_t t, int32_t weight_mode, int32_t filter_mode,
+                  double *beta, double *resid, double *delta,
+                  int32_t *cand, int32_t *kept, double *dbeta, int32_t *counts)
+{
+    int rc = so_sample_mode(X->n_cols, delta, eta, seed, t, n_cand, weight_mode, cand);
+    if (rc) return rc;
+    int32_t nk = 0, ne = 0;
+    if (filter_mode == 0) {
+        so_filter(X, n2, cand, n_cand, n_keep, rho, NULL, 0, 0.0, kept, &nk, &ne, NULL);
+    } else if (filter_mode == 1) {
+        nk = n_cand < n_keep ? n_cand : n_keep;
+        for (int32_t a = 0; a < nk; ++a) kept[a] = cand[a];
+        ne = nk;
+    } else if (filter_mode == 2) {
+        so_filter_dynamic(X, n2, cand, n_cand, n_keep, rho, beta, delta, kept, &nk, &ne);
+    } else {
+        return -1;
+    }
     so_update(X, n2, lambda, kept, nk, beta, resid, delta, dbeta);
     int32_t nz = 0;
     for (int32_t a = 0; a < nk; ++a) nz += dbeta[a] != 0.0;
