@@ -71,6 +71,13 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
                                           walk (default: of a leading window of 1.5 P + 128 first,
                                           of all P' only if the walk runs out of the window)    */
 
+#define STRADS_FLAG_ABS_WEIGHT    32u   /* p(j) ~ |delta_j| + eta, Algorithm 1 as printed ("Draw a set U ..."), instead
+                                          of Theorem 1's delta_j^2 + eta                         */
+#define STRADS_FLAG_DYNAMIC_DEPS  64u   /* dependencies dropped at run time (Section 1, "Dynamic Block Structures";
+                                          SAP step 4): a coefficient that is zero and whose last update left it
+                                          there (beta_j = 0, delta_j = 0) is taken to couple with nobody -- it
+                                          passes the rho test and blocks no other candidate             */
+
 /* limits */
 #define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (positions in the candidate list are packed into 16 bits
                                            in the lists of pairs; the walk holds P' / 32 mask words per CTA) */

@@ -22,6 +22,8 @@ FLAG_NO_FILTER = 2
 FLAG_SIMT_GRAM = 4
 FLAG_GRAM_3XTF32 = 8
 FLAG_FULL_GRAM = 16
+FLAG_ABS_WEIGHT = 32
+FLAG_DYNAMIC_DEPS = 64
 MAX_CANDIDATES = 16384
 STALL_WALK_BARRIER, STALL_GRAM_LOADS = 1, 2
 

@@ -109,7 +109,7 @@ __global__ void __launch_bounds__(kThreads) k_csc_pair_bits(Problem p, const int
     const int ja = cand[a], jb = cand[b];
     const long long a0 = p.xptr[ja];
     const float dot = sparse_dot(p.xrow + a0, p.xv + a0, (int)(p.xptr[ja + 1] - a0), p, jb);
-    const double den = sqrt(p.n2[ja] * p.n2[jb]);
+    const double den = sqrt(coupling_n2(p, ja) * coupling_n2(p, jb));
     if (den > 0.0 && fabs((double)dot) >= rho * den) {
       atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
       list_conflict(p, a, b);                             // (a pair listed twice is listed twice here too: harmless)
@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
   __syncthreads();
   const int* ar = staged ? arow : p.xrow + a0;
   const float* av = staged ? aval : p.xv + a0;
-  const double n2a = p.n2[ja];
+  const double n2a = coupling_n2(p, ja);
   const double rho = (double)p.rho;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
@@ -153,7 +153,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
     if (b < n_cand && b != a) {
       const int jb = cand[b];
       const float dot = sparse_dot(ar, av, na, p, jb);
-      const double den = sqrt(n2a * p.n2[jb]);
+      const double den = sqrt(n2a * coupling_n2(p, jb));
       hit = den > 0.0 && fabs((double)dot) >= rho * den;
       if (gram_dbg != nullptr) {
         gram_dbg[(long long)a * n_cand + b] = dot;

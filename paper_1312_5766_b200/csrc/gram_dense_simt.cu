@@ -50,8 +50,8 @@ __global__ void __launch_bounds__(kThreads) k_gram_dense_simt(Problem p, const i
   const float* colA = ga < n_cand ? p.xv + (long long)cand[ga] * p.ld : nullptr;
   const float* colB = gb < n_cand ? p.xv + (long long)cand[gb] * p.ld : nullptr;
   if (tid < BM) {
-    n2a[tid] = ga < n_cand ? p.n2[cand[ga]] : 0.0;
-    n2b[tid] = gb < n_cand ? p.n2[cand[gb]] : 0.0;
+    n2a[tid] = ga < n_cand ? coupling_n2(p, cand[ga]) : 0.0;
+    n2b[tid] = gb < n_cand ? coupling_n2(p, cand[gb]) : 0.0;
     bits[tid][0] = bits[tid][1] = bits[tid][2] = bits[tid][3] = 0u;
   }
 

@@ -219,7 +219,7 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
   __shared__ float s_E;
   if (threadIdx.x == kPackStream && p.patch_keys != nullptr) {
     s_E = next_round_exponential(p, (uint32_t)j);
-    p.cand_keys[a] = race_key_from(s_E, p.delta[j], p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
+    p.cand_keys[a] = race_key_from(s_E, p.delta[j], p.eta, (uint32_t)j, weight_mode_of(p.flags));
   }
   float h0 = 0.f, l0 = 0.f, h1 = 0.f, l1 = 0.f;
   constexpr int kU = 4;                                 // column loads in flight per thread
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
     p.cand_bnew[a] = b_new;
     p.cand_dbeta64[a] = d;
     if (p.patch_keys != nullptr)
-      p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0);
+      p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, weight_mode_of(p.flags));
   }
 }
 
@@ -302,7 +302,7 @@ __device__ __forceinline__ void recheck_pair(const Problem& p, unsigned int pr, 
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
   if (lane == 0) {
-    const double den = sqrt(p.n2[p.cand_cur[a]]) * sqrt(p.n2[p.cand_cur[b]]);
+    const double den = sqrt(coupling_n2(p, p.cand_cur[a])) * sqrt(coupling_n2(p, p.cand_cur[b]));
     if (den > 0.0 && fabs(acc) >= (double)p.rho * den) {
       atomicOr(&p.conflict[(long long)a * p.mask_words + (b >> 5)], 1u << (b & 31));
       list_conflict(p, a, b);
@@ -557,8 +557,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   // ------------------------------ epilogue (warps 0..3: TMEM lanes 32 w .. 32 w + 31) ------------------------------
   if (warp < kProducerWarps) {                           // (screen: while the main loop runs) the norms of the tile
     const int ga = ti * kTile + tid, gb = tj * kTile + tid;
-    normA[tid] = ga < n_cand ? sqrt(p.n2[p.cand_cur[ga]]) : 0.0;
-    normB[tid] = gb < n_cand ? sqrt(p.n2[p.cand_cur[gb]]) : 0.0;
+    normA[tid] = ga < n_cand ? sqrt(coupling_n2(p, p.cand_cur[ga])) : 0.0;
+    normB[tid] = gb < n_cand ? sqrt(coupling_n2(p, p.cand_cur[gb])) : 0.0;
     asm volatile("bar.sync 1, 128;" ::: "memory");       // the four epilogue warps see all of them
   }
   const double rho = (double)p.rho;

@@ -34,8 +34,8 @@ constexpr int kThreads = 256;
 // a few operations instead of the whole key: T = E / w and the computed E is never below
 // v = (x + 1/2) / 2^32 (-ln(1 - v) >= v; checked against the key's arithmetic over its whole range of x), so
 // v > 1.01 cut w  implies  T > cut.  Nearly all coefficients are far above the boundary of the P' smallest.
-__device__ __forceinline__ bool key_surely_above(float cut, float d, float eta, uint32_t x, bool uniform) {
-  const float w = uniform ? 1.0f : __fmaf_rn(d, d, eta);
+__device__ __forceinline__ bool key_surely_above(float cut, float d, float eta, uint32_t x, int mode) {
+  const float w = priority_weight(d, eta, mode);
   const float v = __fmaf_rn(__uint2float_rn(x), __uint_as_float(0x2f800000u), __uint_as_float(0x2f000000u));
   return v > __fmul_rn(__fmul_rn(cut, w), 1.01f);
 }
@@ -47,13 +47,13 @@ __device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned lon
   uint32_t w[4];
   philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
   const long long j0 = g * 4;
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  const int mode = weight_mode_of(p.flags);
   if (cut > 0.f && p.part_count <= 1 && j0 + 3 < p.J) {
     const float4 d = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
-    if (!key_surely_above(cut, d.x, p.eta, w[0], uniform)) f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, uniform));
-    if (!key_surely_above(cut, d.y, p.eta, w[1], uniform)) f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, uniform));
-    if (!key_surely_above(cut, d.z, p.eta, w[2], uniform)) f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, uniform));
-    if (!key_surely_above(cut, d.w, p.eta, w[3], uniform)) f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, uniform));
+    if (!key_surely_above(cut, d.x, p.eta, w[0], mode)) f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, mode));
+    if (!key_surely_above(cut, d.y, p.eta, w[1], mode)) f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, mode));
+    if (!key_surely_above(cut, d.z, p.eta, w[2], mode)) f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, mode));
+    if (!key_surely_above(cut, d.w, p.eta, w[3], mode)) f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, mode));
     return;
   }
   if (p.part_count > 1) {                              // only the coefficients this scheduler owns take part
@@ -62,21 +62,21 @@ __device__ __forceinline__ void for_keys_of_group(const Problem& p, unsigned lon
     for (unsigned int i = 0; i < 4; ++i)
       if (j0 + i < p.J && (r0 + i) % S == (unsigned)p.part_index) {
         const float d = __ldg(p.delta + j0 + i);
-        if (cut > 0.f && key_surely_above(cut, d, p.eta, w[i], uniform)) continue;
-        f(race_key64(d, p.eta, w[i], (uint32_t)(j0 + i), uniform));
+        if (cut > 0.f && key_surely_above(cut, d, p.eta, w[i], mode)) continue;
+        f(race_key64(d, p.eta, w[i], (uint32_t)(j0 + i), mode));
       }
     return;
   }
   if (j0 + 3 < p.J) {
     const float4 d = __ldg(reinterpret_cast<const float4*>(p.delta + j0));
-    f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, uniform));
-    f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, uniform));
-    f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, uniform));
-    f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, uniform));
+    f(race_key64(d.x, p.eta, w[0], (uint32_t)j0, mode));
+    f(race_key64(d.y, p.eta, w[1], (uint32_t)j0 + 1, mode));
+    f(race_key64(d.z, p.eta, w[2], (uint32_t)j0 + 2, mode));
+    f(race_key64(d.w, p.eta, w[3], (uint32_t)j0 + 3, mode));
   } else {
 #pragma unroll
     for (int i = 0; i < 4; ++i)
-      if (j0 + i < p.J) f(race_key64(p.delta[j0 + i], p.eta, w[i], (uint32_t)(j0 + i), uniform));
+      if (j0 + i < p.J) f(race_key64(p.delta[j0 + i], p.eta, w[i], (uint32_t)(j0 + i), mode));
   }
 }
 
@@ -89,11 +89,11 @@ struct KeyQueue { uint2* slots; int n; };
 
 template <typename F>
 __device__ __forceinline__ void drain_keys(const Problem& p, KeyQueue& q, F&& f) {
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  const int mode = weight_mode_of(p.flags);
   __syncwarp();
   for (int i = (int)(threadIdx.x & 31); i < q.n; i += 32) {
     const uint2 e = q.slots[i];
-    f(race_key64(__ldg(p.delta + e.x), p.eta, e.y, e.x, uniform));
+    f(race_key64(__ldg(p.delta + e.x), p.eta, e.y, e.x, mode));
   }
   __syncwarp();
   q.n = 0;
@@ -104,7 +104,7 @@ __device__ __forceinline__ void queue_keys_of_groups(const Problem& p, unsigned 
                                                      float cut, KeyQueue& q, F&& f) {
   const int lane = threadIdx.x & 31;
   const long long g = g0 + lane;
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  const int mode = weight_mode_of(p.flags);
   uint32_t w[4] = {0u, 0u, 0u, 0u};
   float d[4] = {0.f, 0.f, 0.f, 0.f};
   const long long j0 = g * 4;
@@ -122,7 +122,7 @@ __device__ __forceinline__ void queue_keys_of_groups(const Problem& p, unsigned 
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     const bool in = g < groups && j0 + i < p.J && (S == 1u || (r0 + i) % S == (unsigned)p.part_index) &&
-                    !key_surely_above(cut, d[i], p.eta, w[i], uniform);
+                    !key_surely_above(cut, d[i], p.eta, w[i], mode);
     const unsigned int mask = __ballot_sync(0xffffffffu, in);
     if (in) q.slots[q.n + __popc(mask & ((1u << lane) - 1u))] = make_uint2((uint32_t)(j0 + i), w[i]);
     q.n += __popc(mask);

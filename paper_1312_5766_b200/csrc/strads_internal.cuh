@@ -214,14 +214,20 @@ __device__ __forceinline__ float unit_exponential_rn(uint32_t x) {
 
 // 64-bit ranking key of coefficient j: (bits of T_j) << 32 | j, T_j = E_j / (delta_j^2 + eta).
 // All keys are distinct; ascending key order = ascending T, ties to the smaller j.
-__device__ __forceinline__ unsigned long long race_key_from(float E, float delta_j, float eta, uint32_t j, bool uniform) {
-  const float w = uniform ? 1.0f : __fmaf_rn(delta_j, delta_j, eta);
-  const float T = __fdiv_rn(E, w);
+// `mode`: which importance distribution p(j) the flags ask for.
+enum WeightMode { kWeightSquare = 0, kWeightAbs = 1, kWeightUniform = 2 };   // delta^2 + eta | |delta| + eta | 1
+__host__ __device__ __forceinline__ int weight_mode_of(unsigned int flags) {
+  return (flags & STRADS_FLAG_UNIFORM_DRAW) ? kWeightUniform : ((flags & STRADS_FLAG_ABS_WEIGHT) ? kWeightAbs : kWeightSquare);
+}
+__device__ __forceinline__ float priority_weight(float delta_j, float eta, int mode) {
+  return mode == kWeightUniform ? 1.0f : (mode == kWeightAbs ? __fadd_rn(fabsf(delta_j), eta) : __fmaf_rn(delta_j, delta_j, eta));
+}
+__device__ __forceinline__ unsigned long long race_key_from(float E, float delta_j, float eta, uint32_t j, int mode) {
+  const float T = __fdiv_rn(E, priority_weight(delta_j, eta, mode));
   return ((unsigned long long)__float_as_uint(T) << 32) | j;
 }
-__device__ __forceinline__ unsigned long long race_key64(float delta_j, float eta, uint32_t word, uint32_t j,
-                                                         bool uniform) {
-  return race_key_from(unit_exponential_rn(word), delta_j, eta, j, uniform);
+__device__ __forceinline__ unsigned long long race_key64(float delta_j, float eta, uint32_t word, uint32_t j, int mode) {
+  return race_key_from(unit_exponential_rn(word), delta_j, eta, j, mode);
 }
 
 // The race keys coefficient j has in this scheduler's next round with its priority before (d_old) and after (d_new)
@@ -236,10 +242,18 @@ __device__ __forceinline__ float next_round_exponential(const Problem& p, uint32
 }
 __device__ __forceinline__ void next_round_keys(const Problem& p, uint32_t j, float d_old, float d_new,
                                                 unsigned long long* key_old, unsigned long long* key_new) {
-  const bool uniform = (p.flags & STRADS_FLAG_UNIFORM_DRAW) != 0;
+  const int mode = weight_mode_of(p.flags);
   const float E = next_round_exponential(p, j);
-  *key_old = race_key_from(E, d_old, p.eta, j, uniform);
-  *key_new = race_key_from(E, d_new, p.eta, j, uniform);
+  *key_old = race_key_from(E, d_old, p.eta, j, mode);
+  *key_new = race_key_from(E, d_new, p.eta, j, mode);
+}
+
+// ||x_j||^2 as the dependency check (SAP step 2) sees it.  With STRADS_FLAG_DYNAMIC_DEPS a coefficient that is zero
+// and whose last update left it there couples with nobody: it gets 0 here, and every Gram kernel already treats a
+// pair with a zero column as free of conflict.
+__device__ __forceinline__ double coupling_n2(const Problem& p, int j) {
+  if ((p.flags & STRADS_FLAG_DYNAMIC_DEPS) && p.beta[j] == 0.f && p.delta[j] == 0.f) return 0.0;
+  return p.n2[j];
 }
 
 // x_a^T x_b of two CSC columns (ascending rows): a given as arrays (possibly staged in shared memory), b read

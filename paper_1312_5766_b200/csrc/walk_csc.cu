@@ -144,7 +144,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
       const int j = cand[s_pos[q]];
       const long long a0 = p.xptr[j];
       const int na = (int)(p.xptr[j + 1] - a0);
-      if (lane == 0) { s_col[q] = j; s_ptr[q] = a0; s_len[q] = na; s_n2[q] = p.n2[j]; }
+      if (lane == 0) { s_col[q] = j; s_ptr[q] = a0; s_len[q] = na; s_n2[q] = coupling_n2(p, j); }
       if (na <= kColCap)
         for (int e = lane; e < na; e += 32) { brow[q][e] = __ldg(p.xrow + a0 + e); bval[q][e] = __ldg(p.xv + a0 + e); }
     }
@@ -221,7 +221,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
           const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
           const int jb = cand[b];
           const float dot = sparse_dot_prefetched<32>(ar, av, na, p, jb);
-          const double den = sqrt(s_n2[q] * p.n2[jb]);
+          const double den = sqrt(s_n2[q] * coupling_n2(p, jb));
           hit = den > 0.0 && fabs((double)dot) >= rho * den;
         }
         const unsigned int word = __ballot_sync(full, hit);
