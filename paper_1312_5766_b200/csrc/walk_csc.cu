@@ -75,8 +75,10 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
   if (p.st->status & STRADS_STATUS_WAIT_EXPIRED) return;
   const unsigned int spin_limit = p.wait_limit ? p.wait_limit : kSpinLimit;
   __shared__ unsigned int blocked[kMaxWords];
-  __shared__ int brow[kBatch][kColCap];
-  __shared__ float bval[kBatch][kColCap];
+  __shared__ int brow[kBatch][kColCap + 1];             // (odd pitch: threads that merge different members' columns
+  __shared__ float bval[kBatch][kColCap + 1];           //  read different banks)
+  __shared__ int s_pref[kMaxWords + 1];                  // unblocked candidates before each mask word (step D)
+  __shared__ int s_wsum[kThreads / 32];
   __shared__ int s_pos[kBatch], s_col[kBatch], s_len[kBatch];
   __shared__ long long s_ptr[kBatch];
   __shared__ double s_n2[kBatch];
@@ -139,14 +141,20 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
     const int m = s_m;
     if (m == 0) break;                                 // list exhausted (the same in every CTA)
 
-    // ---- B: stage the members' columns (warp w: members w, w + 8, ...), then the pairs among them ----
-    for (int q = warp; q < m; q += kThreads / 32) {
-      const int j = cand[s_pos[q]];
+    // ---- B: stage the members' columns, all at once (a thread per member finds the column, then eight threads per
+    //      member copy it: three memory round trips for the whole batch), then the pairs among them ----
+    if (tid < m) {
+      const int j = cand[s_pos[tid]];
       const long long a0 = p.xptr[j];
-      const int na = (int)(p.xptr[j + 1] - a0);
-      if (lane == 0) { s_col[q] = j; s_ptr[q] = a0; s_len[q] = na; s_n2[q] = coupling_n2(p, j); }
-      if (na <= kColCap)
-        for (int e = lane; e < na; e += 32) { brow[q][e] = __ldg(p.xrow + a0 + e); bval[q][e] = __ldg(p.xv + a0 + e); }
+      s_col[tid] = j; s_ptr[tid] = a0; s_len[tid] = (int)(p.xptr[j + 1] - a0); s_n2[tid] = coupling_n2(p, j);
+    }
+    __syncthreads();
+    {
+      const int q = tid >> 3;
+      if (q < m && s_len[q] <= kColCap) {
+        const long long a0 = s_ptr[q];
+        for (int e = tid & 7; e < s_len[q]; e += 8) { brow[q][e] = __ldg(p.xrow + a0 + e); bval[q][e] = __ldg(p.xv + a0 + e); }
+      }
     }
     __syncthreads();
     {
@@ -201,31 +209,62 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
     __syncthreads();
     if (s_done) break;                                 // P kept: what they block no longer matters
 
-    // ---- D: the kept members' conflicts with the later unblocked candidates, shared out over the grid:
-    //      task (kept member k, mask word w) -> one warp, a lane per candidate of the word ----
+    // ---- D: the kept members' conflicts with the later candidates that are not blocked yet, shared out over the
+    //      grid with a lane per (candidate, kept member) pair.  Every CTA numbers the unblocked candidates behind the
+    //      first kept member from its own copy of the mask (the same in all CTAs), so that pair number L of the grid is
+    //      member L / U against the (L mod U)-th of them: late batches, in which a dozen members meet a few hundred
+    //      survivors, still use every lane.  A lane fetches its candidate's rows and values together and merges them
+    //      against the member's column in shared memory. ----
     {
       const unsigned int keep = s_keep;
       const int n_new = __popc(keep);
-      const long long tasks = (long long)n_new * W;
-      const long long n_warps = (long long)n_ctas * (kThreads / 32);
-      for (long long t = (long long)blockIdx.x * (kThreads / 32) + warp; t < tasks; t += n_warps) {
-        const int k = (int)(t / W), w = (int)(t - (long long)k * W);
+      const int first_pos = s_pos[__ffs(keep) - 1];      // candidates at or before the first kept member are not touched
+      auto free_word = [&](int w) {                      // unblocked candidates of mask word w behind first_pos
+        unsigned int f = ~blocked[w];
+        const int first = w << 5;
+        if (first + 31 <= first_pos) f = 0u;
+        else if (first <= first_pos) f &= full << (first_pos - first + 1);     // (a shift of 1 .. 31)
+        if (first + 32 > n_cand) f &= first >= n_cand ? 0u : (full >> (first + 32 - n_cand));
+        return f;
+      };
+      // exclusive prefix of the per-word counts: two words per thread (W <= 512), warp scan, then the warps' totals
+      int c0 = 0, c1 = 0;
+      if (2 * tid < W) c0 = __popc(free_word(2 * tid));
+      if (2 * tid + 1 < W) c1 = __popc(free_word(2 * tid + 1));
+      int incl = c0 + c1;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(full, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (lane == 31) s_wsum[warp] = incl;
+      __syncthreads();
+      int before = 0, U = 0;
+#pragma unroll
+      for (int k = 0; k < kThreads / 32; ++k) { const int v = s_wsum[k]; if (k < warp) before += v; U += v; }
+      const int excl = before + incl - c0 - c1;
+      if (2 * tid < W) s_pref[2 * tid] = excl;
+      if (2 * tid + 1 < W) s_pref[2 * tid + 1] = excl + c0;
+      if (tid == 0) s_pref[W] = U;
+      __syncthreads();
+      const long long pairs = (long long)U * n_new;
+      const long long n_lanes = (long long)n_ctas * kThreads;
+      for (long long L = (long long)blockIdx.x * kThreads + tid; L < pairs; L += n_lanes) {
+        const int k = (int)(L / U), u = (int)(L - (long long)k * U);
+        int lo = 0, hi = W;                              // the word that holds the u-th unblocked candidate
+        while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_pref[mid] <= u) lo = mid; else hi = mid; }
+        const int b = (lo << 5) + nth_set_bit(free_word(lo), u - s_pref[lo]);
         const int q = nth_set_bit(keep, k);
-        const int a = s_pos[q];
-        if (w < (a >> 5)) continue;
-        const int b = w * 32 + lane;
-        bool hit = false;
-        if (b < n_cand && b > a && !((blocked[w] >> lane) & 1u)) {
-          const int na = s_len[q];
-          const int* ar = na <= kColCap ? brow[q] : p.xrow + s_ptr[q];
-          const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
-          const int jb = cand[b];
-          const float dot = sparse_dot_prefetched<32>(ar, av, na, p, jb);
-          const double den = sqrt(s_n2[q] * coupling_n2(p, jb));
-          hit = den > 0.0 && fabs((double)dot) >= rho * den;
-        }
-        const unsigned int word = __ballot_sync(full, hit);
-        if (lane == 0 && word != 0u) atomicOr(&blocked_g[w], word);
+        if (s_pos[q] >= b) continue;                     // the member comes later in the list: it cannot block b
+        const int jb = cand[b];
+        const long long q0 = p.xptr[jb];
+        const int nb = (int)(p.xptr[jb + 1] - q0);
+        const double den = sqrt(s_n2[q] * coupling_n2(p, jb));
+        const int na = s_len[q];
+        const int* ar = na <= kColCap ? brow[q] : p.xrow + s_ptr[q];
+        const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
+        const float dot = sparse_dot_fetched<32>(ar, av, na, p, q0, nb);
+        if (den > 0.0 && fabs((double)dot) >= rho * den) atomicOr(&blocked_g[b >> 5], 1u << (b & 31));
       }
     }
     ok = grid_barrier(c, n_ctas, &p.st->status, spin_limit);
