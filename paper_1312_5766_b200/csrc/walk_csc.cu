@@ -161,17 +161,52 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
       const int qa = tid >> 3;                         // eight threads per member qa: partners qb = tid % 8 + 8 k
       if (qa < m) {
         const int na = s_len[qa];
-        const int* ar = na <= kColCap ? brow[qa] : p.xrow + s_ptr[qa];
-        const float* av = na <= kColCap ? bval[qa] : p.xv + s_ptr[qa];
         unsigned int hits = 0u;
-        for (int qb = (tid & 7); qb < m; qb += 8) {
-          if (qb <= qa) continue;
-          const int nb = s_len[qb];
-          const int* br = nb <= kColCap ? brow[qb] : p.xrow + s_ptr[qb];
-          const float* bv = nb <= kColCap ? bval[qb] : p.xv + s_ptr[qb];
-          const float dot = sparse_dot_arrays(ar, av, na, br, bv, nb);
-          const double den = sqrt(s_n2[qa] * s_n2[qb]);
-          if (den > 0.0 && fabs((double)dot) >= rho * den) hits |= 1u << qb;
+        // the (up to four) merges of this thread run side by side, one step of each per trip: the steps of one merge
+        // depend on each other (load, compare, advance), those of different merges do not
+        int qbs[4], nbs[4], ii[4], kk[4];
+        float dots[4];
+        bool staged = na <= kColCap;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int qb = (tid & 7) + 8 * u;
+          const bool on = qb < m && qb > qa;
+          qbs[u] = on ? qb : qa;
+          nbs[u] = on ? s_len[qb] : 0;
+          staged = staged && nbs[u] <= kColCap;
+          ii[u] = 0; kk[u] = 0; dots[u] = 0.f;
+        }
+        if (staged) {
+          bool any = true;
+          while (any) {
+            any = false;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+              const bool on = ii[u] < na && kk[u] < nbs[u];
+              const int i = on ? ii[u] : 0, k = on ? kk[u] : 0;
+              const int ra = brow[qa][i], rb = brow[qbs[u]][k];
+              const float pa = bval[qa][i], pb = bval[qbs[u]][k];
+              dots[u] = (on && ra == rb) ? fmaf(pa, pb, dots[u]) : dots[u];
+              ii[u] += (on && ra <= rb) ? 1 : 0;
+              kk[u] += (on && rb <= ra) ? 1 : 0;
+              any = any || on;
+            }
+          }
+        } else {                                       // a column too long for its slot: plain merges from global memory
+          const int* ar = na <= kColCap ? brow[qa] : p.xrow + s_ptr[qa];
+          const float* av = na <= kColCap ? bval[qa] : p.xv + s_ptr[qa];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int qb = qbs[u], nb = nbs[u];
+            const int* br = nb <= kColCap ? brow[qb] : p.xrow + s_ptr[qb];
+            const float* bv = nb <= kColCap ? bval[qb] : p.xv + s_ptr[qb];
+            dots[u] = sparse_dot_arrays(ar, av, na, br, bv, nb);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const double den = sqrt(s_n2[qa] * s_n2[qbs[u]]);
+          if (nbs[u] > 0 && den > 0.0 && fabs((double)dots[u]) >= rho * den) hits |= 1u << qbs[u];
         }
         if (hits) atomicOr(&s_conf[qa], hits);
       }
@@ -249,7 +284,9 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
       __syncthreads();
       const long long pairs = (long long)U * n_new;
       const long long n_lanes = (long long)n_ctas * kThreads;
-      for (long long L = (long long)blockIdx.x * kThreads + tid; L < pairs; L += n_lanes) {
+      // (warp g of the grid = warp g / n_ctas of CTA g mod n_ctas: a few hundred pairs spread over all SMs instead of
+      //  filling the first few CTAs)
+      for (long long L = ((long long)warp * n_ctas + blockIdx.x) * 32 + lane; L < pairs; L += n_lanes) {
         const int k = (int)(L / U), u = (int)(L - (long long)k * U);
         int lo = 0, hi = W;                              // the word that holds the u-th unblocked candidate
         while (hi - lo > 1) { const int mid = (lo + hi) >> 1; if (s_pref[mid] <= u) lo = mid; else hi = mid; }
@@ -263,7 +300,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
         const int na = s_len[q];
         const int* ar = na <= kColCap ? brow[q] : p.xrow + s_ptr[q];
         const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
-        const float dot = sparse_dot_fetched<32>(ar, av, na, p, q0, nb);
+        const float dot = nb <= 24 ? sparse_dot_fetched<24>(ar, av, na, p, q0, nb) : sparse_dot_fetched<32>(ar, av, na, p, q0, nb);
         if (den > 0.0 && fabs((double)dot) >= rho * den) atomicOr(&blocked_g[b >> 5], 1u << (b & 31));
       }
     }
