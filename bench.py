@@ -39,7 +39,12 @@ GRAPH_ROUNDS = 16        # untimed rounds that make sure the captured launch seq
 # DRAM bytes (read + write) per launch of the dominant kernel from ncu (dram__bytes_read.sum + dram__bytes_write.sum),
 # keyed by (workload, kernel); None where the kernel has changed since its counters were taken.  Sources: the summaries
 # under profiles/ named for the kernel and workload.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/ncu_k_gram_dense_tc_window_c3_J20000.md: 25.75 MB read + 0 written per launch (captured with J cut to 20,000;
+    # the kernel reads the window's BF16 copies only, so its traffic does not depend on J) = the algorithmic 2 N W
+    ("c3", "k_gram_dense_tc<screen>"): 25.75e6,
+    # k_walk_csc spins on a grid barrier: no multi-pass capture of it is made (one-pass launch list only)
+}
 
 
 def measured_peaks():
@@ -205,7 +210,7 @@ def rooflines(p: wl.LassoProblem, workload: str, step_ms: dict, kept_per_round: 
     if p.layout == wl.DENSE:
         # dominant: the tensor-core Gram of the window (screen on BF16 operands, split K combined inside thread-block
         # clusters, exact recheck and the greedy walk by the last CTA).  Algorithmic flops W(W-1)N.
-        kernel = "k_gram_dense_tc<screen> + k_gram_reduce"
+        kernel = "k_gram_dense_tc<screen>"
         flops = float(window) * (window - 1) * p.n_rows
         achieved = flops / (step_ms["gram_ms"] * 1e-3) / 1e12
         peak = peaks["bf16_tflops"]
@@ -272,9 +277,11 @@ def launches_per_round(p: wl.LassoProblem) -> int:
         n += 2             # pack, window Gram (screen + cluster split-K + recheck + walk)
         n += 1             # update
         if window < p.n_candidates:
-            nt = (p.n_candidates + 127) // 128
-            split = nt * (nt + 1) // 2 * 2 <= 148
-            n += 3 + (1 if split else 0) + 1 + 1 + 1   # retry branch: pack, screen, (reduce), recheck, 3xTF32, walk, gated update
+            # retry branch: walk kernel on the window (if the Gram's last CTA left it the job), pack, screen, recheck, 3xTF32,
+            # walk of the whole list, gated correction of the early list, gated update
+            n += 8
+        else:
+            n += 3         # no window: recheck, 3xTF32 fallback, walk kernel
         return n
     n = 3 + 4 + 1 + 3      # draw; bucket fill, bucket pairs, pair bits, all-pairs fallback; walk; dot, scatter, apply
     if window < p.n_candidates:

@@ -219,12 +219,10 @@ int window_of(const Problem& p, int n_cand) {
   return w * 2 <= n_cand ? (int)w : n_cand;          // a window only pays when it is well below the list
 }
 
-// retry_stream (with retry_fork): where the whole-list retry of a dense window goes instead of `s`; *branched tells
-// the caller that it did, and that the update has to be enqueued on both streams, gated either way.
+// Everything on `s`, one launch behind the other (strads_run with sampling ahead puts the retry on a branch of its
+// own instead: round_sampling_ahead).
 int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_cand, float* gram_dbg,
-                    cudaEvent_t after_pack = nullptr, cudaEvent_t after_gram = nullptr, cudaStream_t retry_stream = nullptr,
-                    cudaEvent_t retry_fork = nullptr, bool* branched = nullptr) {
-  if (branched) *branched = false;
+                    cudaEvent_t after_pack = nullptr, cudaEvent_t after_gram = nullptr) {
   const Problem& p = sc.p;
   if (p.flags & STRADS_FLAG_NO_FILTER) {
     if (after_pack) CK(cudaEventRecord(after_pack, s));
@@ -236,16 +234,7 @@ int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_
   bool walked = false;
   CK(launch_gram(sc, s, cand, window, n_cand, gram_dbg, false, after_pack, &walked));
   if (after_gram) CK(cudaEventRecord(after_gram, s));
-  // the whole-list retry -- and, behind a Gram kernel that walks, the walk kernel it may leave the job to -- go to a
-  // branch of their own when the caller has one, so that launches that normally return at once do not stand between the
-  // window and the update
   cudaStream_t rs = s;
-  if (walked && window < n_cand && retry_stream != nullptr && branched != nullptr) {
-    CK(cudaEventRecord(retry_fork, s));
-    CK(cudaStreamWaitEvent(retry_stream, retry_fork, 0));
-    rs = retry_stream;
-    *branched = true;
-  }
   CK(launch_filter(p, cand, window, n_cand, false, p.kept, rs, walked));
   if (window < n_cand) {
     if (p.layout == STRADS_CSC) {
@@ -316,7 +305,8 @@ int retry_sequence(strads_lasso_s* h, const Scheduler& sc, int window, bool earl
 // the correction and the update, gated on DeviceState::route like the copies on `main`, so that exactly one of each
 // runs.  (Tried and dropped: the branch as the body of a CUDA-graph IF node whose condition the window Gram's last CTA
 // sets -- c2 44.0 -> 42.4 us per round, c3 unchanged: evaluating the node costs about what the launches that return at
-// once do.)
+// once do.  Nor does it help to let those launches test the flags before the chain's wait: what orders them is the
+// launching of their CTAs, 4,096 for the pack and 528 with nearly all of an SM's shared memory for each Gram kernel.)
 int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
   const Scheduler& sc = h->sch[0];
   const Problem& p = sc.p;
