@@ -189,15 +189,11 @@ __device__ __forceinline__ void store_bf16x4(unsigned short* row, long long g, c
 constexpr int kPackStream = 256;                 // threads that copy (and multiply) the column
 constexpr int kPackThreads = kPackStream + 32;   // + one warp with no streaming work, for the next round's keys
 
-// One CTA per candidate: xc[a][0 .. ldc) = column cand[a] of X (128-bit copies).  With p.proposals the column is
+// One CTA per candidate at a time: xcb[a][0 .. ldc) = column cand[a] of X rounded to BF16.  With p.proposals the column is
 // also multiplied into the residual as it streams by (fixed order: per-thread strided sums, lanes by shuffle
 // tree, warps in index order) and the candidate's would-be update follows from it at once (Eq. 2): the update
 // step then only has to apply the proposals of the kept candidates.
-__global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
-                                                         int only_if_short) {
-  chain_begin();
-  const int a = blockIdx.x;
-  if (a >= n_cand || (only_if_short && !p.st->window_short)) return;
+__device__ __forceinline__ void pack_candidate(const Problem& p, const int* __restrict__ cand, int a) {
   const int j = cand[a];
   const float4* src = reinterpret_cast<const float4*>(p.xv + (long long)j * p.ld);
   const long long n4 = p.ldc >> 2;                      // ldc = N rounded up to 4 <= ld
@@ -281,6 +277,18 @@ __global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, con
     p.cand_dbeta64[a] = d;
     if (p.patch_keys != nullptr)
       p.cand_keys[p.n_cand + a] = race_key_from(s_E, (float)fabs(d), p.eta, (uint32_t)j, weight_mode_of(p.flags));
+  }
+}
+
+// The CTAs take the candidates in turn (the window's launch has one CTA per candidate; the whole-list retry, which
+// normally returns at once, a grid of a few CTAs per SM, so that an idle launch costs little).
+__global__ void __launch_bounds__(kPackThreads) k_pack_candidates(Problem p, const int* __restrict__ cand, int n_cand,
+                                                         int only_if_short) {
+  chain_begin();
+  if (only_if_short && !p.st->window_short) return;
+  for (int a = blockIdx.x; a < n_cand; a += gridDim.x) {
+    pack_candidate(p, cand, a);
+    __syncthreads();                                    // (the shared words of one candidate are reused by the next)
   }
 }
 
@@ -395,11 +403,13 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const uint32_t wait_limit = p.wait_limit ? p.wait_limit : kWaitLimit;
   if (k3x && !(p.flags & STRADS_FLAG_GRAM_3XTF32) && blockIdx.x == 0 && tid == 0)
     atomicOr(&p.st->status, STRADS_STATUS_GRAM_FALLBACK);
-  // With n_split > 1 the K range of a tile is shared by the n_split CTAs of a cluster (consecutive block indices).
-  const int tile = blockIdx.x / n_split, split = blockIdx.x - tile * n_split;
-  int ti = 0, rem = tile;                              // linear index -> (ti, tj), ti <= tj
-  while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
-  const int tj = ti + rem;
+  // With n_split > 1 the K range of a tile is shared by the n_split CTAs of a cluster (consecutive block indices), one
+  // tile per cluster.  Without a split the CTAs take the tiles in turn (a grid of at most one CTA per SM: a launch
+  // that has nothing to do -- the whole-list retry of a round whose window sufficed -- then costs one wave of CTAs, not
+  // one per tile); the ring's stages and the barriers' phases simply run on from tile to tile.
+  const int split = blockIdx.x % n_split;
+  const int tile_first = blockIdx.x / n_split, tile_step = gridDim.x / n_split;
+  const int tiles_total = n_tiles * (n_tiles + 1) / 2;
 
   const uint32_t tiles0 = (smem_u32(dyn_smem) + 1023u) & ~1023u;      // swizzle atoms need 1024-byte alignment
   unsigned char* tiles_ptr = dyn_smem + (tiles0 - smem_u32(dyn_smem));
@@ -426,14 +436,21 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const int n_st_all = (int)((N + (long long)kBK * kSub - 1) / ((long long)kBK * kSub));   // stages of K
   const int per_split = (n_st_all + n_split - 1) / n_split;
   const int st_first = min(n_st_all, split * per_split);
-  const int n_st = min(n_st_all, st_first + per_split) - st_first;     // this CTA's stages (may be 0)
+  const int n_st = min(n_st_all, st_first + per_split) - st_first;     // this CTA's stages per tile (may be 0)
+
+  int iter = 0;
+  for (int tile = tile_first; tile < tiles_total; tile += tile_step, ++iter) {
+  const int g0 = iter * n_st;                          // stages this CTA has put through the ring before this tile
+  int ti = 0, rem = tile;                              // linear index -> (ti, tj), ti <= tj
+  while (rem >= n_tiles - ti) { rem -= n_tiles - ti; ++ti; }
+  const int tj = ti + rem;
 
   if (!k3x && warp == kTmaWarp) {
     // ------------------------------ screen: TMA producer (one lane) ------------------------------
     for (int st = 0; st < n_st; ++st) {
-      const int s = st % kStages;
+      const int g = g0 + st, s = g % kStages;
       bool got = !s_abort;
-      if (got && st >= kStages) got = mbar_wait(empty0 + 8 * s, (uint32_t)(st / kStages - 1) & 1u, wait_limit);
+      if (got && g >= kStages) got = mbar_wait(empty0 + 8 * s, (uint32_t)(g / kStages - 1) & 1u, wait_limit);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
         break;
@@ -466,7 +483,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       dst_off[i] = (uint32_t)(row * 128 + ((chunk ^ (row & 7)) << 4));
     }
     auto issue = [&](int st) {                         // all copies of one stage
-      const uint32_t sb = tiles0 + (uint32_t)(st % kStages) * kStageBytes;
+      const uint32_t sb = tiles0 + (uint32_t)((g0 + st) % kStages) * kStageBytes;
       const long long k = (long long)(st_first + st) * kBlockK + chunk * 4;
       const long long left = N - k;                    // floats of this chunk that exist
       const uint32_t bytes = left >= 4 ? 16u : (left > 0 ? (uint32_t)left * 4u : 0u);
@@ -478,12 +495,12 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
                    srcB[i] ? bytes : 0u);
       }
     };
-    for (int st = 0; st < kAhead; ++st) {              // prologue: the ring is empty, fill kAhead stages
+    for (int st = 0; st < kAhead; ++st) {              // prologue: the ring is empty (the last tile is all done), fill kAhead stages
       if (st < n_st) issue(st);
       cp_async_commit();
     }
     for (int st = 0; st < n_st; ++st) {
-      const int s = st % kStages;
+      const int s = (g0 + st) % kStages;
       cp_async_wait<kAhead - 1>();                     // this thread's copies of stage st have landed
       unsigned char* sp = tiles_ptr + (size_t)s * kStageBytes;
 #pragma unroll
@@ -500,7 +517,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
       const int nxt = st + kAhead;                     // refill the stage that st - 1 used
       if (nxt < n_st) {
         bool got = !s_abort;
-        if (got && nxt >= kStages) got = mbar_wait(empty0 + 8 * (nxt % kStages), (uint32_t)(nxt / kStages - 1) & 1u, wait_limit);
+        const int gn = g0 + nxt;
+        if (got && gn >= kStages) got = mbar_wait(empty0 + 8 * (gn % kStages), (uint32_t)(gn / kStages - 1) & 1u, wait_limit);
         if (!__all_sync(0xffffffffu, got)) {
           if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
           break;
@@ -517,8 +535,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     const uint32_t idesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
     uint32_t acc = 0;
     for (int st = 0; st < n_st; ++st) {
-      const int s = st % kStages;
-      const uint32_t ph = (uint32_t)(st / kStages) & 1u;
+      const int s = (g0 + st) % kStages;
+      const uint32_t ph = (uint32_t)((g0 + st) / kStages) & 1u;
       const bool got = !s_abort && mbar_wait(full0 + 8 * s, ph, wait_limit);
       if (!__all_sync(0xffffffffu, got)) {
         if (lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
@@ -565,7 +583,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
   const double band = screen_band(N);
   if (n_split == 1) {
     if (warp < kProducerWarps) {
-      bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
+      bool ok = !s_abort && mbar_wait(done_bar, (uint32_t)iter & 1u, wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -590,7 +608,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     // q ^ (r & 31) so that neither the row-per-thread stores nor the row-per-warp loads meet bank conflicts.
     float* park = reinterpret_cast<float*>(tiles_ptr);
     if (warp < kProducerWarps) {
-      bool ok = !s_abort && mbar_wait(done_bar, 0u, wait_limit);
+      bool ok = !s_abort && mbar_wait(done_bar, (uint32_t)iter & 1u, wait_limit);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok && lane == 0) { s_abort = 1; atomicOr(&p.st->status, STRADS_STATUS_WAIT_EXPIRED); }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -659,6 +677,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_gram_dense_tc(Problem p, const 
     asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
   }
   __syncthreads();
+  if (s_abort) break;                                  // (a wait gave up: nothing more is issued)
+  }                                                    // next tile of this CTA
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
@@ -754,18 +774,21 @@ cudaError_t launch_gram_dense_tc(const Problem& p, const void* tmap, const int* 
   q.cand_cur = cand;
   const CUtensorMap& tm = *static_cast<const CUtensorMap*>(tmap);
   cudaError_t e;
-  if ((e = launch_chained(k_pack_candidates, n_cand, kPackThreads, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
+  const int pack_ctas = only_if_short ? (n_cand < 4 * p.sm_count ? n_cand : 4 * p.sm_count) : n_cand;
+  if ((e = launch_chained(k_pack_candidates, pack_ctas, kPackThreads, 0, s, q, cand, n_cand, ois)) != cudaSuccess) return e;
   if (after_pack != nullptr && (e = cudaEventRecord(after_pack, s)) != cudaSuccess) return e;   // optional step timing
   if (!(p.flags & STRADS_FLAG_GRAM_3XTF32)) {
     const int tail = (fallback_elsewhere && !only_if_short) ? 1 : 0;
-    if ((e = launch_chained_cluster(k_gram_dense_tc<false>, tiles * n_split, kThreads, kDynSmem, s, n_split, q, tm, n_cand, n_total,
+    const int ctas = n_split > 1 ? tiles * n_split : (tiles < p.sm_count ? tiles : p.sm_count);
+    if ((e = launch_chained_cluster(k_gram_dense_tc<false>, ctas, kThreads, kDynSmem, s, n_split, q, tm, n_cand, n_total,
                                     n_tiles, n_split, ois, tail)) != cudaSuccess)
       return e;
     if (tail && walked != nullptr) *walked = true;
     if (!tail && (e = launch_chained(k_gram_recheck, p.sm_count * 2, 256, 0, s, q, ois)) != cudaSuccess) return e;
   }
   if (!fallback_elsewhere || (p.flags & STRADS_FLAG_GRAM_3XTF32))
-    return launch_chained(k_gram_dense_tc<true>, tiles, kThreads, kDynSmem, s, q, tm, n_cand, n_total, n_tiles, 1, ois, 0);
+    return launch_chained(k_gram_dense_tc<true>, tiles < p.sm_count ? tiles : p.sm_count, kThreads, kDynSmem, s, q, tm, n_cand, n_total,
+                          n_tiles, 1, ois, 0);
   return cudaSuccess;
 }
 
