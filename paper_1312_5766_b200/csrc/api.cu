@@ -168,7 +168,8 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_bin_cur = take(sizeof(unsigned int) * kHistBins);
   // sampling ahead (one scheduler, P <= kAheadMaxKeep): a second set of sampler buffers for P' + P winners.
   // Dense layouts only: measured on the CSC workloads, a draw running beside the round's many-CTA, latency-bound
-  // Gram kernels did not shorten it (c4: 102 -> 106 us per round, c5: 350 -> 384 us).
+  // Gram kernels did not shorten it (c4: 102 -> 106 us per round, c5: 350 -> 384 us; again with the on-demand walk cut
+  // to one CTA per SM so that the draw has registers to run in: c4 99 -> 103 us, c5 230 -> 281 us).
   const bool ahead = first && n_sched_of(c) == 1 && c->n_keep <= kAheadMaxKeep && c->layout == STRADS_DENSE_COLMAJOR;
   const long long n_ahead = (long long)c->n_candidates + c->n_keep < c->n_cols ? (long long)c->n_candidates + c->n_keep : c->n_cols;
   L.n_ahead = ahead ? (int)n_ahead : 0;

@@ -330,7 +330,9 @@ cudaError_t prepare_walk_csc(const Problem& p, int* grid_out) {
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_walk_csc, kThreads, 0);
   if (e != cudaSuccess) return e;
   if (per_sm < 1) return cudaErrorLaunchOutOfResources;
-  *grid_out = p.sm_count * (per_sm < 2 ? per_sm : 2);
+  // one CTA per SM: the serial part of a batch is the same in every CTA, and the grid-wide part is short, so the
+  // second CTA of an SM only slowed its neighbour and the barrier down (c5 walk 131 -> 117 us)
+  *grid_out = p.sm_count * (per_sm < 1 ? per_sm : 1);
   return cudaSuccess;
 }
 
