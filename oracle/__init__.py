@@ -66,6 +66,7 @@ def _load():
             lib.so_corr.restype = C.c_double
             lib.so_objective.restype = C.c_double
             lib.so_objective_from_scratch.restype = C.c_double
+            lib.so_objective_logistic.restype = C.c_double
             _lib = lib
     return _lib
 
@@ -279,3 +280,52 @@ def gradient(X: Matrix, resid):
     g = np.empty(X.n_cols)
     _load().so_gradient(X.ref, _p(_f64(resid)), _p(g))
     return g
+
+
+# ---- logistic loss (labels y in {0, 1}; state: beta, the margin X beta, r = y - sigma(margin), delta) ----
+def init_logistic(X: Matrix, y, c_init):
+    """Returns (n2, beta, margin, resid, delta) as float64 arrays."""
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    n2, beta, delta = np.empty(X.n_cols), np.empty(X.n_cols), np.empty(X.n_cols)
+    margin, resid = np.empty(X.n_rows), np.empty(X.n_rows)
+    _load().so_init_logistic(X.ref, _p(y), C.c_double(c_init), _p(n2), _p(beta), _p(margin), _p(resid), _p(delta))
+    return n2, beta, margin, resid, delta
+
+
+def update_logistic(X: Matrix, y, n2, lam, kept, beta, margin, resid, delta):
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    for a in (beta, margin, resid, delta):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    kept = np.ascontiguousarray(kept, dtype=np.int32)
+    dbeta = np.zeros(len(kept), dtype=np.float64)
+    _load().so_update_logistic(X.ref, _p(y), _p(_f64(n2)), C.c_double(lam), _p(kept), C.c_int32(len(kept)),
+                               _p(beta), _p(margin), _p(resid), _p(delta), _p(dbeta))
+    return dbeta
+
+
+def objective_logistic(y, margin, beta, lam):
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    margin, beta = _f64(margin), _f64(beta)
+    return float(_load().so_objective_logistic(C.c_int64(len(margin)), C.c_int64(len(beta)), _p(y), _p(margin), _p(beta),
+                                               C.c_double(lam)))
+
+
+def round_logistic(X: Matrix, y, n2, lam, eta, rho, n_cand, n_keep, seed, t, beta, margin, resid, delta, weight="square",
+                   filter="rho"):
+    """One round in place with the logistic loss.  Returns dict(cand, kept, dbeta, counts)."""
+    y = np.ascontiguousarray(y, dtype=np.float32)
+    for a in (beta, margin, resid, delta):
+        assert a.dtype == np.float64 and a.flags.c_contiguous
+    n2 = _f64(n2)
+    cand = np.empty(n_cand, dtype=np.int32)
+    kept = np.full(n_keep, -1, dtype=np.int32)
+    dbeta = np.zeros(n_keep, dtype=np.float64)
+    counts = np.zeros(4, dtype=np.int32)
+    rc = _load().so_round_logistic(X.ref, _p(y), _p(n2), C.c_double(lam), C.c_double(eta), C.c_double(rho),
+                                   C.c_int32(n_cand), C.c_int32(n_keep), C.c_uint64(seed), C.c_uint64(t),
+                                   C.c_int32(WEIGHT_MODES[weight]), C.c_int32(FILTER_MODES[filter]),
+                                   _p(beta), _p(margin), _p(resid), _p(delta), _p(cand), _p(kept), _p(dbeta), _p(counts))
+    if rc:
+        raise ValueError(f"so_round_logistic failed: {rc}")
+    nk = int(counts[2])
+    return {"cand": cand, "kept": kept[:nk].copy(), "dbeta": dbeta[:nk].copy(), "counts": counts}

@@ -510,3 +510,91 @@ void so_gradient(const so_matrix *X, const double *resid, double *g)
 {
     for (int64_t j = 0; j < X->n_cols; ++j) g[j] = col_dot_vec(X, j, resid);
 }
+
+/* ------------------------------------------------------------------------- */
+/* Logistic loss (Section 2.1, remark after Eq. 1: "it is straightforward to   */
+/* use other loss functions such as logistic-loss using the same approach      */
+/* shown in" the Shotgun paper).  Labels y_i in {0, 1}, margin m = X beta,     */
+/*   F(beta) = sum_i [ log(1 + exp(m_i)) - y_i m_i ] + lambda ||beta||_1.      */
+/* The coordinate step is that of Shotgun for this loss: the second derivative */
+/* of the loss along coordinate j is at most n_j / 4, so with g_j = x_j^T r,   */
+/* r = y - sigma(m) (minus the gradient), the minimiser of the quadratic upper */
+/* bound is                                                                    */
+/*   beta_j' = S(beta_j + 4 g_j / n_j, 4 lambda / n_j).                        */
+/* Everything else of the round (draw, filter, parallel application from one   */
+/* snapshot, delta_j = |change|) is Algorithm 1 unchanged.  State: beta, the   */
+/* margin m, and r = y - sigma(m), which plays the residual's part.            */
+/* ------------------------------------------------------------------------- */
+static double sigmoid(double m) { return m >= 0.0 ? 1.0 / (1.0 + exp(-m)) : exp(m) / (1.0 + exp(m)); }
+
+void so_init_logistic(const so_matrix *X, const float *y, double c_init, double *n2,
+                      double *beta, double *margin, double *resid, double *delta)
+{
+    so_colnorm2(X, n2);
+    for (int64_t j = 0; j < X->n_cols; ++j) { beta[j] = 0.0; delta[j] = c_init; }
+    for (int64_t i = 0; i < X->n_rows; ++i) { margin[i] = 0.0; resid[i] = (double)y[i] - 0.5; }
+}
+
+int so_update_logistic(const so_matrix *X, const float *y, const double *n2, double lambda,
+                       const int32_t *kept, int32_t n_kept,
+                       double *beta, double *margin, double *resid, double *delta, double *dbeta)
+{
+    for (int32_t a = 0; a < n_kept; ++a) {
+        const int32_t j = kept[a];
+        double d = 0.0;
+        if (n2[j] > 0.0) {
+            const double g = col_dot_vec(X, j, resid);
+            d = soft_threshold(beta[j] + 4.0 * g / n2[j], 4.0 * lambda / n2[j]) - beta[j];
+        }
+        dbeta[a] = d;
+    }
+    for (int32_t a = 0; a < n_kept; ++a) {
+        const int32_t j = kept[a];
+        const double d = dbeta[a];
+        beta[j] += d;
+        delta[j] = fabs(d);
+        if (d != 0.0) {
+            if (X->layout == 0) {
+                const float *x = X->values + j * X->ld;
+                for (int64_t i = 0; i < X->n_rows; ++i) margin[i] += (double)x[i] * d;
+            } else {
+                for (int64_t p = X->col_ptr[j]; p < X->col_ptr[j + 1]; ++p)
+                    margin[X->row_idx[p]] += (double)X->values[p] * d;
+            }
+        }
+    }
+    for (int64_t i = 0; i < X->n_rows; ++i) resid[i] = (double)y[i] - sigmoid(margin[i]);
+    return 0;
+}
+
+double so_objective_logistic(int64_t N, int64_t J, const float *y, const double *margin,
+                             const double *beta, double lambda)
+{
+    double loss = 0.0, l1 = 0.0;
+    for (int64_t i = 0; i < N; ++i) {
+        const double m = margin[i];
+        loss += (m > 0.0 ? m : 0.0) + log1p(exp(-fabs(m))) - (double)y[i] * m;      /* log(1 + e^m) - y m */
+    }
+    for (int64_t j = 0; j < J; ++j) l1 += fabs(beta[j]);
+    return loss + lambda * l1;
+}
+
+/* One whole round with the logistic loss (weight_mode / filter_mode as so_round_mode). */
+int so_round_logistic(const so_matrix *X, const float *y, const double *n2, double lambda, double eta, double rho,
+                      int32_t n_cand, int32_t n_keep, uint64_t seed, uint64_t t, int32_t weight_mode, int32_t filter_mode,
+                      double *beta, double *margin, double *resid, double *delta,
+                      int32_t *cand, int32_t *kept, double *dbeta, int32_t *counts)
+{
+    int rc = so_sample_mode(X->n_cols, delta, eta, seed, t, n_cand, weight_mode, cand);
+    if (rc) return rc;
+    int32_t nk = 0, ne = 0;
+    if (filter_mode == 0) so_filter(X, n2, cand, n_cand, n_keep, rho, NULL, 0, 0.0, kept, &nk, &ne, NULL);
+    else if (filter_mode == 1) { nk = n_cand < n_keep ? n_cand : n_keep; for (int32_t a = 0; a < nk; ++a) kept[a] = cand[a]; ne = nk; }
+    else if (filter_mode == 2) so_filter_dynamic(X, n2, cand, n_cand, n_keep, rho, beta, delta, kept, &nk, &ne);
+    else return -1;
+    so_update_logistic(X, y, n2, lambda, kept, nk, beta, margin, resid, delta, dbeta);
+    int32_t nz = 0;
+    for (int32_t a = 0; a < nk; ++a) nz += dbeta[a] != 0.0;
+    counts[0] = n_cand; counts[1] = ne; counts[2] = nk; counts[3] = nz;
+    return 0;
+}

@@ -199,3 +199,21 @@ def make_problem(cfg: dict | str, seed: int = 0, device="cpu", eta: float = 1e-6
                                    device, c["nnz_col"], c.get("zipf_a", 1.1))
         return LassoProblem(CSC, c["n_rows"], c["n_cols"], v, r, p, y, bs, lam, **common)
     raise ValueError(f"unknown kind {kind!r}")
+
+
+def to_logistic(p: LassoProblem, lam_frac: float = 0.1) -> LassoProblem:
+    """The same design with binary labels for the logistic loss: y_i = 1 where the linear response
+    x_i^T beta* + noise is positive, else 0; lambda = lam_frac * ||X^T (y - 1/2)||_inf (the smallest lambda
+    for which beta = 0 is optimal, times lam_frac)."""
+    y = (p.y > 0).to(torch.float32)
+    c = (y.double() - 0.5)
+    if p.layout == DENSE:
+        xty_max = 0.0
+        for j0 in range(0, p.n_cols, 4096):
+            xty_max = max(xty_max, float((p.values[j0:j0 + 4096, : p.n_rows].double() @ c).abs().max()))
+    else:
+        contrib = p.values.double() * c[p.row_idx.long()]
+        seg = torch.repeat_interleave(torch.arange(p.n_cols, device=p.values.device), p.col_ptr[1:] - p.col_ptr[:-1])
+        xty = torch.zeros(p.n_cols, dtype=torch.float64, device=p.values.device).index_add_(0, seg, contrib)
+        xty_max = float(xty.abs().max())
+    return dataclasses.replace(p, y=y, lam=lam_frac * xty_max, name=p.name + "+logistic")
