@@ -78,6 +78,14 @@ typedef enum { STRADS_DENSE_COLMAJOR = 0, STRADS_CSC = 1 } strads_layout_t;
                                           there (beta_j = 0, delta_j = 0) is taken to couple with nobody -- it
                                           passes the rho test and blocks no other candidate             */
 
+#define STRADS_FLAG_LOGISTIC     128u   /* logistic loss instead of the squared loss (Section 2.1, remark after Eq. 1):
+                                          y_i in {0, 1}, F = sum_i [log(1 + exp(m_i)) - y_i m_i] + lambda ||beta||_1 with
+                                          the margin m = X beta.  `resid` then holds y - sigma(m), minus the gradient
+                                          with respect to m, which plays the residual's part in every step; the
+                                          coordinate step is Shotgun's for this loss (curvature at most n_j / 4):
+                                          beta_j' = S(beta_j + 4 x_j^T resid / n_j, 4 lambda / n_j).  The margin is kept
+                                          in the workspace (strads_margin); strads_round_host is not available.     */
+
 /* limits */
 #define STRADS_MAX_CANDIDATES 16384     /* P' <= 16384 (positions in the candidate list are packed into 16 bits
                                            in the lists of pairs; the walk holds P' / 32 mask words per CTA) */
@@ -233,6 +241,10 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out);
 int strads_set_wait_limit(strads_handle_t h, uint32_t iterations);
 int strads_inject_stall(strads_handle_t h, int32_t which);
 int strads_recover(strads_handle_t h);
+
+/* STRADS_FLAG_LOGISTIC: the margin m = X beta, FP32, device [N] (points into the workspace); with beta, resid,
+ * delta and the round index it is the resumable state.  STRADS_ERR_INVALID_ARG without the flag. */
+int strads_margin(strads_handle_t h, float** dev_ptr_out);
 
 /* ||x_j||^2 as computed by init, FP64, device [J] (points into the workspace). */
 int strads_colnorm2(strads_handle_t h, const double** dev_ptr_out);

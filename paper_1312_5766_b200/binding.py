@@ -24,6 +24,7 @@ FLAG_GRAM_3XTF32 = 8
 FLAG_FULL_GRAM = 16
 FLAG_ABS_WEIGHT = 32
 FLAG_DYNAMIC_DEPS = 64
+FLAG_LOGISTIC = 128
 MAX_CANDIDATES = 16384
 STALL_WALK_BARRIER, STALL_GRAM_LOADS = 1, 2
 
@@ -32,7 +33,7 @@ EXPORTS = [
     "strads_objective", "strads_sample", "strads_filter", "strads_update", "strads_get_round",
     "strads_set_round", "strads_totals", "strads_status", "strads_colnorm2", "strads_destroy",
     "strads_error_string", "strads_last_cuda_error", "strads_profile_begin", "strads_profile_end",
-    "strads_sample_static", "strads_set_wait_limit", "strads_inject_stall", "strads_recover",
+    "strads_sample_static", "strads_set_wait_limit", "strads_inject_stall", "strads_recover", "strads_margin",
 ]
 
 
@@ -90,6 +91,7 @@ def load() -> C.CDLL:
         lib.strads_set_wait_limit.argtypes = [C.c_void_p, C.c_uint32]
         lib.strads_inject_stall.argtypes = [C.c_void_p, C.c_int32]
         lib.strads_recover.argtypes = [C.c_void_p]
+        lib.strads_margin.argtypes = [C.c_void_p, C.POINTER(C.c_void_p)]
         lib.strads_sample_static.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_uint64, C.c_uint64, C.c_int32,
                                              C.c_uint32, C.c_void_p, C.c_void_p]
         lib.strads_profile_end.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
@@ -173,6 +175,7 @@ class StradsLasso:
         cfg.layout, cfg.n_rows, cfg.n_cols, cfg.nnz, cfg.ld = self.layout, self.N, self.J, nnz, ld
         cfg.n_candidates, cfg.n_keep = self.n_candidates, self.n_keep
         self.n_schedulers = cfg.n_schedulers = int(n_schedulers)
+        cfg.flags = flags                      # (the logistic loss adds the margin to the workspace)
         need = C.c_size_t(0)
         _check(lib.strads_workspace_bytes(C.byref(cfg), C.byref(need)), "strads_workspace_bytes")
         self.workspace = torch.empty(int(need.value), dtype=torch.uint8, device=dev)
@@ -276,6 +279,13 @@ class StradsLasso:
         _check(load().strads_colnorm2(self._h, C.byref(ptr)), "strads_colnorm2")
         off = ptr.value - self.workspace.data_ptr()
         return self.workspace[off:off + 8 * self.J].view(torch.float64)
+
+    def margin(self) -> torch.Tensor:
+        """The margin X beta (FP32), a view into the workspace (logistic loss only)."""
+        ptr = C.c_void_p(None)
+        _check(load().strads_margin(self._h, C.byref(ptr)), "strads_margin")
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + 4 * self.N].view(torch.float32)
 
     def profile_begin(self, max_rounds: int) -> None:
         _check(load().strads_profile_begin(self._h, int(max_rounds)), "strads_profile_begin")

@@ -86,7 +86,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_margin, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl,
       off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
@@ -141,6 +141,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   L.off_cand_bnew = take(dense ? sizeof(float) * (size_t)c->n_candidates : 0);
   L.off_dot_partial = take(sizeof(double) * (size_t)c->n_keep * L.dot_parts);
   L.off_dot_ticket = take(sizeof(unsigned int) * (size_t)c->n_keep);
+  L.off_margin = take(first && (c->flags & STRADS_FLAG_LOGISTIC) ? sizeof(float) * (size_t)c->n_rows : 0);
   L.off_obj = take(first ? sizeof(double) * 2 * kObjBlocks : 0);
   L.cap_amb = c->layout == STRADS_DENSE_COLMAJOR ? (1 << 18) : 0;   // pairs the BF16 screen leaves to the exact recheck (1 MB)
   L.off_amb = take(sizeof(unsigned int) * (size_t)L.cap_amb);
@@ -411,6 +412,7 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.dot_partial = reinterpret_cast<double*>(ws + L.off_dot_partial);
   p.dot_ticket = reinterpret_cast<unsigned int*>(ws + L.off_dot_ticket);
   p.dot_parts = L.dot_parts;
+  p.margin = first ? first->margin : ((c->flags & STRADS_FLAG_LOGISTIC) ? reinterpret_cast<float*>(ws + L.off_margin) : nullptr);
   p.obj_partial = first ? first->obj_partial : reinterpret_cast<double*>(ws + L.off_obj);
   p.amb_pairs = reinterpret_cast<unsigned int*>(ws + L.off_amb);
   p.cap_amb = L.cap_amb;
@@ -714,6 +716,7 @@ int strads_round_host(strads_handle_t h, float* beta_host, float* resid_host, fl
                       int32_t* kept_host, float* dbeta_host, int32_t* counts_host) {
   if (h == nullptr || !beta_host || !resid_host || !delta_host) return STRADS_ERR_INVALID_ARG;
   const Problem& p = on_turn(h).p;
+  if (p.flags & STRADS_FLAG_LOGISTIC) return STRADS_ERR_UNSUPPORTED;      // (the margin lives on the device)
   // delta first, on the handle's stream: the draw can start as soon as it is there; beta and the residual follow on
   // a second stream (behind whatever the handle's stream still has in flight) and are awaited before the Gram
   CK(cudaEventRecord(h->copy_fork, h->stream));
@@ -869,6 +872,12 @@ int strads_recover(strads_handle_t h) {
   if (had_stall) drop_round_graph(h);
   h->ahead_round = -1;                                   // (whatever was drawn ahead belongs to the abandoned rounds)
   CK(cudaStreamSynchronize(h->stream));
+  return STRADS_OK;
+}
+
+int strads_margin(strads_handle_t h, float** dev_ptr_out) {
+  if (h == nullptr || dev_ptr_out == nullptr || h->sch[0].p.margin == nullptr) return STRADS_ERR_INVALID_ARG;
+  *dev_ptr_out = h->sch[0].p.margin;
   return STRADS_OK;
 }
 

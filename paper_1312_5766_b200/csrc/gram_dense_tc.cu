@@ -268,8 +268,9 @@ __device__ __forceinline__ void pack_candidate(const Problem& p, const int* __re
     for (int w = 0; w < kPackStream / 32; ++w) g += wsum[w];
     float b_new = b_old;
     if (n > 0.0) {
-      const double z = (double)b_old + g / n;
-      const double m = fabs(z) - (double)p.lambda / n;
+      const double c = step_scale(p);
+      const double z = (double)b_old + c * g / n;
+      const double m = fabs(z) - c * (double)p.lambda / n;
       b_new = (float)(m <= 0.0 ? 0.0 : (z > 0.0 ? m : -m));
     }
     const double d = isfinite(g) ? (double)b_new - (double)b_old : g - g;      // a non-finite product shows as NaN

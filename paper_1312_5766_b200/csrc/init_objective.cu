@@ -68,7 +68,11 @@ __global__ void k_fill_state(Problem p) {
   const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long j = i; j < p.J; j += stride) p.delta[j] = p.c_init;
-  for (long long r = i; r < p.N; r += stride) p.resid[r] = p.y[r];
+  const bool logistic = (p.flags & STRADS_FLAG_LOGISTIC) != 0;        // margin 0: resid = y - sigma(0)
+  for (long long r = i; r < p.N; r += stride) {
+    p.resid[r] = logistic ? p.y[r] - 0.5f : p.y[r];
+    if (logistic) p.margin[r] = 0.f;
+  }
   if (i == 0) {
     DeviceState* st = p.st;
     st->round = 0;
@@ -89,7 +93,12 @@ __global__ void k_resid_dense(Problem p) {
     const float b = p.beta[j];
     if (b != 0.f) acc += (double)p.xv[j * p.ld + i] * (double)b;
   }
-  p.resid[i] = (float)((double)p.y[i] - acc);
+  if (p.flags & STRADS_FLAG_LOGISTIC) {
+    p.margin[i] = (float)acc;
+    p.resid[i] = (float)((double)p.y[i] - sigmoid64((double)(float)acc));
+  } else {
+    p.resid[i] = (float)((double)p.y[i] - acc);
+  }
 }
 
 // CSC: one CTA walks the columns in index order; rows inside a column are distinct, so the
@@ -99,10 +108,16 @@ __global__ void __launch_bounds__(1024) k_resid_csc(Problem p) {
   for (long long j = 0; j < p.J; ++j) {
     const float b = p.beta[j];
     if (b == 0.f) continue;
-    for (long long q = p.xptr[j] + threadIdx.x; q < p.xptr[j + 1]; q += blockDim.x)
-      p.resid[p.xrow[q]] = (float)((double)p.resid[p.xrow[q]] - (double)p.xv[q] * (double)b);
+    for (long long q = p.xptr[j] + threadIdx.x; q < p.xptr[j + 1]; q += blockDim.x) {
+      const int r = p.xrow[q];
+      if (p.flags & STRADS_FLAG_LOGISTIC) p.margin[r] = (float)((double)p.margin[r] + (double)p.xv[q] * (double)b);
+      else p.resid[r] = (float)((double)p.resid[r] - (double)p.xv[q] * (double)b);
+    }
     __syncthreads();
   }
+  if (p.flags & STRADS_FLAG_LOGISTIC)
+    for (long long r = threadIdx.x; r < p.N; r += blockDim.x)
+      p.resid[r] = (float)((double)p.y[r] - sigmoid64((double)p.margin[r]));
 }
 
 __global__ void k_any_nonzero(Problem p) {
@@ -115,7 +130,14 @@ __global__ void __launch_bounds__(256) k_objective_partial(Problem p) {
   double sq = 0.0, l1 = 0.0;
   const long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   const long long stride = (long long)gridDim.x * blockDim.x;
-  for (long long i = i0; i < p.N; i += stride) { const double r = p.resid[i]; sq += r * r; }
+  if (p.flags & STRADS_FLAG_LOGISTIC) {                  // sum_i log(1 + exp(m_i)) - y_i m_i (twice: halved with the squares' 1/2)
+    for (long long i = i0; i < p.N; i += stride) {
+      const double m = p.margin[i];
+      sq += 2.0 * ((m > 0.0 ? m : 0.0) + log1p(exp(-fabs(m))) - (double)p.y[i] * m);
+    }
+  } else {
+    for (long long i = i0; i < p.N; i += stride) { const double r = p.resid[i]; sq += r * r; }
+  }
   for (long long j = i0; j < p.J; j += stride) l1 += fabs((double)p.beta[j]);
   const double a = block_sum(sq);
   const double b = block_sum(l1);

@@ -92,6 +92,7 @@ struct Problem {
   double* dot_partial;          // [n_keep][dot_parts]
   unsigned int* dot_ticket;     // [n_keep]
   int dot_parts;
+  float* margin;                // STRADS_FLAG_LOGISTIC: [N] the margin X beta (shared by all schedulers)
   double* obj_partial;          // [2 * kObjBlocks]
   unsigned int* amb_pairs;      // [cap_amb] (a << 16 | b), positions in the candidate list
   int cap_amb;
@@ -254,6 +255,22 @@ __device__ __forceinline__ void next_round_keys(const Problem& p, uint32_t j, fl
 __device__ __forceinline__ double coupling_n2(const Problem& p, int j) {
   if ((p.flags & STRADS_FLAG_DYNAMIC_DEPS) && p.beta[j] == 0.f && p.delta[j] == 0.f) return 0.0;
   return p.n2[j];
+}
+
+// The two losses.  Squared loss: resid = y - X beta, the step of Eq. 2.  Logistic loss (STRADS_FLAG_LOGISTIC): resid =
+// y - sigma(margin), and the second derivative of the loss along x_j is at most n_j / 4, which scales the step and its
+// threshold by 4 (Shotgun's step for this loss).
+__device__ __forceinline__ double step_scale(const Problem& p) { return (p.flags & STRADS_FLAG_LOGISTIC) ? 4.0 : 1.0; }
+__device__ __forceinline__ double sigmoid64(double m) { return m >= 0.0 ? 1.0 / (1.0 + exp(-m)) : exp(m) / (1.0 + exp(m)); }
+// Row i after the kept coefficients have moved the linear predictor x_i^T beta by s.
+__device__ __forceinline__ void apply_row(const Problem& p, long long i, double s) {
+  if (p.flags & STRADS_FLAG_LOGISTIC) {
+    const float m = (float)((double)p.margin[i] + s);
+    p.margin[i] = m;
+    p.resid[i] = (float)((double)p.y[i] - sigmoid64((double)m));
+  } else {
+    p.resid[i] = (float)((double)p.resid[i] - s);
+  }
 }
 
 // x_a^T x_b of two CSC columns (ascending rows): a given as arrays (possibly staged in shared memory), b read

@@ -32,8 +32,9 @@ __device__ void finish_coefficient(const Problem& p, int a, int j, double g) {
   const float b_old = p.beta[j];
   float b_new = b_old;
   if (n > 0.0) {
-    const double z = (double)b_old + g / n;
-    const double m = fabs(z) - (double)p.lambda / n;
+    const double c = step_scale(p);
+    const double z = (double)b_old + c * g / n;
+    const double m = fabs(z) - c * (double)p.lambda / n;
     b_new = (float)(m <= 0.0 ? 0.0 : (z > 0.0 ? m : -m));
   }
   const double d = (double)b_new - (double)b_old;        // the change that beta (FP32) really makes
@@ -209,7 +210,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_dense(Problem p, const int* 
       double s = 0.0;
 #pragma unroll
       for (int w = 0; w < kColSlots; ++w) s += part[w][tid];
-      if (s != 0.0) p.resid[r] = (float)((double)p.resid[r] - s);
+      if (s != 0.0) apply_row(p, r, s);
     }
   }
   DeviceState* st = p.st;
@@ -305,7 +306,7 @@ __global__ void __launch_bounds__(kThreads) k_apply_csc(Problem p, int advance) 
     for (long long r = (long long)blockIdx.x * kThreads + threadIdx.x; r < p.N; r += stride) {
       const long long v = p.resid_acc[r];
       if (v != 0) {
-        p.resid[r] = (float)((double)p.resid[r] - ldexp((double)v, -shift));
+        apply_row(p, r, ldexp((double)v, -shift));
         p.resid_acc[r] = 0;
       }
     }
