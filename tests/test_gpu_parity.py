@@ -644,3 +644,32 @@ def test_state_written_by_the_caller_between_runs():
     for x, y in ((a.beta, ref.beta), (a.resid, ref.resid), (a.delta, ref.delta)):
         assert torch.equal(x, y)
     assert a.get_round() == ref.get_round() == 55
+
+
+@pytest.mark.parametrize("name", ["csc", "csc_zipf"])
+def test_csc_residual_update_is_exact_to_fp32_rounding(name):
+    """CSC residual update: contributions are added as 64-bit fixed-point integers (unit 2^-(61 - e), 2^e above the
+    largest possible row sum), so what reaches a row is the exact sum to ~2^-60 of that bound, whatever the order of
+    the additions -- hot rows of the Zipf design collect hundreds of terms.  The new residual must therefore be the
+    FP32 rounding of the exact one: equal to it, or one ulp off where the exact value sits on a rounding boundary."""
+    p = wl.make_problem(_small_problems()[name], seed=61)
+    s = _solver(p)
+    v, r_idx, cp = p.values.numpy().astype(np.float64), p.row_idx.numpy(), p.col_ptr.numpy()
+    rng = np.random.default_rng(3)
+    for step in range(4):
+        s.run(3)                                            # some state with non-trivial beta
+        kept = rng.permutation(p.n_cols)[: p.n_keep].astype(np.int32)
+        b_old = s.beta.cpu().numpy().astype(np.float64)
+        r_old = s.resid.cpu().numpy().astype(np.float64)
+        s.update(torch.from_numpy(kept).cuda())
+        d = s.beta.cpu().numpy().astype(np.float64) - b_old                  # the changes, exactly (differences of floats)
+        assert np.count_nonzero(d) > p.n_keep // 4 and not d[np.setdiff1d(np.arange(p.n_cols), kept)].any()
+        moved = np.zeros(p.n_rows)
+        for j in np.flatnonzero(d):
+            np.add.at(moved, r_idx[cp[j]:cp[j + 1]], v[cp[j]:cp[j + 1]] * d[j])
+        want = (r_old - moved).astype(np.float32)
+        got = s.resid.cpu().numpy()
+        ulp = np.spacing(np.abs(want).astype(np.float32))
+        assert np.all(np.abs(got.astype(np.float64) - want.astype(np.float64)) <= ulp)
+        assert np.mean(got != want) < 1e-3                  # (ties of the last bit only)
+    assert s.status() == (0, 0)
