@@ -36,16 +36,17 @@ __global__ void __launch_bounds__(kThreads) k_csc_bucket_fill(Problem p, const i
   if (blockIdx.x == 0 && threadIdx.x == 0) { st->bucket_used = use ? 1 : 0; st->pair_count = 0; st->bucket_failed = 0; }
   if (!use) return;
   const int lane = threadIdx.x & 31;
-  const int a = (int)((blockIdx.x * (unsigned)kThreads + threadIdx.x) >> 5);
-  if (a >= n_cand) return;
   const int words = (n_cand + 31) >> 5;
-  for (int w = lane; w < words; w += 32) p.conflict[(long long)a * p.mask_words + w] = 0u;
-  const int ja = cand[a];
-  const long long q1 = p.xptr[ja + 1];
-  for (long long q = p.xptr[ja] + lane; q < q1; q += 32) {
-    const int r = __ldg(p.xrow + q);
-    const unsigned int slot = atomicAdd(&p.bucket_count[r], 1u);
-    if (slot < (unsigned)kBucketSlots) p.bucket_items[(long long)r * kBucketSlots + slot] = a;
+  const int n_warps = (int)(gridDim.x * (unsigned)kThreads) >> 5;
+  for (int a = (int)((blockIdx.x * (unsigned)kThreads + threadIdx.x) >> 5); a < n_cand; a += n_warps) {
+    for (int w = lane; w < words; w += 32) p.conflict[(long long)a * p.mask_words + w] = 0u;
+    const int ja = cand[a];
+    const long long q1 = p.xptr[ja + 1];
+    for (long long q = p.xptr[ja] + lane; q < q1; q += 32) {
+      const int r = __ldg(p.xrow + q);
+      const unsigned int slot = atomicAdd(&p.bucket_count[r], 1u);
+      if (slot < (unsigned)kBucketSlots) p.bucket_items[(long long)r * kBucketSlots + slot] = a;
+    }
   }
 }
 
@@ -54,8 +55,11 @@ __global__ void __launch_bounds__(kThreads) k_csc_bucket_pairs(Problem p) {
   chain_begin();
   DeviceState* st = p.st;
   if (!st->bucket_used) return;
-  const long long r = (long long)blockIdx.x * kThreads + threadIdx.x;
   const int lane = threadIdx.x & 31;
+  // (the grid is capped, so that a launch with nothing to do costs little: a thread takes several rows in turn; the
+  //  trip count is the same for all lanes of a warp)
+  for (long long r0 = (long long)blockIdx.x * kThreads; r0 < p.N; r0 += (long long)gridDim.x * kThreads) {
+  const long long r = r0 + threadIdx.x;
   unsigned int c = 0;
   if (r < p.N) {
     c = p.bucket_count[r];
@@ -70,15 +74,15 @@ __global__ void __launch_bounds__(kThreads) k_csc_bucket_pairs(Problem p) {
     if (lane >= o) incl += v;
   }
   const unsigned int total = __shfl_sync(0xffffffffu, incl, 31);
-  if (total == 0) return;
+  if (total == 0) continue;
   unsigned int base = 0;
   if (lane == 31) base = atomicAdd(&st->pair_count, total);
   base = __shfl_sync(0xffffffffu, base, 31);
   if (base + total > (unsigned)p.pair_cap) {          // the list is full: this round falls back to all pairs
     if (lane == 31) st->bucket_failed = 1;
-    return;
+    continue;
   }
-  if (mine == 0) return;
+  if (mine == 0) continue;
   unsigned int at = base + incl - mine;
   const int* items = p.bucket_items + r * kBucketSlots;
   int it[kBucketSlots];
@@ -92,6 +96,7 @@ __global__ void __launch_bounds__(kThreads) k_csc_bucket_pairs(Problem p) {
         const int lo = min(it[i], it[j]), hi = max(it[i], it[j]);
         p.pair_list[at++] = ((unsigned int)lo << 16) | (unsigned int)hi;
       }
+  }
 }
 
 // Step 3: a thread per listed pair merges the two columns and sets the pair's conflict bit in the row of the
@@ -132,8 +137,8 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
   if (blockIdx.x == 0 && threadIdx.x == 0) p.st->edges_off = 1;     // this kernel sets bits without listing the pairs
   __shared__ int arow[kStage];
   __shared__ float aval[kStage];
-  const int a = blockIdx.x;
-  if (a >= n_cand) return;
+  for (int a = blockIdx.x; a < n_cand; a += gridDim.x) {   // (capped grid: the CTAs take the candidates in turn)
+  if (a != (int)blockIdx.x) __syncthreads();               // the staged column of the last candidate is no longer read
   const int ja = cand[a];
   const long long a0 = p.xptr[ja];
   const int na = (int)(p.xptr[ja + 1] - a0);
@@ -165,6 +170,7 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
     const unsigned int word = __ballot_sync(0xffffffffu, hit);
     if (lane == 0) p.conflict[(long long)a * p.mask_words + w] = word;
   }
+  }
 }
 
 }  // namespace
@@ -172,14 +178,18 @@ __global__ void __launch_bounds__(kThreads) k_gram_csc(Problem p, const int* __r
 cudaError_t launch_gram_csc(const Problem& p, const int* cand, int n_cand, float* gram_dbg, bool only_if_short,
                             bool window, cudaStream_t s) {
   const int ois = only_if_short ? 1 : 0, win = window ? 1 : 0;
+  // grids of at most eight CTAs per SM: in many rounds (a window that keeps failing is skipped) these launches have
+  // nothing to do, and what an idle launch costs is the launching of its CTAs
+  const long long cap = (long long)p.sm_count * 8;
+  auto capped = [&](long long n) { return (unsigned)(n < cap ? (n > 0 ? n : 1) : cap); };
   if (p.bucket_count == nullptr || gram_dbg != nullptr || n_cand > 65535)
-    return launch_chained(k_gram_csc, n_cand, kThreads, 0, s, p, cand, n_cand, gram_dbg, ois, win, 0);
+    return launch_chained(k_gram_csc, capped(n_cand), kThreads, 0, s, p, cand, n_cand, gram_dbg, ois, win, 0);
   cudaError_t e;
-  if ((e = launch_chained(k_csc_bucket_fill, (n_cand * 32 + kThreads - 1) / kThreads, kThreads, 0, s, p, cand, n_cand, ois, win)) != cudaSuccess)
+  if ((e = launch_chained(k_csc_bucket_fill, capped(((long long)n_cand * 32 + kThreads - 1) / kThreads), kThreads, 0, s, p, cand, n_cand, ois, win)) != cudaSuccess)
     return e;
-  if ((e = launch_chained(k_csc_bucket_pairs, (unsigned)((p.N + kThreads - 1) / kThreads), kThreads, 0, s, p)) != cudaSuccess) return e;
+  if ((e = launch_chained(k_csc_bucket_pairs, capped((p.N + kThreads - 1) / kThreads), kThreads, 0, s, p)) != cudaSuccess) return e;
   if ((e = launch_chained(k_csc_pair_bits, p.sm_count * 8, kThreads, 0, s, p, cand)) != cudaSuccess) return e;
-  return launch_chained(k_gram_csc, n_cand, kThreads, 0, s, p, cand, n_cand, gram_dbg, ois, win, 1);
+  return launch_chained(k_gram_csc, capped(n_cand), kThreads, 0, s, p, cand, n_cand, gram_dbg, ois, win, 1);
 }
 
 }  // namespace strads
