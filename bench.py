@@ -234,8 +234,8 @@ def rooflines(p: wl.LassoProblem, workload: str, step_ms: dict, kept_per_round: 
             ops = kept_per_round * examined_per_round * (2.0 * nnz_col - 1.0)
             ms = step_ms["walk_ms"]
         else:
-            # dominant: the merges of the window's pairs that share a row
-            kernel = "k_csc_pair_bits"
+            # dominant: the inner products of the window's pairs that share a row
+            kernel = "k_csc_bucket_dots"
             ops = 0.5 * window * (window - 1) * (nnz_col * nnz_col / p.n_rows) * (2.0 * nnz_col - 1.0)
             ms = step_ms["gram_ms"]
         peak = 148 * 128 * peaks["sm_max_mhz"] * 1e6 / 1e12        # integer / FP32 lanes x clock, T op/s
@@ -283,7 +283,7 @@ def launches_per_round(p: wl.LassoProblem) -> int:
         else:
             n += 3         # no window: recheck, 3xTF32 fallback, walk kernel
         return n
-    n = 3 + 4 + 1 + 3      # draw; bucket fill, bucket pairs, pair bits, all-pairs fallback; walk; dot, scatter, apply
+    n = 3 + 3 + 1 + 3      # draw; bucket fill, bucket dots, all-pairs fallback; walk; dot, scatter, apply
     if window < p.n_candidates:
         n += 1             # cooperative on-demand walk
     return n

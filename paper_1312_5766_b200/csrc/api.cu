@@ -87,10 +87,11 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
       off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_margin, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl,
-      off_bucket_count, off_bucket_items, off_pairs, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
+      off_bucket_count, off_bucket_items, off_bucket_vals, off_bucket_cols, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
-  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, pair_cap, n_ahead, cap_ahead_boundary, cap_survivors;
+  int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, n_ahead, cap_ahead_boundary, cap_survivors;
   long long ldc, ldcb;
+  bool buckets;
 };
 
 int n_sched_of(const strads_lasso_config_t* c) { return c->n_schedulers > 1 ? c->n_schedulers : 1; }
@@ -151,12 +152,12 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
-  // CSC Gram by row buckets: provided for while the buckets stay below 64 MB (N <= 2^20)
-  const bool buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);
-  L.pair_cap = buckets ? (1 << 20) : 0;
-  L.off_bucket_count = take(buckets ? sizeof(unsigned int) * (size_t)c->n_rows : 0);
-  L.off_bucket_items = take(buckets ? sizeof(int) * (size_t)c->n_rows * kBucketSlots : 0);
-  L.off_pairs = take(sizeof(unsigned int) * (size_t)L.pair_cap);
+  // CSC Gram by row buckets: provided for while the buckets' candidate lists stay below 64 MB (N <= 2^20; their values take as much)
+  L.buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);
+  L.off_bucket_count = take(L.buckets ? sizeof(unsigned int) * (size_t)c->n_rows : 0);
+  L.off_bucket_items = take(L.buckets ? sizeof(int) * (size_t)c->n_rows * kBucketSlots : 0);
+  L.off_bucket_vals = take(L.buckets ? sizeof(float) * (size_t)c->n_rows * kBucketSlots : 0);
+  L.off_bucket_cols = take(L.buckets ? sizeof(BucketColumn) * (size_t)c->n_candidates : 0);
   L.off_resid_acc = take(csc ? sizeof(long long) * (size_t)c->n_rows : 0);
   L.off_delta_prev = take(sizeof(float) * (size_t)c->n_keep);
   L.off_edges = take(sizeof(unsigned int) * kEdgeCap);
@@ -428,10 +429,10 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
   p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
   p.resid_acc = reinterpret_cast<long long*>(ws + L.off_resid_acc);
-  p.pair_cap = L.pair_cap;
-  p.bucket_count = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
-  p.bucket_items = L.pair_cap ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;
-  p.pair_list = L.pair_cap ? reinterpret_cast<unsigned int*>(ws + L.off_pairs) : nullptr;
+  p.bucket_count = L.buckets ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
+  p.bucket_items = L.buckets ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;
+  p.bucket_vals = L.buckets ? reinterpret_cast<float*>(ws + L.off_bucket_vals) : nullptr;
+  p.bucket_cols = L.buckets ? reinterpret_cast<BucketColumn*>(ws + L.off_bucket_cols) : nullptr;
   p.part_count = S; p.part_index = s;
   p.sm_count = first ? first->sm_count : 0;
   p.round_ptr = &p.st->round; p.round_ahead = 0;

@@ -32,7 +32,6 @@ struct DeviceState {
   unsigned int amb_count;       // pairs the BF16 screen of the dense Gram left to the exact recheck
   int window_short;             // the filter ran out of its candidate window before P were kept: redo on all P'
   int prefer_walk;              // CSC: the last round needed the whole list, so skip the window attempt for a while
-  unsigned int pair_count;      // CSC Gram by row buckets: candidate pairs found to share a row (append cursor)
   int bucket_failed;            // ... a bucket or the pair list overflowed this round: the all-pairs kernel redoes the bits
   int bucket_avoid;             // ... it overflowed lately: go straight to the all-pairs kernel for a while
   unsigned long long dmax_bits; // CSC update: bits of max |change| of this round (non-negative doubles order like integers)
@@ -57,6 +56,13 @@ struct WalkControl {            // shared by the CTAs of the cooperative on-dema
 };
 
 static constexpr int kBucketSlots = 16;   // candidates per row bucket (more: the round falls back to all pairs)
+// What the bucket kernels need of a candidate's column, gathered once per round (one access instead of a chain of three).
+struct BucketColumn {
+  long long q0;     // first stored entry
+  int n;            // entries
+  int j;            // the column
+  double n2;        // its coupling_n2
+};
 static constexpr int kHistBits = 12;
 static constexpr int kHistBins = 1 << kHistBits;
 
@@ -111,8 +117,8 @@ struct Problem {
   // CSC Gram by row buckets (null / 0 when not provided for)
   unsigned int* bucket_count;   // [N] candidates of this round's list with an entry in row i (zero between rounds)
   int* bucket_items;            // [N][kBucketSlots] their positions in the list
-  unsigned int* pair_list;      // [pair_cap] (a << 16 | b), a < b: positions of two candidates that share a row
-  int pair_cap;
+  float* bucket_vals;           // [N][kBucketSlots] their values in row i
+  BucketColumn* bucket_cols;    // [P'] where each candidate's column lies, as the bucket kernels need it
   int sm_count;
   // sampling ahead (one scheduler): the draw of round t + 1 is made during round t from the priorities of its start
   // and corrected for the coefficients that round t updates (k_sample_patch)

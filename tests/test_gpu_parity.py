@@ -215,6 +215,45 @@ def test_filter_matches_oracle(name):
         assert rejected > 0
 
 
+CSC_GRAM_CASES = {
+    # most pairs share no row: the Gram comes from the row buckets (a few candidates per row)
+    "few_per_row": (dict(kind="csc_uniform", n_rows=5000, n_cols=20000, n_true=100, lam_frac=0.01, nnz_col=50,
+                         n_candidates=1024, n_keep=128, rho=0.1), [1024, 700, 33, 2]),
+    # rows of Zipf frequency hold far more candidates than a bucket does: all pairs instead
+    "crowded_rows": (dict(kind="csc_zipf", n_rows=2000, n_cols=30000, n_true=100, lam_frac=0.01, nnz_col=20,
+                          n_candidates=1024, n_keep=128, rho=0.1, zipf_a=1.1), [1024, 300]),
+    # no bucket overflows (16 candidates in all), but every candidate shares ~40 rows with every other: more terms
+    # than one candidate's sort takes, all pairs instead
+    "everyone_meets_everyone": (dict(kind="csc_uniform", n_rows=48, n_cols=64, n_true=4, lam_frac=0.01, nnz_col=44,
+                                     n_candidates=16, n_keep=8, rho=0.1), [16, 12]),
+}
+
+
+@pytest.mark.parametrize("case", list(CSC_GRAM_CASES))
+def test_csc_filter_without_gram_output(case):
+    """The filter as the rounds run it (no Gram matrix asked for, so the CSC path may take its inner products from the
+    row buckets), on designs that keep to the buckets, overflow them, or collect too many terms for one candidate."""
+    cfg, sizes = CSC_GRAM_CASES[case]
+    p = wl.make_problem(cfg, seed=5)
+    X = oracle_matrix(p)
+    n2 = oracle.colnorm2(X)
+    s = _solver(p)
+    rho = float(np.float32(p.rho))
+    rng = np.random.default_rng(1)
+    rejected = 0
+    for rep in range(3):                                    # (a failed attempt changes what the next call tries first)
+        for n_cand in sizes:
+            cand = rng.permutation(p.n_cols)[:n_cand].astype(np.int32)
+            kept_d, counts_d = s.filter(torch.from_numpy(cand).cuda(), want_gram=False)
+            counts = counts_d.cpu().numpy()
+            kept = kept_d.cpu().numpy()
+            nk = int(counts[2])
+            assert np.all(kept[nk:] == -1) and counts[0] == n_cand
+            _assert_kept_matches(X, n2, cand, p.n_keep, rho, kept[:nk], int(counts[1]))
+            rejected += int(counts[1]) - nk
+    assert rejected > 0
+
+
 @pytest.mark.parametrize("name", list(_small_problems()))
 def test_update_matches_oracle(name):
     p = wl.make_problem(_small_problems()[name], seed=4)
