@@ -167,7 +167,7 @@ __device__ void find_bin(const unsigned int* h, int nbins, long long k_rem, int*
 // mode 0: plain.  mode 1: bins only the keys below a cutoff carried over from the previous round (four times that
 // round's boundary; the keys certainly above it are not even computed); if fewer than P' keys turn out to lie
 // below it, the last CTA redoes the pass in full by itself.
-__global__ void __launch_bounds__(kThreads) k_sample_hist(Problem p, int mode) {
+__global__ void __launch_bounds__(kThreads, 4) k_sample_hist(Problem p, int mode) {
   chain_begin();
   __shared__ unsigned int sh[kHistBins];
   __shared__ int s_last;
@@ -634,7 +634,9 @@ cudaError_t launch_sample(const Problem& p, int* cand_out, cudaStream_t s) {
   const long long groups = (p.J + 3) >> 2;
   long long blocks = (groups + kThreads - 1) / kThreads;
   // (an early draw runs beside the round's Gram and walk and leaves them most of every SM)
-  const long long cap = (long long)p.sm_count * (p.round_ahead ? 2 : 8);
+  // otherwise as many CTAs as run at once (four per SM, by the kernels' registers): each pays for its own histogram
+  // (cleared, then merged into the global one) once, and the passes are bound by arithmetic, not by the grid's size
+  const long long cap = (long long)p.sm_count * (p.round_ahead ? 2 : 4);
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   cudaError_t e;
