@@ -309,7 +309,12 @@ int retry_sequence(strads_lasso_s* h, const Scheduler& sc, int window, bool earl
 // runs.  (Tried and dropped: the branch as the body of a CUDA-graph IF node whose condition the window Gram's last CTA
 // sets -- c2 44.0 -> 42.4 us per round, c3 unchanged: evaluating the node costs about what the launches that return at
 // once do.  Nor does it help to let those launches test the flags before the chain's wait: what orders them is the
-// launching of their CTAs, 4,096 for the pack and 528 with nearly all of an SM's shared memory for each Gram kernel.)
+// launching of their CTAs, 4,096 for the pack and 528 with nearly all of an SM's shared memory for each Gram kernel.
+// Also tried and dropped: the pack step taken apart between captured rounds -- the BF16 copies of the next window
+// behind the correction of its list, beside this round's update, and the proposals (which need the residual that
+// update leaves) on a stream of their own beside the next Gram, so that the path would be correction -> copies -> Gram.
+// Same results, but the columns are read twice and the kernels that overlap share one memory system: c3 68 -> 86 us
+// per round, c2 39 -> 42 us.)
 int round_sampling_ahead(strads_lasso_s* h, bool have_list, cudaStream_t main) {
   const Scheduler& sc = h->sch[0];
   const Problem& p = sc.p;
