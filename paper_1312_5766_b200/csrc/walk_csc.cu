@@ -158,22 +158,23 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
     }
     __syncthreads();
     {
-      const int qa = tid >> 3;                         // eight threads per member qa: partners qb = tid % 8 + 8 k
-      if (qa < m) {
-        const int na = s_len[qa];
-        unsigned int hits = 0u;
-        // the (up to four) merges of this thread run side by side, one step of each per trip: the steps of one merge
-        // depend on each other (load, compare, advance), those of different merges do not
-        int qbs[4], nbs[4], ii[4], kk[4];
-        float dots[4];
-        bool staged = na <= kColCap;
+      // the m (m - 1) / 2 pairs (qa < qb) in turn over the threads: two per thread for a full batch, side by side,
+      // one step of each per trip (the steps of one merge depend on each other, those of different merges do not)
+      constexpr int kSide = 2;
+      const int n_pairs = m * (m - 1) / 2;
+      for (int p0 = tid; p0 < n_pairs; p0 += kSide * kThreads) {
+        int qas[kSide], qbs[kSide], nas[kSide], nbs[kSide], ii[kSide], kk[kSide];
+        float dots[kSide];
+        bool staged = true;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int qb = (tid & 7) + 8 * u;
-          const bool on = qb < m && qb > qa;
-          qbs[u] = on ? qb : qa;
-          nbs[u] = on ? s_len[qb] : 0;
-          staged = staged && nbs[u] <= kColCap;
+        for (int u = 0; u < kSide; ++u) {
+          int left = p0 + u * kThreads;
+          const bool on = left < n_pairs;
+          int qa = 0;
+          if (on) while (left >= m - 1 - qa) { left -= m - 1 - qa; ++qa; }     // pair number -> (qa, qb), rows of m-1, m-2, ...
+          qas[u] = qa; qbs[u] = on ? qa + 1 + left : qa;
+          nas[u] = on ? s_len[qa] : 0; nbs[u] = on ? s_len[qbs[u]] : 0;
+          staged = staged && nas[u] <= kColCap && nbs[u] <= kColCap;
           ii[u] = 0; kk[u] = 0; dots[u] = 0.f;
         }
         if (staged) {
@@ -181,11 +182,11 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
           while (any) {
             any = false;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const bool on = ii[u] < na && kk[u] < nbs[u];
+            for (int u = 0; u < kSide; ++u) {
+              const bool on = ii[u] < nas[u] && kk[u] < nbs[u];
               const int i = on ? ii[u] : 0, k = on ? kk[u] : 0;
-              const int ra = brow[qa][i], rb = brow[qbs[u]][k];
-              const float pa = bval[qa][i], pb = bval[qbs[u]][k];
+              const int ra = brow[qas[u]][i], rb = brow[qbs[u]][k];
+              const float pa = bval[qas[u]][i], pb = bval[qbs[u]][k];
               dots[u] = (on && ra == rb) ? fmaf(pa, pb, dots[u]) : dots[u];
               ii[u] += (on && ra <= rb) ? 1 : 0;
               kk[u] += (on && rb <= ra) ? 1 : 0;
@@ -193,22 +194,21 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
             }
           }
         } else {                                       // a column too long for its slot: plain merges from global memory
-          const int* ar = na <= kColCap ? brow[qa] : p.xrow + s_ptr[qa];
-          const float* av = na <= kColCap ? bval[qa] : p.xv + s_ptr[qa];
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int qb = qbs[u], nb = nbs[u];
+          for (int u = 0; u < kSide; ++u) {
+            const int qa = qas[u], qb = qbs[u], na = nas[u], nb = nbs[u];
+            const int* ar = na <= kColCap ? brow[qa] : p.xrow + s_ptr[qa];
+            const float* av = na <= kColCap ? bval[qa] : p.xv + s_ptr[qa];
             const int* br = nb <= kColCap ? brow[qb] : p.xrow + s_ptr[qb];
             const float* bv = nb <= kColCap ? bval[qb] : p.xv + s_ptr[qb];
             dots[u] = sparse_dot_arrays(ar, av, na, br, bv, nb);
           }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const double den = sqrt(s_n2[qa] * s_n2[qbs[u]]);
-          if (nbs[u] > 0 && den > 0.0 && fabs((double)dots[u]) >= rho * den) hits |= 1u << qbs[u];
+        for (int u = 0; u < kSide; ++u) {
+          const double den = sqrt(s_n2[qas[u]] * s_n2[qbs[u]]);
+          if (nbs[u] > 0 && nas[u] > 0 && den > 0.0 && fabs((double)dots[u]) >= rho * den) atomicOr(&s_conf[qas[u]], 1u << qbs[u]);
         }
-        if (hits) atomicOr(&s_conf[qa], hits);
       }
     }
     __syncthreads();
