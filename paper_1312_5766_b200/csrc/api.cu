@@ -86,7 +86,7 @@ int pow2_ceil(int n) { int v = 1; while (v < n) v <<= 1; return v; }
 
 struct Layout {
   size_t off_state, off_n2, off_hist, off_sure, off_boundary, off_cand, off_kept, off_kept_pos, off_dbeta, off_dbeta64,
-      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_margin, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl,
+      off_conflict, off_cand_dbeta64, off_cand_bnew, off_dot_partial, off_dot_ticket, off_margin, off_obj, off_amb, off_xcb, off_walk_blocked, off_walk_ctl, off_walk_cols,
       off_bucket_count, off_bucket_items, off_bucket_vals, off_bucket_cols, off_resid_acc, off_delta_prev, off_edges, off_patch_keys, off_cand_keys, off_survivors, off_bin_off, off_bin_cur, off_ahead_bin_off, off_ahead_bin_cur,
       off_ahead_state, off_ahead_hist, off_ahead_sure, off_ahead_boundary, off_ahead_keys, off_ahead_idx, total;
   int cap_sure, cap_boundary, mask_words, dot_parts, cap_amb, n_ahead, cap_ahead_boundary, cap_survivors;
@@ -152,6 +152,7 @@ Layout carve(const strads_lasso_config_t* c, bool first = true) {
   const bool csc = c->layout == STRADS_CSC;                            // on-demand walk (CSC)
   L.off_walk_blocked = take(csc ? sizeof(unsigned int) * (size_t)L.mask_words : 0);
   L.off_walk_ctl = take(csc ? sizeof(WalkControl) : 0);
+  L.off_walk_cols = take(csc ? sizeof(WalkColumn) * (size_t)c->n_candidates : 0);
   // CSC Gram by row buckets: provided for while the buckets' candidate lists stay below 64 MB (N <= 2^20; their values take as much)
   L.buckets = csc && (size_t)c->n_rows * kBucketSlots * sizeof(int) <= ((size_t)64 << 20);
   L.off_bucket_count = take(L.buckets ? sizeof(unsigned int) * (size_t)c->n_rows : 0);
@@ -399,6 +400,7 @@ int pipelined_rounds(strads_lasso_s* h, long long count, cudaStream_t main) {
 void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, char* ws, int s, int S, const Problem* first) {
   p.layout = c->layout; p.N = c->n_rows; p.J = c->n_cols; p.ld = c->ld;
   p.xv = c->x_values; p.xrow = c->x_row_idx; p.xptr = reinterpret_cast<const long long*>(c->x_col_ptr);
+  p.nnz = c->layout == STRADS_CSC ? c->nnz : 0;
   p.y = c->y; p.beta = c->beta; p.resid = c->resid; p.delta = c->delta;
   p.lambda = c->lambda; p.eta = c->eta; p.rho = c->rho; p.c_init = c->c_init;
   p.n_cand = c->n_candidates; p.n_keep = c->n_keep; p.seed = c->seed; p.flags = c->flags;
@@ -433,6 +435,7 @@ void fill_problem(Problem& p, const strads_lasso_config_t* c, const Layout& L, c
   p.cand_cur = nullptr;
   p.walk_blocked = reinterpret_cast<unsigned int*>(ws + L.off_walk_blocked);
   p.walk_ctl = reinterpret_cast<WalkControl*>(ws + L.off_walk_ctl);
+  p.walk_cols = reinterpret_cast<WalkColumn*>(ws + L.off_walk_cols);
   p.resid_acc = reinterpret_cast<long long*>(ws + L.off_resid_acc);
   p.bucket_count = L.buckets ? reinterpret_cast<unsigned int*>(ws + L.off_bucket_count) : nullptr;
   p.bucket_items = L.buckets ? reinterpret_cast<int*>(ws + L.off_bucket_items) : nullptr;

@@ -56,6 +56,15 @@ struct WalkControl {            // shared by the CTAs of the cooperative on-dema
 };
 
 static constexpr int kBucketSlots = 16;   // candidates per row bucket (more: the round falls back to all pairs)
+// What the on-demand walk needs of a candidate's column, gathered once per walk (two 16-byte loads instead of a chain
+// of three accesses per merge).
+struct __align__(16) WalkColumn {
+  long long q0;     // first stored entry
+  int n;            // entries
+  int j;            // the column
+  double n2;        // its coupling_n2
+  double unused;
+};
 // What the bucket kernels need of a candidate's column, gathered once per round (one access instead of a chain of three).
 struct BucketColumn {
   long long q0;     // first stored entry
@@ -73,6 +82,7 @@ struct Problem {
   const float* xv;
   const int* xrow;
   const long long* xptr;
+  long long nnz;                // CSC: stored entries (the length of xv and xrow)
   const float* y;
   float* beta;
   float* resid;
@@ -113,6 +123,7 @@ struct Problem {
   const int* cand_cur;          // candidate list of the Gram in flight (set per launch)
   unsigned int* walk_blocked;   // CSC on-demand walk: running mask [mask_words], OR-ed into by the whole grid
   WalkControl* walk_ctl;
+  WalkColumn* walk_cols;        // ... [P'] where each candidate's column lies, gathered when the walk starts
   long long* resid_acc;         // CSC: [N] fixed-point accumulators of the residual update (zero between rounds)
   // CSC Gram by row buckets (null / 0 when not provided for)
   unsigned int* bucket_count;   // [N] candidates of this round's list with an entry in row i (zero between rounds)
@@ -347,6 +358,48 @@ __device__ __forceinline__ float sparse_dot_fetched(const int* ar, const float* 
     return dot;
   }
   return sparse_dot_arrays(ar, av, na, p.xrow + q0, p.xv + q0, nb);      // a long column: plain merge
+}
+
+// The same with column b fetched as aligned groups of four entries (16-byte loads; xv and xrow 16-byte aligned): a
+// lane that merges a column of its own touches a cache line per load, and it is the number of such loads, not their
+// size, that an SM can take per cycle.  The groups start at the aligned entry at or before q0 and cover
+// (q0 mod 4) + nb <= 4 kVec entries; those outside the column count as absent.  A group that would reach past the
+// last stored entry of the matrix is read entry by entry.
+template <int kVec>
+__device__ __forceinline__ float sparse_dot_fetched4(const int* ar, const float* av, int na, const Problem& p, long long q0, int nb) {
+  const long long e0 = q0 & ~3ll;
+  const int head = (int)(q0 - e0), need = head + nb;
+  int rb[4 * kVec];
+  float vb[4 * kVec];
+#pragma unroll
+  for (int v = 0; v < kVec; ++v) {
+    int4 r = make_int4(0, 0, 0, 0);
+    float4 x = make_float4(0.f, 0.f, 0.f, 0.f);
+    const long long e = e0 + 4 * v;
+    if (4 * v < need) {
+      if (e + 4 <= p.nnz) {
+        r = __ldg(reinterpret_cast<const int4*>(p.xrow + e));
+        x = __ldg(reinterpret_cast<const float4*>(p.xv + e));
+      } else {
+        if (e < p.nnz) { r.x = __ldg(p.xrow + e); x.x = __ldg(p.xv + e); }
+        if (e + 1 < p.nnz) { r.y = __ldg(p.xrow + e + 1); x.y = __ldg(p.xv + e + 1); }
+        if (e + 2 < p.nnz) { r.z = __ldg(p.xrow + e + 2); x.z = __ldg(p.xv + e + 2); }
+      }
+    }
+    const int i0 = 4 * v;
+    rb[i0] = (i0 >= head && i0 < need) ? r.x : 0x7fffffff;             vb[i0] = x.x;
+    rb[i0 + 1] = (i0 + 1 >= head && i0 + 1 < need) ? r.y : 0x7fffffff; vb[i0 + 1] = x.y;
+    rb[i0 + 2] = (i0 + 2 >= head && i0 + 2 < need) ? r.z : 0x7fffffff; vb[i0 + 2] = x.z;
+    rb[i0 + 3] = (i0 + 3 >= head && i0 + 3 < need) ? r.w : 0x7fffffff; vb[i0 + 3] = x.w;
+  }
+  float dot = 0.f;
+  for (int i = 0; i < na; ++i) {
+    const int ra = ar[i];
+    const float va = av[i];
+#pragma unroll
+    for (int k = 0; k < 4 * kVec; ++k) dot = rb[k] == ra ? fmaf(va, vb[k], dot) : dot;
+  }
+  return dot;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -41,6 +41,15 @@ __device__ __forceinline__ int nth_set_bit(unsigned int x, int n) {
   return at;
 }
 
+// (written by other SMs earlier in the same launch: read past L1)
+__device__ __forceinline__ WalkColumn load_walk_column(const WalkColumn* at) {
+  const longlong2 a = __ldcg(reinterpret_cast<const longlong2*>(at));
+  const double2 b = __ldcg(reinterpret_cast<const double2*>(at) + 1);
+  WalkColumn col;
+  col.q0 = a.x; col.n = (int)(a.y & 0xffffffffll); col.j = (int)(a.y >> 32); col.n2 = b.x; col.unused = 0.0;
+  return col;
+}
+
 // Grid-wide barrier.  Returns false when the wait gave up (or an earlier one did).
 __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* status, unsigned int limit) {
   __shared__ int s_ok;
@@ -92,50 +101,59 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
   const unsigned int full = 0xffffffffu;
   unsigned int* blocked_g = p.walk_blocked;
   const double rho = (double)p.rho;
+  const bool rows_aligned = (reinterpret_cast<unsigned long long>(p.xrow) & 15ull) == 0ull;   // (xv always is)
 
   for (int w = tid; w < W; w += kThreads) blocked[w] = 0u;
   if (blockIdx.x == 0)
     for (int w = tid; w < W; w += kThreads) blocked_g[w] = 0u;
+  // where every candidate's column lies, gathered by the whole grid once (the first barrier publishes it): a merge
+  // of step D then finds its column in one access instead of three dependent ones
+  for (int a = (int)(blockIdx.x * kThreads) + tid; a < n_cand; a += (int)(n_ctas * kThreads)) {
+    WalkColumn col;
+    col.j = cand[a];
+    col.q0 = p.xptr[col.j];
+    col.n = (int)(p.xptr[col.j + 1] - col.q0);
+    col.n2 = coupling_n2(p, col.j);
+    col.unused = 0.0;
+    p.walk_cols[a] = col;
+  }
   if (tid == 0) { s_cursor = 0; s_kept = 0; s_examined = n_cand; s_done = 0; }
   bool ok = grid_barrier(c, n_ctas, &p.st->status, spin_limit);       // nobody ORs into the global mask before it is cleared
 
   while (ok) {
-    // ---- A: the next <= 32 candidates at or after the cursor that are not blocked (warp 0) ----
-    if (tid < 32) {
-      int m = 0;
-      int cur = s_cursor;
-      while (cur < n_cand && m < kBatch) {
-        const int wbase = (cur >> 5) + lane;           // 32 mask words at a time, one per lane
-        unsigned int freew = 0u;
-        if (wbase < W) {
-          freew = ~blocked[wbase];
-          const int first = wbase << 5;
-          if (first < cur) freew &= full << (cur - first);                                  // only lane 0 can be cut
-          if (first + 32 > n_cand) freew &= first >= n_cand ? 0u : (full >> (first + 32 - n_cand));
-        }
-        const int cnt = __popc(freew);
-        int incl = cnt;
+    // ---- A: the next <= 32 candidates at or after the cursor that are not blocked: every thread counts the free
+    //      positions of two mask words, a scan over the CTA numbers them, and the first 32 are the batch (late batches
+    //      find theirs thousands of positions further on: one warp scanning 1,024 positions per trip took 4 us) ----
+    {
+      const int cur = s_cursor;
+      auto free_from = [&](int w) {                      // unblocked candidates of mask word w at or behind the cursor
+        if (w >= W) return 0u;
+        unsigned int f = ~blocked[w];
+        const int first = w << 5;
+        if (first + 32 <= cur) f = 0u;
+        else if (first < cur) f &= full << (cur - first);                                   // (a shift of 1 .. 31)
+        if (first + 32 > n_cand) f &= first >= n_cand ? 0u : (full >> (first + 32 - n_cand));
+        return f;
+      };
+      unsigned int f0 = free_from(2 * tid), f1 = free_from(2 * tid + 1);
+      const int c0 = __popc(f0), c1 = __popc(f1);
+      int incl = c0 + c1;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(full, incl, o);
-          if (lane >= o) incl += v;
-        }
-        const int total = __shfl_sync(full, incl, 31);
-        // slot `lane` of the batch takes the (lane - m)-th free position of these 32 words
-        const int want = lane - m;
-        int wi = 0;                                    // first lane whose inclusive count exceeds `want`
-#pragma unroll
-        for (int step = 16; step > 0; step >>= 1)
-          if (__shfl_sync(full, incl, wi + step - 1) <= want) wi += step;
-        wi = min(wi, 31);
-        const int ex = __shfl_sync(full, incl - cnt, wi);
-        const unsigned int word = __shfl_sync(full, freew, wi);
-        if (want >= 0 && want < total) s_pos[lane] = (((cur >> 5) + wi) << 5) + nth_set_bit(word, want - ex);
-        m = min(kBatch, m + total);
-        if (m < kBatch) cur = ((cur >> 5) + 32) << 5;  // all 32 words consumed
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(full, incl, o);
+        if (lane >= o) incl += v;
       }
-      if (lane == 0) s_m = m;
-      s_conf[lane] = 0u;
+      if (lane == 31) s_wsum[warp] = incl;
+      __syncthreads();
+      int before = 0, total = 0;
+#pragma unroll
+      for (int k = 0; k < kThreads / 32; ++k) { const int v = s_wsum[k]; if (k < warp) before += v; total += v; }
+      int idx = before + incl - c0 - c1;
+      for (; f0 != 0u && idx < kBatch; f0 &= f0 - 1u, ++idx) s_pos[idx] = ((2 * tid) << 5) + __ffs((int)f0) - 1;
+      idx = before + incl - c1;
+      for (; f1 != 0u && idx < kBatch; f1 &= f1 - 1u, ++idx) s_pos[idx] = ((2 * tid + 1) << 5) + __ffs((int)f1) - 1;
+      if (tid == 0) s_m = min(kBatch, total);
+      if (tid < 32) s_conf[tid] = 0u;
     }
     __syncthreads();
     const int m = s_m;
@@ -144,9 +162,8 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
     // ---- B: stage the members' columns, all at once (a thread per member finds the column, then eight threads per
     //      member copy it: three memory round trips for the whole batch), then the pairs among them ----
     if (tid < m) {
-      const int j = cand[s_pos[tid]];
-      const long long a0 = p.xptr[j];
-      s_col[tid] = j; s_ptr[tid] = a0; s_len[tid] = (int)(p.xptr[j + 1] - a0); s_n2[tid] = coupling_n2(p, j);
+      const WalkColumn col = load_walk_column(p.walk_cols + s_pos[tid]);
+      s_col[tid] = col.j; s_ptr[tid] = col.q0; s_len[tid] = col.n; s_n2[tid] = col.n2;
     }
     __syncthreads();
     {
@@ -186,8 +203,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
               const bool on = ii[u] < nas[u] && kk[u] < nbs[u];
               const int i = on ? ii[u] : 0, k = on ? kk[u] : 0;
               const int ra = brow[qas[u]][i], rb = brow[qbs[u]][k];
-              const float pa = bval[qas[u]][i], pb = bval[qbs[u]][k];
-              dots[u] = (on && ra == rb) ? fmaf(pa, pb, dots[u]) : dots[u];
+              if (on && ra == rb) dots[u] = fmaf(bval[qas[u]][i], bval[qbs[u]][k], dots[u]);   // (the values only then)
               ii[u] += (on && ra <= rb) ? 1 : 0;
               kk[u] += (on && rb <= ra) ? 1 : 0;
               any = any || on;
@@ -293,14 +309,20 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
         const int b = (lo << 5) + nth_set_bit(free_word(lo), u - s_pref[lo]);
         const int q = nth_set_bit(keep, k);
         if (s_pos[q] >= b) continue;                     // the member comes later in the list: it cannot block b
-        const int jb = cand[b];
-        const long long q0 = p.xptr[jb];
-        const int nb = (int)(p.xptr[jb + 1] - q0);
-        const double den = sqrt(s_n2[q] * coupling_n2(p, jb));
+        const WalkColumn cb = load_walk_column(p.walk_cols + b);
+        const long long q0 = cb.q0;
+        const int nb = cb.n;
+        const double den = sqrt(s_n2[q] * cb.n2);
         const int na = s_len[q];
         const int* ar = na <= kColCap ? brow[q] : p.xrow + s_ptr[q];
         const float* av = na <= kColCap ? bval[q] : p.xv + s_ptr[q];
-        const float dot = nb <= 24 ? sparse_dot_fetched<24>(ar, av, na, p, q0, nb) : sparse_dot_fetched<32>(ar, av, na, p, q0, nb);
+        float dot;
+        const int need = (int)(q0 & 3) + nb;               // entries of the aligned groups of four that hold column b
+        if (!rows_aligned) dot = nb <= 24 ? sparse_dot_fetched<24>(ar, av, na, p, q0, nb) : sparse_dot_fetched<32>(ar, av, na, p, q0, nb);
+        else if (need <= 20) dot = sparse_dot_fetched4<5>(ar, av, na, p, q0, nb);
+        else if (need <= 28) dot = sparse_dot_fetched4<7>(ar, av, na, p, q0, nb);
+        else if (need <= 36) dot = sparse_dot_fetched4<9>(ar, av, na, p, q0, nb);
+        else dot = sparse_dot_arrays(ar, av, na, p.xrow + q0, p.xv + q0, nb);
         if (den > 0.0 && fabs((double)dot) >= rho * den) atomicOr(&blocked_g[b >> 5], 1u << (b & 31));
       }
     }
