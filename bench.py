@@ -43,6 +43,8 @@ NCU_TRAFFIC = {
     # profiles/ncu_k_gram_dense_tc_window_c3_J20000.md: 25.75 MB read + 0 written per launch (captured with J cut to 20,000;
     # the kernel reads the window's BF16 copies only, so its traffic does not depend on J) = the algorithmic 2 N W
     ("c3", "k_gram_dense_tc<screen>"): 25.75e6,
+    # profiles/ncu_full_round_kernels_c4.md: 6.82 MB read per launch (the buckets of the window candidates' rows)
+    ("c4", "k_csc_bucket_dots"): 6.82e6,
     # k_walk_csc spins on a grid barrier: no multi-pass capture of it is made (one-pass launch list only)
 }
 
@@ -245,7 +247,8 @@ def rooflines(p: wl.LassoProblem, workload: str, step_ms: dict, kept_per_round: 
             "frac": achieved / peak, "traffic": NCU_TRAFFIC.get((workload, kernel)), "window": window, "launch_ms": ms,
             "algorithmic_ops_per_launch": ops,
             "peak_source": "148 SMs x 128 lanes x max SM clock: one merge step (compare + advance) per lane per cycle",
-            "note": "sorted-list merges over a few MB of columns: bound by dependent loads and grid barriers, not by HBM"}
+            "note": "inner products of sparse columns counted as sorted-list merge steps, over a few MB of columns: bound by "
+                    "dependent loads and barriers, not by HBM"}
         upd_bytes = 8.0 * nnz_col * kept_per_round + 8.0 * p.n_rows
         pack_bytes = 0.0
         ns_bytes = 8.0 * nnz_col * (p.n_candidates + kept_per_round) + 8.0 * p.n_rows
