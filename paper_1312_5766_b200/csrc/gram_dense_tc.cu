@@ -702,8 +702,11 @@ __global__ void __launch_bounds__(256) k_gram_recheck(Problem p, int only_if_sho
 }  // namespace
 
 // Clusters of up to kMaxSplit CTAs share a tile; how many clusters of each size the device can hold at once
-// (one CTA per SM: the ring takes nearly all of its shared memory) decides the split of a launch.
-constexpr int kMaxSplit = 16;
+// (one CTA per SM: the ring takes nearly all of its shared memory) decides the split of a launch.  Eight, the
+// portable limit: clusters of 9 to 16 (which the device accepts on request) fill more SMs and shorten the kernel
+// when it runs alone (c2's window 22 -> 19 us), but the round as replayed, with the draw of the next round on a stream
+// beside it, measured slower with them (c3: 68.4 us per round with clusters of 9, 65.9 with 8; c2 39.1 / 38.2).
+constexpr int kMaxSplit = 8;
 static int g_max_clusters[kMaxSplit + 1];     // [size]; 0: size not available
 
 cudaError_t prepare_gram_dense_tc() {
@@ -711,11 +714,8 @@ cudaError_t prepare_gram_dense_tc() {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(k_gram_dense_tc<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDynSmem);
   if (e != cudaSuccess) return e;
-  const bool beyond8 = cudaFuncSetAttribute(k_gram_dense_tc<false>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
-  cudaGetLastError();
   for (int size = 2; size <= kMaxSplit; ++size) {
     g_max_clusters[size] = 0;
-    if (size > 8 && !beyond8) continue;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)size; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;

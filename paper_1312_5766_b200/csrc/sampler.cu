@@ -105,6 +105,29 @@ __device__ __forceinline__ void queue_keys_of_groups(const Problem& p, unsigned 
   const int lane = threadIdx.x & 31;
   const long long g = g0 + lane;
   const int mode = weight_mode_of(p.flags);
+  if (p.part_count <= 1 && (g0 + 32) * 4 <= p.J) {
+    // The common case, kept lean because the pass is bound by instruction issue (about 300 instructions per lane
+    // and call before, a third of them Philox): one scheduler and all 32 blocks of the warp whole, so no bounds or
+    // ownership tests; and since survivors are rare (a fraction of a percent of the coefficients), one vote tells
+    // the warp whether there is anything to queue at all -- the four ballots with their ranks run only then.
+    uint32_t w[4];
+    philox4x32_10((uint32_t)g, (uint32_t)t, (uint32_t)(t >> 32), 0u, (uint32_t)p.seed, (uint32_t)(p.seed >> 32), w);
+    const float4 v = __ldg(reinterpret_cast<const float4*>(p.delta) + g);
+    const float d[4] = {v.x, v.y, v.z, v.w};
+    bool in[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) in[i] = !key_surely_above(cut, d[i], p.eta, w[i], mode);
+    if (!__any_sync(0xffffffffu, in[0] | in[1] | in[2] | in[3])) return;
+    const uint32_t j0 = (uint32_t)g * 4u;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const unsigned int mask = __ballot_sync(0xffffffffu, in[i]);
+      if (in[i]) q.slots[q.n + __popc(mask & ((1u << lane) - 1u))] = make_uint2(j0 + i, w[i]);
+      q.n += __popc(mask);
+    }
+    if (q.n > kQueue - 128) drain_keys(p, q, f);
+    return;
+  }
   uint32_t w[4] = {0u, 0u, 0u, 0u};
   float d[4] = {0.f, 0.f, 0.f, 0.f};
   const long long j0 = g * 4;
