@@ -712,3 +712,55 @@ def test_csc_residual_update_is_exact_to_fp32_rounding(name):
         assert np.all(np.abs(got.astype(np.float64) - want.astype(np.float64)) <= ulp)
         assert np.mean(got != want) < 1e-3                  # (ties of the last bit only)
     assert s.status() == (0, 0)
+
+
+# --------------------------------------------------------------------------------------------------
+# The walk from the list of conflicting pairs settles first-fit in passes, one per link of the longest chain of
+# decisions that depend on each other, and hands over to the walk over the bit rows past 24 passes.  Columns
+# c_k = (z_k + z_{k+1}) / sqrt(2) with orthonormal z make such chains: neighbours correlate at 0.5, everybody else at
+# 0.  In list order k = 0, 1, 2, ... every decision waits for the one before it (one chain as long as the list: the
+# hand-over); in random order the chains are short; blocks of a few neighbours give chains of every length below the
+# limit.  Every case must give the oracle's kept list, stop at P included.
+# --------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("n_links,n_keep", [(200, 200), (200, 37), (700, 512)])
+def test_walk_settles_chains_of_dependent_decisions(n_links, n_keep):
+    b = _binding()
+    rng = np.random.default_rng(31)
+    n_rows = ((n_links + 1 + 63) // 64) * 64
+    z, _ = np.linalg.qr(rng.normal(size=(n_rows, n_links + 1)))
+    cols = ((z[:, :-1] + z[:, 1:]) / np.sqrt(2.0)).T.astype(np.float32)          # [J, N]: row k is column c_k
+    y = torch.from_numpy(rng.normal(size=n_rows).astype(np.float32))
+    J = n_links
+    s = b.StradsLasso(wl.DENSE, n_rows, J, torch.from_numpy(cols).contiguous().cuda(), y.cuda(), 0.01, 1e-6, 0.1, J, n_keep, seed=3)
+    X = oracle.Matrix.dense(cols, n_rows=n_rows)
+    n2 = oracle.colnorm2(X)
+    rho = float(np.float32(0.1))
+    # blocks of 2 .. 30 consecutive links, the blocks shuffled: chains of every length up to the pass limit and past it
+    blocks, at = [], 0
+    while at < J:
+        n = int(rng.integers(2, 31))
+        blocks.append(np.arange(at, min(at + n, J)))
+        at += n
+    orders = {
+        "in_order": np.arange(J),
+        "reversed": np.arange(J)[::-1].copy(),
+        "random": rng.permutation(J),
+        "blocks": np.concatenate([blocks[i] for i in rng.permutation(len(blocks))]),
+    }
+    for name, order in orders.items():
+        cand = order.astype(np.int32)[:J]
+        kept_d, counts_d = s.filter(torch.from_numpy(cand).cuda())
+        c = counts_d.cpu().numpy(); nk = int(c[2])
+        want = _assert_kept_matches(X, n2, cand, n_keep, rho, kept_d.cpu().numpy()[:nk], int(c[1]))
+        assert nk == len(want) and (nk == n_keep or int(c[1]) == J), name
+        if name == "in_order" and n_keep >= J:
+            assert nk == (J + 1) // 2                       # every other link
+    assert s.status()[0] == 0
+    # whole rounds (candidate window, walk by the Gram kernel's last CTA, retry) against rounds one by one
+    a, ref = (b.StradsLasso(wl.DENSE, n_rows, J, torch.from_numpy(cols).contiguous().cuda(), y.cuda(), 0.01, 1e-6, 0.1,
+                            J, min(n_keep, J // 4), seed=3) for _ in range(2))
+    a.run(12)
+    for _ in range(12):
+        ref.round()
+    for u, v in ((a.beta, ref.beta), (a.resid, ref.resid), (a.delta, ref.delta)):
+        assert torch.equal(u, v)
