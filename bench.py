@@ -312,7 +312,8 @@ def measure(workload: str, args, device, rank: int, world: int, dist_ok: bool, p
 
     # ---- device-resident timing: REPEATS regions of K rounds after the warm-up ------------------------------
     s.run(args.warmup)
-    s.run(1 + GRAPH_ROUNDS)                # whatever W is: the captured launch sequences have run before the clock starts
+    s.run(GRAPH_ROUNDS + 7)                # whatever W is: every captured launch sequence (8 rounds, and 4, 2, 1 for what is
+                                           # left over: 8 + 8 + 4 + 2 + 1 here) has run before the clock starts
     tot0 = s.totals()
     evs = [torch.cuda.Event(enable_timing=True) for _ in range(REPEATS + 1)]
     barrier()

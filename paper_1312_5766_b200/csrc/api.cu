@@ -35,8 +35,9 @@ struct strads_lasso_s {
   cudaStream_t capture_stream;
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
-  cudaGraph_t tail_graph;    // sampling ahead: one round from an early list, for what is left over of the sequences
-  cudaGraphExec_t tail_exec;
+  // sampling ahead: shorter sequences from an early list (4, 2 and 1 rounds), for what is left over of the long ones
+  cudaGraph_t tail_graph[3];
+  cudaGraphExec_t tail_exec[3];
   cudaEvent_t fork;          // S > 1: where the schedulers' streams join the caller's stream
   // Sampling ahead (one scheduler; strads_run only): the draw of round t + 1 runs on its own stream beside the Gram
   // and walk of round t, and the round then starts from that list corrected for round t's update.
@@ -64,6 +65,10 @@ namespace {
 constexpr int kProfEvents = 6;   // per round: start, after sample, pack, Gram, walk, update
 constexpr int kGraphTurns = 16;  // S > 1: turns of every scheduler in the captured sequence
 constexpr int kGraphRoundsAhead = 8;  // one scheduler, sampling ahead: rounds in the captured sequence
+constexpr int kTailKinds = 3;         // and in the shorter ones for what is left over: 4, 2, 1 (a run of 20 rounds: 8 + 8 + 4)
+constexpr int tail_rounds(int kind) { return kGraphRoundsAhead >> (kind + 1); }
+static_assert(tail_rounds(kTailKinds - 1) == 1, "the shortest left-over sequence is one round");
+static_assert(sizeof(strads_lasso_s::tail_exec) / sizeof(cudaGraphExec_t) == kTailKinds, "one slot per left-over sequence");
 constexpr int kEdgeCap = 8192;        // conflicting pairs the Gram kernels can list for the walk (32 KB)
 constexpr int kAheadMaxKeep = 4096;   // sampling ahead: the patch kernel holds 2 P keys in shared memory
 
@@ -498,8 +503,10 @@ void release(strads_lasso_s* h) {
   if (h->copy_done != nullptr) cudaEventDestroy(h->copy_done);
   if (h->round_exec != nullptr) cudaGraphExecDestroy(h->round_exec);
   if (h->round_graph != nullptr) cudaGraphDestroy(h->round_graph);
-  if (h->tail_exec != nullptr) cudaGraphExecDestroy(h->tail_exec);
-  if (h->tail_graph != nullptr) cudaGraphDestroy(h->tail_graph);
+  for (int k = 0; k < kTailKinds; ++k) {
+    if (h->tail_exec[k] != nullptr) cudaGraphExecDestroy(h->tail_exec[k]);
+    if (h->tail_graph[k] != nullptr) cudaGraphDestroy(h->tail_graph[k]);
+  }
   if (h->capture_stream != nullptr) cudaStreamDestroy(h->capture_stream);
   delete h;
 }
@@ -623,8 +630,10 @@ static long long graph_rounds(const strads_lasso_s* h) {
 
 // Captures the launch sequence of graph_rounds() rounds into a graph (on a private stream: the caller's may be
 // the legacy default stream, which cannot be captured; nothing executes during capture).  With several
-// schedulers the sequence starts with scheduler 0.  `tail`: one round from an early list instead (sampling ahead).
-static int build_round_graph(strads_lasso_s* h, bool tail = false) {
+// schedulers the sequence starts with scheduler 0.  `tail_kind` >= 0: one of the shorter sequences from an early
+// list instead (sampling ahead).
+static int build_round_graph(strads_lasso_s* h, int tail_kind = -1) {
+  const bool tail = tail_kind >= 0;
   if (h->capture_stream == nullptr) {
     int prio_least = 0, prio_greatest = 0;
     CK(cudaDeviceGetStreamPriorityRange(&prio_least, &prio_greatest));
@@ -640,12 +649,12 @@ static int build_round_graph(strads_lasso_s* h, bool tail = false) {
     if (h->n_sched > 1) {
       rc = pipelined_rounds(h, graph_rounds(h), h->capture_stream);
     } else if (h->ahead_ok) {
-      const long long n = tail ? 1 : graph_rounds(h);
+      const long long n = tail ? tail_rounds(tail_kind) : graph_rounds(h);
       for (long long i = 0; i < n && rc == STRADS_OK; ++i) rc = round_sampling_ahead(h, true, h->capture_stream);
     } else {
       rc = one_round(h, nullptr);
     }
-    e = cudaStreamEndCapture(h->capture_stream, tail ? &h->tail_graph : &h->round_graph);
+    e = cudaStreamEndCapture(h->capture_stream, tail ? &h->tail_graph[tail_kind] : &h->round_graph);
     h->ahead_round = ahead_before;
   }
   h->stream = user;
@@ -653,8 +662,8 @@ static int build_round_graph(strads_lasso_s* h, bool tail = false) {
   if (rc) return rc;
   if (e != cudaSuccess) return cuda_fail(e, "stream capture of a round");
   // instantiated and uploaded now, so that the first launch does not pay for either
-  cudaGraphExec_t* exec = tail ? &h->tail_exec : &h->round_exec;
-  CK(cudaGraphInstantiate(exec, tail ? h->tail_graph : h->round_graph, 0));
+  cudaGraphExec_t* exec = tail ? &h->tail_exec[tail_kind] : &h->round_exec;
+  CK(cudaGraphInstantiate(exec, tail ? h->tail_graph[tail_kind] : h->round_graph, 0));
   CK(cudaGraphUpload(*exec, user));
   return STRADS_OK;
 }
@@ -689,8 +698,9 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
     const int rc = build_round_graph(h);
     if (rc) return rc;
   }
-  if (use_graph && h->ahead_ok && h->tail_exec == nullptr) {
-    const int rc = build_round_graph(h, true);
+  for (int k = 0; use_graph && h->ahead_ok && k < kTailKinds; ++k) {
+    if (h->tail_exec[k] != nullptr) continue;
+    const int rc = build_round_graph(h, k);
     if (rc) return rc;
   }
   const long long R = graph_rounds(h);
@@ -702,10 +712,13 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
         h->round_host += R;
         h->ahead_round = h->round_host;
         i += R - 1;
-      } else if (have_list) {                          // fewer rounds left than a sequence holds: one at a time
-        CK(cudaGraphLaunch(h->tail_exec, h->stream));
-        h->round_host += 1;
+      } else if (have_list) {                          // fewer rounds left than a sequence holds: the longest shorter one
+        int k = 0;
+        while (tail_rounds(k) > n_rounds - i) ++k;     // (the last kind is one round)
+        CK(cudaGraphLaunch(h->tail_exec[k], h->stream));
+        h->round_host += tail_rounds(k);
         h->ahead_round = h->round_host;
+        i += tail_rounds(k) - 1;
       } else {                                         // first round of a run: draw now, start drawing ahead
         const int rc = round_sampling_ahead(h, false, h->stream);
         if (rc) return rc;
@@ -835,8 +848,10 @@ int strads_status(strads_handle_t h, uint32_t* bits_host_out) {
 static void drop_round_graph(strads_lasso_s* h) {
   if (h->round_exec != nullptr) { cudaGraphExecDestroy(h->round_exec); h->round_exec = nullptr; }
   if (h->round_graph != nullptr) { cudaGraphDestroy(h->round_graph); h->round_graph = nullptr; }
-  if (h->tail_exec != nullptr) { cudaGraphExecDestroy(h->tail_exec); h->tail_exec = nullptr; }
-  if (h->tail_graph != nullptr) { cudaGraphDestroy(h->tail_graph); h->tail_graph = nullptr; }
+  for (int k = 0; k < kTailKinds; ++k) {
+    if (h->tail_exec[k] != nullptr) { cudaGraphExecDestroy(h->tail_exec[k]); h->tail_exec[k] = nullptr; }
+    if (h->tail_graph[k] != nullptr) { cudaGraphDestroy(h->tail_graph[k]); h->tail_graph[k] = nullptr; }
+  }
 }
 
 int strads_set_wait_limit(strads_handle_t h, uint32_t iterations) {

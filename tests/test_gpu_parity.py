@@ -571,7 +571,8 @@ def test_sampling_ahead_equals_round_by_round(name, cfg_over, flags):
             assert torch.equal(x, y), (name, done)
 
     # runs of several lengths; between them calls that leave the early list stale or unusable
-    for step in (3, 1, 40, "round", 2, "filter", 25, "set_round", 30, "round_host", 12):
+    # (strads_run replays sequences of 8 rounds and, for what is left over, of 4, 2 and 1: 7 = 4 + 2 + 1 from a list in place)
+    for step in (3, 1, 40, "round", 2, "filter", 25, "set_round", 30, "round_host", 12, 7):
         if step == "round":
             a.round(); n = 1
         elif step == "filter":
