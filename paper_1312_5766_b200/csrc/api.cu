@@ -625,7 +625,7 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out) {
 
 // Rounds that one launch of the captured sequence runs.
 static long long graph_rounds(const strads_lasso_s* h) {
-  return h->n_sched > 1 ? (long long)kGraphTurns * h->n_sched : (h->ahead_ok ? kGraphRoundsAhead : 1);
+  return h->n_sched > 1 ? (long long)kGraphTurns * h->n_sched : kGraphRoundsAhead;
 }
 
 // Captures the launch sequence of graph_rounds() rounds into a graph (on a private stream: the caller's may be
@@ -652,7 +652,8 @@ static int build_round_graph(strads_lasso_s* h, int tail_kind = -1) {
       const long long n = tail ? tail_rounds(tail_kind) : graph_rounds(h);
       for (long long i = 0; i < n && rc == STRADS_OK; ++i) rc = round_sampling_ahead(h, true, h->capture_stream);
     } else {
-      rc = one_round(h, nullptr);
+      const long long n = tail ? tail_rounds(tail_kind) : graph_rounds(h);
+      for (long long i = 0; i < n && rc == STRADS_OK; ++i) rc = one_round(h, nullptr);
     }
     e = cudaStreamEndCapture(h->capture_stream, tail ? &h->tail_graph[tail_kind] : &h->round_graph);
     h->ahead_round = ahead_before;
@@ -698,15 +699,16 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
     const int rc = build_round_graph(h);
     if (rc) return rc;
   }
-  for (int k = 0; use_graph && h->ahead_ok && k < kTailKinds; ++k) {
+  for (int k = 0; use_graph && k < kTailKinds; ++k) {
     if (h->tail_exec[k] != nullptr) continue;
     const int rc = build_round_graph(h, k);
     if (rc) return rc;
   }
   const long long R = graph_rounds(h);
   for (int64_t i = 0; i < n_rounds; ++i) {
-    if (use_graph && h->ahead_ok) {
-      const bool have_list = h->ahead_round == h->round_host;
+    if (use_graph) {
+      // (without sampling ahead every round draws its own list: nothing to have in place)
+      const bool have_list = !h->ahead_ok || h->ahead_round == h->round_host;
       if (have_list && n_rounds - i >= R) {            // the early list of this round is in place: captured rounds
         CK(cudaGraphLaunch(h->round_exec, h->stream));
         h->round_host += R;
@@ -723,9 +725,6 @@ int strads_run(strads_handle_t h, int64_t n_rounds) {
         const int rc = round_sampling_ahead(h, false, h->stream);
         if (rc) return rc;
       }
-    } else if (use_graph) {
-      CK(cudaGraphLaunch(h->round_exec, h->stream));
-      h->round_host += 1;
     } else {
       const int rc = one_round(h, nullptr);
       if (rc) return rc;
