@@ -248,7 +248,7 @@ int gram_and_filter(const Scheduler& sc, cudaStream_t s, const int* cand, int n_
   if (window < n_cand) {
     if (p.layout == STRADS_CSC) {
       // whole list, conflict rows formed only for the candidates the walk keeps
-      CK(launch_walk_csc(p, cand, n_cand, sc.walk_grid, true, p.kept, s));
+      CK(launch_walk_csc(p, cand, n_cand, window, sc.walk_grid, true, p.kept, s));
     } else {
       CK(launch_gram(sc, rs, cand, n_cand, n_cand, nullptr, true));
       CK(launch_filter(p, cand, n_cand, n_cand, true, p.kept, rs));

@@ -39,6 +39,7 @@ struct DeviceState {
   float t_cut;                  // sampler: cutoff for the next round's first pass (0: none), see k_sample_hist
   int sample_redo;              // sampler: the guided first pass found too few keys; the plain pass behind it runs
   int walk_streak;              // CSC: window attempts in a row that were too short (each doubles the wait for the next)
+  int window_hopeless;          // CSC: the last whole-list walk kept fewer than P, or found its P-th member behind the window
   int bucket_used;              // ... this round's Gram went through the buckets (decided once, by the first kernel)
   unsigned int surv_count;      // sampler: keys the guided first pass found below its cutoff and saved (append cursor)
   int surv_valid;               // ... they are all there (no overflow, no repeat): the collect pass reads them, not delta[J]
@@ -164,10 +165,12 @@ __device__ __forceinline__ void list_conflict(const Problem& p, int a, int b) {
 
 // CSC: whether this round leaves the candidate window out and goes straight to the on-demand walk: after a
 // window that was too short, the next attempt comes 64 rounds (of this scheduler) later, and twice as late
-// after every further failure (up to 65,536).
+// after every further failure (up to 65,536); and not even then while the whole-list walk of the round before shows that
+// a window would have been too short again (a failed attempt costs the window's whole Gram: 5 ms on c5, 28 rounds' worth).
 __device__ __forceinline__ bool window_skipped(const Problem& p) {
   const DeviceState* st = p.st;
   if (!st->prefer_walk) return false;
+  if (st->window_hopeless) return true;                  // (the last round's walk says a window would have been too short again)
   const unsigned long long period = 64ull << min(max(st->walk_streak - 1, 0), 10);
   return ((st->round / (unsigned)p.part_count) & (period - 1ull)) != 0ull;
 }
@@ -470,7 +473,7 @@ cudaError_t prepare_filter(const Problem& p);
 // Walks cand[0 .. n_cand); n_total >= n_cand is the length of the whole list (n_cand < n_total: a window).
 // CSC: greedy walk that forms conflict rows only for the candidates it is about to keep (cooperative kernel).
 cudaError_t prepare_walk_csc(const Problem& p, int* grid_out);
-cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int grid, bool only_if_short, int* kept_out,
+cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int window, int grid, bool only_if_short, int* kept_out,
                             cudaStream_t s);
 // only_if_pending: the launch follows a window Gram whose last CTA walks; it does nothing unless that CTA left the
 // walk to it (DeviceState::walk_pending).

@@ -76,7 +76,7 @@ __device__ bool grid_barrier(WalkControl* c, unsigned int n_ctas, unsigned int* 
   return s_ok != 0;
 }
 
-__global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __restrict__ cand, int n_cand,
+__global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __restrict__ cand, int n_cand, int window,
                                                         int only_if_short, int* __restrict__ kept_out) {
   if (only_if_short && !p.st->window_short) return;      // uniform over the grid: nobody reaches a barrier
   // a wait that expired in an earlier launch left the barrier's counter where it was: nothing runs on this handle
@@ -339,6 +339,8 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
     if (tid == 0) {
       p.st->counts[1] = s_examined; p.st->counts[2] = nk; p.st->counts[3] = 0;
       p.st->amb_count = 0; p.st->window_short = 0; p.st->prefer_walk = 1;
+      // would a window of the first `window` candidates have done?  (window_skipped consults this in the next round)
+      p.st->window_hopeless = (nk == p.n_keep && s_examined <= window) ? 0 : 1;
       c->failed = 0;
     }
   }
@@ -358,11 +360,11 @@ cudaError_t prepare_walk_csc(const Problem& p, int* grid_out) {
   return cudaSuccess;
 }
 
-cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int grid, bool only_if_short, int* kept_out,
+cudaError_t launch_walk_csc(const Problem& p, const int* cand, int n_cand, int window, int grid, bool only_if_short, int* kept_out,
                             cudaStream_t s) {
   Problem q = p;
   int ois = only_if_short ? 1 : 0;
-  void* args[] = {&q, &cand, &n_cand, &ois, &kept_out};
+  void* args[] = {&q, &cand, &n_cand, &window, &ois, &kept_out};
   return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_walk_csc), dim3(grid), dim3(kThreads), args, 0, s);
 }
 
