@@ -170,7 +170,9 @@ int strads_round(strads_handle_t h, const strads_round_out_t* out);
  * round t's start, and round t + 1 starts from that list corrected for the coefficients round t updated
  * (they are struck and entered again with their new keys; the P' smallest remain).  The candidates are
  * exactly those of a draw made at the round's start; the state after strads_run equals that of the same
- * rounds run with strads_round, bit for bit.  Eight rounds are replayed per captured launch sequence; the
+ * rounds run with strads_round, bit for bit.  Eight rounds are replayed per captured launch sequence, and what is
+ * left over of a run as sequences of four, two and one round (with any layout and number of schedulers the rounds
+ * of a run are replayed from captured sequences; with several schedulers 16 turns of each per sequence); the
  * streams and events this needs belong to the handle (no device memory is allocated). */
 int strads_run(strads_handle_t h, int64_t n_rounds);
 

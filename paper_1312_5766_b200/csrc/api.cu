@@ -30,12 +30,12 @@ struct strads_lasso_s {
   // optional step timing: 6 events per round (start, after sample, pack, Gram, walk, update)
   cudaEvent_t* prof_events;
   long long prof_cap, prof_rounds;
-  // strads_run replays a captured launch sequence (fixed for a handle): one round with one scheduler,
+  // strads_run replays captured launch sequences (fixed for a handle): eight rounds with one scheduler,
   // kGraphTurns turns of every scheduler, pipelined, with several
   cudaStream_t capture_stream;
   cudaGraph_t round_graph;
   cudaGraphExec_t round_exec;
-  // sampling ahead: shorter sequences from an early list (4, 2 and 1 rounds), for what is left over of the long ones
+  // one scheduler: shorter sequences (4, 2 and 1 rounds; with sampling ahead, from an early list) for what is left over
   cudaGraph_t tail_graph[3];
   cudaGraphExec_t tail_exec[3];
   cudaEvent_t fork;          // S > 1: where the schedulers' streams join the caller's stream

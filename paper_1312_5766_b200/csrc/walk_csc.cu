@@ -4,7 +4,7 @@
 // candidates are kept out of 16,384 -- forming all P'(P'-1)/2 correlations first would do 100x more merges
 // than the walk consults.
 //
-// One cooperative kernel, two CTAs per SM, in batches of 32 candidates.  Every CTA holds the running
+// One cooperative kernel, one CTA per SM, in batches of 32 candidates.  Every CTA holds the running
 // `blocked` mask in shared memory and does the cheap, serial part of a batch itself, identically to all the
 // others, so that nothing has to be broadcast:
 //   A  pick the next 32 candidates that are not blocked yet;
@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(kThreads) k_walk_csc(Problem p, const int* __r
 
 }  // namespace
 
-// Largest cooperative grid (at most 2 CTAs per SM) for this device.
+// The cooperative grid for this device: one CTA per SM.
 cudaError_t prepare_walk_csc(const Problem& p, int* grid_out) {
   int per_sm = 0;
   cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_walk_csc, kThreads, 0);
